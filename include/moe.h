@@ -1,0 +1,215 @@
+/*
+ * moe.h -- C ABI of the B200 (sm_100a) hot path of the Sparsely-Gated Mixture-of-Experts layer
+ * (Shazeer et al., 2017): noisy top-k gating, dispatch, one-hidden-layer ReLU experts,
+ * gate-weighted combine, Importance / Load balancing losses, and their backward passes.
+ *
+ * Conventions, valid for every call unless a comment says otherwise
+ * -----------------------------------------------------------------
+ *  - Every pointer is a DEVICE pointer except `const moe_config*`, `moe_sizes*`,
+ *    `moe_ctx_layout*` and pointers whose name starts with `host_`.
+ *  - The caller owns every buffer (inputs, outputs, workspace, context). The library never
+ *    allocates or frees device memory, keeps no state between calls and never synchronises
+ *    the host with the device (except moe_check_status, which says so). All work is enqueued
+ *    on `stream` (a cudaStream_t passed as void*; NULL is the default stream).
+ *  - Tensors are row-major, contiguous, and start on a 16-byte boundary (256-byte for the
+ *    workspace and the context). Outputs are overwritten, not accumulated into.
+ *  - "act" tensors (x, xs, hid, ys, y, W1, b1, W2, b2 and their gradients) have the element
+ *    type moe_config.act (float or bfloat16). Gating tensors (W_g, W_noise, noise, clean,
+ *    raw_noise, gates, importance, load, losses and their gradients) are always float.
+ *    Index tensors are int32.
+ *  - Every function returns a moe_status; nothing is launched when it is not MOE_OK. Argument
+ *    and shape errors are reported, never faulted on. Nothing is printed.
+ *  - Notation: T tokens, d model width, h expert hidden width, n experts, k experts per token,
+ *    R = T*k dispatched rows. A "slot" is p = t*k + s, the s-th kept expert of token t.
+ *
+ * Hierarchical layer (Appendix B; moe_config.a > 0): a groups with top-k1, b experts per group
+ * with top-k2; n = a*b, k = k1*k2, flat expert id i*b + j, slot order primary-slot major.
+ * Every gating tensor is then its primary part followed by its secondary part:
+ *     Wg, Wnoise   : [d, a]  then [a, d, b]
+ *     noise, clean, raw_noise : [T, a] then [T, k1, b]   (secondary indexed by PRIMARY SLOT)
+ *     kth_vals, kth_idx       : [T, 2] then [T, k1, 2]
+ *     gates        : [T, k] products, then [T, k1] primary gates, then [T, k1, k2] secondary gates
+ *     topk_idx     : [T, k] flat expert ids (group = id / b, expert in group = id % b)
+ *     importance   : [a*b]
+ *     load         : [a*b] Load_H, then [a] primary Load, [a,b] per-group Load_i(X^(i)), [a] |X^(i)|
+ *     dload        : [a] d/d(primary Load), then [a,b] d/d(per-group Load)
+ * moe_query_sizes gives the element counts.
+ */
+#ifndef MOE_B200_H
+#define MOE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MOE_OK = 0,
+    MOE_ERR_INVALID_ARG = 1, /* NULL pointer, misaligned pointer, inconsistent or non-positive size */
+    MOE_ERR_UNSUPPORTED = 2, /* valid in the method but outside what this build implements          */
+    MOE_ERR_WORKSPACE = 3,   /* reserved: workspace too small (sizes are the caller's contract)     */
+    MOE_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                              */
+    MOE_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see moe_check_status)           */
+} moe_status;
+
+typedef enum { MOE_F32 = 0, MOE_BF16 = 1 } moe_dtype;
+
+#define MOE_MAX_K 8          /* k, k1, k2 and k1*k2 are at most this                 */
+#define MOE_MAX_EXPERTS 8192 /* n (flat) and a, b (hierarchical levels) are at most this */
+
+typedef struct moe_config {
+    int32_t T, d, h;            /* tokens, model width, expert hidden width                              */
+    int32_t n, k;               /* experts, experts per token (hierarchical: n = a*b, k = k1*k2)         */
+    int32_t a, k1, b, k2;       /* hierarchical levels; a = 0 selects the flat layer (k1, b, k2 ignored) */
+    int32_t act;                /* moe_dtype of the "act" tensors                                        */
+    float w_importance, w_load; /* scale factors of Eq. 7 and Eq. 11                                     */
+} moe_config;
+
+typedef struct moe_sizes {
+    int64_t R;            /* T*k                                                                    */
+    int64_t gate_cols;    /* gating columns per token: n (flat) or a + k1*b (hierarchical)          */
+    int64_t logits_elems; /* elements of noise, clean, raw_noise: T*gate_cols                       */
+    int64_t gates_elems;  /* elements of gates (and dgates): flat T*k, hierarchical T*(2k + k1)     */
+    int64_t kth_elems;    /* elements of kth_vals, kth_idx: flat 2T, hierarchical 2T(1 + k1)        */
+    int64_t wg_elems;     /* elements of Wg (and of Wnoise): flat d*n, hierarchical d*a + a*d*b     */
+    int64_t load_elems;   /* elements of load: flat n, hierarchical 2ab + 2a                        */
+    int64_t dload_elems;  /* elements of dload: flat n, hierarchical a + ab                         */
+    int64_t ws_bytes;     /* workspace every stage call accepts (the largest any stage needs)       */
+    int64_t ws_fwd_bytes; /* workspace of moe_forward                                               */
+    int64_t ws_bwd_bytes; /* workspace of moe_backward                                              */
+    int64_t ctx_bytes;    /* context written by moe_forward and read by moe_backward                */
+} moe_sizes;
+
+/* Byte offsets, inside the context of moe_forward, of the tensors it saves (same layouts as
+ * the stage calls). Lets a caller inspect intermediate results of the fused call. */
+typedef struct moe_ctx_layout {
+    int64_t topk_idx, gates, clean, raw_noise, kth_vals, kth_idx; /* moe_gate outputs     */
+    int64_t xs, perm, inv_perm, counts, offsets;                  /* moe_dispatch outputs */
+    int64_t hid, ys;                                              /* moe_expert_ffn outputs */
+    int64_t importance, load, losses;                             /* moe_losses outputs   */
+} moe_ctx_layout;
+
+/* Checks a configuration: positive sizes, 1 <= k <= min(n, MOE_MAX_K), n <= MOE_MAX_EXPERTS,
+ * rows of x / hid a multiple of 16 bytes, hierarchical fields consistent (n = a*b, k = k1*k2). */
+int32_t moe_validate(const moe_config *cfg);
+int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *host_out);
+int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *host_out);
+const char *moe_status_string(int32_t status);
+
+/* Synchronises `stream`, then reads the status word the kernels of the last call that used
+ * `ws` left there. MOE_OK, or MOE_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel
+ * gave up (its outputs are then undefined; the context stays usable). */
+int32_t moe_check_status(const void *ws, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Forward stages
+ * ------------------------------------------------------------------------------------------ */
+
+/* Noisy top-k gating (Section 2.1, Eq. 3-5):
+ *   clean = x.W_g, raw_noise = x.W_noise, H = clean + noise * softplus(raw_noise),
+ *   topk_idx = the k largest H of each token in descending order (lowest index wins ties),
+ *   gates = softmax over those k values (all other gate values are exactly 0 and not stored),
+ *   kth_vals/kth_idx[t] = value/index of the k-th and (k+1)-th largest H (the latter is
+ *   (-inf, -1) when k = n); they are what Eq. 9's kth_excluding needs.
+ * The logits that decide the routing are evaluated in single precision in one fixed order
+ * (one fused-multiply-add chain per output over ascending input feature; softplus in double
+ * rounded once; H by one fused multiply-add), so the routing is reproducible bit for bit.
+ * `noise` is an input: standard normal draws, or zeros for noiseless gating.
+ * in : x [T,d] act, Wg/Wnoise [d,n], noise [T,n]
+ * out: topk_idx [T,k], gates [T,k], clean [T,n], raw_noise [T,n], kth_vals [T,2], kth_idx [T,2] */
+int32_t moe_gate(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
+                 int32_t *topk_idx, float *gates, float *clean, float *raw_noise, float *kth_vals,
+                 int32_t *kth_idx, void *ws, void *stream);
+
+/* Dispatch (Section 3.1: each expert receives the batch of the examples that selected it):
+ * stable counting sort of the slots by expert.
+ * out: counts [n]; offsets [n+1] exclusive prefix sum, offsets[n] = R; perm [R] slot of sorted
+ *      row r; inv_perm [R] sorted row of slot p; xs [R,d] act, xs[r] = x[perm[r] / k]. */
+int32_t moe_dispatch(const moe_config *cfg, const void *x, const int32_t *topk_idx, void *xs, int32_t *perm,
+                     int32_t *inv_perm, int32_t *counts, int32_t *offsets, void *ws, void *stream);
+
+/* Experts (Section 3.2, Appendix C): on the rows offsets[e] <= r < offsets[e+1],
+ *   hid = relu(xs.W1[e] + b1[e]),  ys = hid.W2[e] + b2[e],
+ * float accumulation, one rounding to the act type at hid and at ys.
+ * in : xs [R,d], offsets [n+1], W1 [n,d,h], b1 [n,h], W2 [n,h,d], b2 [n,d]   out: hid [R,h], ys [R,d] */
+int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
+                       const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws,
+                       void *stream);
+
+/* Combine (Eq. 1): y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]], float sum in slot order.
+ * `gates` is the [T,k] (product) gate tensor.   out: y [T,d] act */
+int32_t moe_combine(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm, void *y,
+                    void *stream);
+
+/* Balancing losses (Section 4, Appendix A; hierarchical: Appendix B, Eq. 13-14):
+ *   importance = batch sum of the gate vectors (Eq. 6); load_i = sum_t Phi((clean_i - thr_i) /
+ *   softplus(raw_noise_i)) with thr = (k+1)-th largest H for a kept expert, k-th otherwise (Eq. 9-10);
+ *   losses = { w_importance * CV^2(importance), w_load * CV^2(load) } with the population variance.
+ * out: importance [n], load [moe_sizes.load_elems], losses [2] */
+int32_t moe_losses(const moe_config *cfg, const int32_t *topk_idx, const float *gates, const float *clean,
+                   const float *raw_noise, const float *kth_vals, float *importance, float *load, float *losses,
+                   void *ws, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Backward stages (Section 2.1, "Training the Gating Network": plain back-propagation)
+ * ------------------------------------------------------------------------------------------ */
+
+/* Adjoint of Eq. 1. in: dY [T,d] act, ys, gates [T,k], inv_perm
+ * out: dgates [T,k] = <dY[t], ys[row]>,  dys [R,d] act = gates[t,s] * dY[t] */
+int32_t moe_combine_bwd(const moe_config *cfg, const void *dY, const void *ys, const float *gates,
+                        const int32_t *inv_perm, float *dgates, void *dys, void *stream);
+
+/* Back-propagation through the experts (ReLU derivative 0 at 0):
+ *   db2 = sum dys, dW2 = hid^T.dys, dz = (dys.W2^T) * [hid > 0] (rounded to act), db1 = sum dz,
+ *   dW1 = xs^T.dz, dxs = dz.W1^T; experts with no rows get zero gradients.
+ * out: dxs [R,d], dW1 [n,d,h], db1 [n,h], dW2 [n,h,d], db2 [n,d] (all act); dz lives in ws. */
+int32_t moe_expert_ffn_bwd(const moe_config *cfg, const void *xs, const void *hid, const void *dys,
+                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1,
+                           void *db1, void *dW2, void *db2, void *ws, void *stream);
+
+/* Adjoint of the dispatch copies: dX_expert[t] = sum_s dxs[inv_perm[t*k+s]].  out: [T,d] float */
+int32_t moe_dispatch_bwd(const moe_config *cfg, const void *dxs, const int32_t *inv_perm, float *dX_expert,
+                         void *stream);
+
+/* Gradient of the two losses (upstream gradient 1) w.r.t. importance and load (Eq. 7, 11):
+ *   dgates[t,s] += w_importance * dCV^2/dimportance[topk_idx[t,s]]   (in-out: the [T,k] product part)
+ *   dload[i]     = w_load * dCV^2/dload[i]                          (out: [moe_sizes.dload_elems])   */
+int32_t moe_losses_bwd(const moe_config *cfg, const float *importance, const float *load,
+                       const int32_t *topk_idx, float *dgates, float *dload, void *ws, void *stream);
+
+/* Back-propagation through the gating network: softmax over the kept slots, the normal-CDF
+ * load estimator including its threshold (another expert's noisy logit), softplus, and the two
+ * projections. dgates is d(loss)/d(gates) [T,k] product part (the other parts are scratch for
+ * the hierarchical layer); dload [n] is d(loss)/d(load).
+ * out: dWg, dWnoise (layout of Wg), dX_gate [T,d] float */
+int32_t moe_gate_bwd(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise,
+                     const float *noise, const float *clean, const float *raw_noise, const int32_t *topk_idx,
+                     const float *gates, const float *kth_vals, const int32_t *kth_idx, float *dgates,
+                     const float *dload, float *dWg, float *dWnoise, float *dX_gate,
+                     void *ws, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Fused layer
+ * ------------------------------------------------------------------------------------------ */
+
+/* gate -> dispatch -> experts -> combine -> losses. Saves what the backward needs in `ctx`
+ * (moe_sizes.ctx_bytes, layout from moe_query_ctx_layout).
+ * out: y [T,d] act, losses [2], importance [n], load [n], counts [n] */
+int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
+                    const void *W1, const void *b1, const void *W2, const void *b2, void *y, float *losses,
+                    float *importance, float *load, int32_t *counts, void *ctx, void *ws, void *stream);
+
+/* Backward of moe_forward for upstream dY plus both balancing losses with upstream gradient 1
+ * (they are added to the model's loss, Section 4).
+ * out: dX [T,d] act, dWg, dWnoise (float, layout of Wg), dW1, db1, dW2, db2 (act) */
+int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const float *Wg, const float *Wnoise,
+                     const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                     const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
+                     void *db2, void *ws, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H */

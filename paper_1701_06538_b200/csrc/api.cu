@@ -1,0 +1,562 @@
+// The C ABI (include/moe.h): argument checks, workspace carving and the order of the launches.
+#include <string.h>
+
+#include "moe_internal.cuh"
+
+using namespace moe;
+
+namespace {
+
+struct Dims {
+    int64_t T, d, h, n, k, R;
+    bool hier;
+    int64_t a, k1, b, k2;
+    int64_t gate_cols, logits, gates, kth, wg, load, dload;
+    int32_t act;
+    size_t esz;
+};
+
+int32_t check_config(const moe_config *c) {
+    if (!c) return MOE_ERR_INVALID_ARG;
+    if (c->T < 0 || c->d <= 0 || c->h <= 0 || c->n <= 0 || c->k <= 0) return MOE_ERR_INVALID_ARG;
+    if (c->act != MOE_F32 && c->act != MOE_BF16) return MOE_ERR_INVALID_ARG;
+    if (c->k > c->n || c->k > MOE_MAX_K) return MOE_ERR_INVALID_ARG;
+    const size_t esz = act_bytes(c->act);
+    if ((c->d * esz) % 16 != 0 || (c->h * esz) % 16 != 0) return MOE_ERR_INVALID_ARG;
+    if ((int64_t)c->T * c->k >= (int64_t)1 << 31) return MOE_ERR_INVALID_ARG;
+    if (c->a < 0) return MOE_ERR_INVALID_ARG;
+    if (c->a > 0) {
+        if (c->b <= 0 || c->k1 <= 0 || c->k2 <= 0) return MOE_ERR_INVALID_ARG;
+        if (c->k1 > c->a || c->k2 > c->b) return MOE_ERR_INVALID_ARG;
+        if ((int64_t)c->a * c->b != c->n || c->k1 * c->k2 != c->k) return MOE_ERR_INVALID_ARG;
+        if (c->a > MOE_MAX_EXPERTS || c->b > MOE_MAX_EXPERTS) return MOE_ERR_INVALID_ARG;
+        if ((int64_t)c->a * c->b > (int64_t)1 << 20) return MOE_ERR_INVALID_ARG;
+    } else if (c->n > MOE_MAX_EXPERTS) {
+        return MOE_ERR_INVALID_ARG;
+    }
+    if (!(c->w_importance >= 0.0f) || !(c->w_load >= 0.0f)) return MOE_ERR_INVALID_ARG;
+    return MOE_OK;
+}
+
+Dims dims_of(const moe_config *c) {
+    Dims D;
+    D.T = c->T; D.d = c->d; D.h = c->h; D.n = c->n; D.k = c->k;
+    D.R = D.T * D.k;
+    D.hier = c->a > 0;
+    D.a = c->a; D.k1 = c->k1; D.b = c->b; D.k2 = c->k2;
+    D.act = c->act;
+    D.esz = act_bytes(c->act);
+    if (D.hier) {
+        D.gate_cols = D.a + D.k1 * D.b;
+        D.gates = D.T * (2 * D.k + D.k1);
+        D.kth = 2 * D.T * (1 + D.k1);
+        D.wg = D.d * D.a + D.a * D.d * D.b;
+        D.load = 2 * D.a * D.b + 2 * D.a;
+        D.dload = D.a + D.a * D.b;
+    } else {
+        D.gate_cols = D.n;
+        D.gates = D.T * D.k;
+        D.kth = 2 * D.T;
+        D.wg = D.d * D.n;
+        D.load = D.n;
+        D.dload = D.n;
+    }
+    D.logits = D.T * D.gate_cols;
+    return D;
+}
+
+bool bad_ptr(const void *p) { return p == nullptr || !aligned16(p); }
+#define REQUIRE_PTRS(...)                                             \
+    do {                                                              \
+        const void *ps_[] = {__VA_ARGS__};                            \
+        for (size_t i_ = 0; i_ < sizeof(ps_) / sizeof(ps_[0]); ++i_)  \
+            if (bad_ptr(ps_[i_])) return MOE_ERR_INVALID_ARG;         \
+    } while (0)
+
+cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
+
+int32_t *status_word(void *ws) { return static_cast<int32_t *>(ws); }
+
+int32_t reset_status(void *ws, cudaStream_t st) {
+    MOE_CUDA(cudaMemsetAsync(ws, 0, kWsHeader, st));
+    return MOE_OK;
+}
+
+// ---------------------------------------------------------------------------- stage workspaces
+struct GateWs {
+    int32_t *idx_p, *idx_s, *perm_p, *inv_perm_p, *counts_p, *offsets_p, *scratch, *tile_prefix;
+    GateWs(Carver &cv, const Dims &D) {
+        idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
+        if (!D.hier) return;
+        idx_p = cv.take<int32_t>(D.T * D.k1);
+        idx_s = cv.take<int32_t>(D.T * D.k);
+        perm_p = cv.take<int32_t>(D.T * D.k1);
+        inv_perm_p = cv.take<int32_t>(D.T * D.k1);
+        counts_p = cv.take<int32_t>(D.a);
+        offsets_p = cv.take<int32_t>(D.a + 1);
+        scratch = cv.take<int32_t>(dispatch_ws_elems(D.T * D.k1, (int32_t)D.a));
+        tile_prefix = cv.take<int32_t>(D.a + 1);
+    }
+};
+
+struct DispatchWs {
+    int32_t *scratch;
+    DispatchWs(Carver &cv, const Dims &D) { scratch = cv.take<int32_t>(dispatch_ws_elems(D.R, (int32_t)D.n)); }
+};
+
+struct FfnWs {
+    int32_t *tile_prefix;
+    void *tc;
+    FfnWs(Carver &cv, const Dims &D, const moe_config *c) {
+        tile_prefix = cv.take<int32_t>(D.n + 1);
+        tc = tc_ffn_supported(*c) ? cv.take_bytes(tc_ffn_ws_bytes(*c)) : nullptr;
+    }
+};
+
+struct LossesWs {
+    float *scratch;
+    LossesWs(Carver &cv, const Dims &D) {
+        scratch = cv.take<float>(losses_ws_floats(D.T, (int32_t)(D.hier ? D.a : D.n)));
+    }
+};
+
+struct FfnBwdWs {
+    void *dz;
+    int32_t *tile_prefix;
+    float *colsum;
+    FfnBwdWs(Carver &cv, const Dims &D) {
+        dz = cv.take_bytes(D.R * D.h * (int64_t)D.esz);
+        tile_prefix = cv.take<int32_t>(D.n + 1);
+        colsum = cv.take<float>(colsum_ws_floats(D.R, (int32_t)D.n, (int32_t)(D.h > D.d ? D.h : D.d)));
+    }
+};
+
+struct LossesBwdWs {
+    float *dimp;
+    LossesBwdWs(Carver &cv, const Dims &D) { dimp = cv.take<float>(D.n); }
+};
+
+struct GateBwdWs {
+    float *dclean, *draw;
+    GateBwdWs(Carver &cv, const Dims &D) {
+        dclean = cv.take<float>(D.logits);
+        draw = cv.take<float>(D.logits);
+    }
+};
+
+template <typename F> int64_t measure(F f) {
+    Carver cv(nullptr);
+    cv.take_bytes(kWsHeader);
+    f(cv);
+    return (int64_t)cv.off;
+}
+
+struct Ctx {
+    int32_t *topk_idx, *kth_idx, *perm, *inv_perm, *counts, *offsets;
+    float *gates, *clean, *raw_noise, *kth_vals, *importance, *load, *losses;
+    void *xs, *hid, *ys;
+    moe_ctx_layout off;
+    Ctx(void *base, const Dims &D) {
+        Carver cv(base);
+        auto at = [&]() { return (int64_t)cv.off; };
+        off.topk_idx = at(); topk_idx = cv.take<int32_t>(D.R);
+        off.gates = at(); gates = cv.take<float>(D.gates);
+        off.clean = at(); clean = cv.take<float>(D.logits);
+        off.raw_noise = at(); raw_noise = cv.take<float>(D.logits);
+        off.kth_vals = at(); kth_vals = cv.take<float>(D.kth);
+        off.kth_idx = at(); kth_idx = cv.take<int32_t>(D.kth);
+        off.xs = at(); xs = cv.take_bytes(D.R * D.d * (int64_t)D.esz);
+        off.perm = at(); perm = cv.take<int32_t>(D.R);
+        off.inv_perm = at(); inv_perm = cv.take<int32_t>(D.R);
+        off.counts = at(); counts = cv.take<int32_t>(D.n);
+        off.offsets = at(); offsets = cv.take<int32_t>(D.n + 1);
+        off.hid = at(); hid = cv.take_bytes(D.R * D.h * (int64_t)D.esz);
+        off.ys = at(); ys = cv.take_bytes(D.R * D.d * (int64_t)D.esz);
+        off.importance = at(); importance = cv.take<float>(D.n);
+        off.load = at(); load = cv.take<float>(D.load);
+        off.losses = at(); losses = cv.take<float>(2);
+        bytes = (int64_t)cv.off;
+    }
+    int64_t bytes;
+};
+
+struct BwdWs {
+    float *dgates, *dload, *dX_gate;
+    void *dys, *dxs;
+    BwdWs(Carver &cv, const Dims &D) {
+        dgates = cv.take<float>(D.gates);
+        dload = cv.take<float>(D.dload);
+        dX_gate = cv.take<float>(D.T * D.d);
+        dys = cv.take_bytes(D.R * D.d * (int64_t)D.esz);
+        dxs = cv.take_bytes(D.R * D.d * (int64_t)D.esz);
+    }
+};
+
+// ---------------------------------------------------------------------------- stage bodies
+// (pointers already checked; `cv` positioned after the workspace header)
+
+int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *Wg, const float *Wnoise,
+                const float *noise, int32_t *topk_idx, float *gates, float *clean, float *raw_noise,
+                float *kth_vals, int32_t *kth_idx, Carver &cv, cudaStream_t st) {
+    GateWs w(cv, D);
+    if (!D.hier) {
+        MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, (int32_t)D.n, Wg, Wnoise, clean, raw_noise, nullptr,
+                                  0, nullptr, 1, nullptr, st));
+        return launch_gate_select(clean, raw_noise, noise, D.T, (int32_t)D.n, (int32_t)D.k, topk_idx, gates,
+                                  kth_vals, kth_idx, st);
+    }
+    // primary gate over the a groups
+    const int64_t P1 = D.T * D.k1;
+    float *g_p = gates + D.T * D.k, *g_s = g_p + P1;
+    MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, (int32_t)D.a, Wg, Wnoise, clean, raw_noise, nullptr, 0,
+                              nullptr, 1, nullptr, st));
+    MOE_TRY(launch_gate_select(clean, raw_noise, noise, D.T, (int32_t)D.a, (int32_t)D.k1, w.idx_p, g_p, kth_vals,
+                               kth_idx, st));
+    // secondary gates: rows (t, s1) grouped by their group so each tile uses one group's matrices
+    MOE_TRY(launch_dispatch_index(w.idx_p, P1, (int32_t)D.a, w.perm_p, w.inv_perm_p, w.counts_p, w.offsets_p,
+                                  w.scratch, st));
+    const int64_t lp = D.T * D.a;  // elements of the primary part of the logits tensors
+    MOE_TRY(launch_projection(x, D.act, P1, (int32_t)D.d, (int32_t)D.b, Wg + D.d * D.a, Wnoise + D.d * D.a,
+                              clean + lp, raw_noise + lp, w.offsets_p, (int32_t)D.a, w.perm_p, (int32_t)D.k1,
+                              w.tile_prefix, st));
+    MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s,
+                               g_s, kth_vals + 2 * D.T, kth_idx + 2 * D.T, st));
+    return launch_hier_merge(D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.b, w.idx_p, g_p, w.idx_s, g_s, topk_idx,
+                             gates, st);
+}
+
+int32_t do_dispatch(const Dims &D, const void *x, const int32_t *topk_idx, void *xs, int32_t *perm,
+                    int32_t *inv_perm, int32_t *counts, int32_t *offsets, Carver &cv, cudaStream_t st) {
+    DispatchWs w(cv, D);
+    MOE_TRY(launch_dispatch_index(topk_idx, D.R, (int32_t)D.n, perm, inv_perm, counts, offsets, w.scratch, st));
+    return launch_dispatch_rows(x, D.act, D.T, (int32_t)D.k, (int32_t)D.d, inv_perm, xs, st);
+}
+
+SimtGemm base_gemm(const Dims &D) {
+    SimtGemm g;
+    memset(&g, 0, sizeof(g));
+    g.ta = g.tb = g.tc = D.act == MOE_BF16 ? G_BF16 : G_F32;
+    g.a_row_div = 1;
+    return g;
+}
+
+int32_t do_expert_ffn(const moe_config *c, const Dims &D, const void *xs, const int32_t *offsets, const void *W1,
+                      const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws_base,
+                      Carver &cv, cudaStream_t st) {
+    FfnWs w(cv, D, c);
+    if (w.tc) return launch_tc_ffn(*c, xs, offsets, W1, b1, W2, b2, hid, ys, w.tc, status_word(ws_base), st);
+    SimtGemm g = base_gemm(D);  // hid = relu(xs.W1 + b1)
+    g.A = xs; g.B = W1; g.C = hid; g.bias = b1; g.relu = 1;
+    g.sa_i = D.d; g.sa_k = 1; g.sb_k = D.h; g.sb_j = 1; g.sc_i = D.h; g.sc_j = 1;
+    g.mode = 0; g.offsets = offsets; g.nseg = (int32_t)D.n; g.M = D.R; g.N = D.h; g.K = D.d; g.b_e = D.d * D.h;
+    MOE_TRY(launch_simt_gemm(g, w.tile_prefix, st));
+    g = base_gemm(D);  // ys = hid.W2 + b2
+    g.A = hid; g.B = W2; g.C = ys; g.bias = b2;
+    g.sa_i = D.h; g.sa_k = 1; g.sb_k = D.d; g.sb_j = 1; g.sc_i = D.d; g.sc_j = 1;
+    g.mode = 0; g.offsets = offsets; g.nseg = (int32_t)D.n; g.M = D.R; g.N = D.d; g.K = D.h; g.b_e = D.h * D.d;
+    return launch_simt_gemm(g, w.tile_prefix, st);
+}
+
+int32_t do_losses(const moe_config *c, const Dims &D, const int32_t *topk_idx, const float *gates,
+                  const float *clean, const float *raw_noise, const float *kth_vals, float *importance, float *load,
+                  float *losses, Carver &cv, cudaStream_t st) {
+    LossesWs w(cv, D);
+    if (D.hier) return MOE_ERR_UNSUPPORTED;
+    MOE_TRY(launch_level_sums(topk_idx, gates, clean, raw_noise, kth_vals, D.T, (int32_t)D.n, (int32_t)D.k,
+                              importance, load, w.scratch, st));
+    return launch_cv2(importance, (int32_t)D.n, load, (int32_t)D.n, c->w_importance, c->w_load, losses, st);
+}
+
+int32_t do_expert_ffn_bwd(const Dims &D, const void *xs, const void *hid, const void *dys, const int32_t *offsets,
+                          const void *W1, const void *W2, void *dxs, void *dW1, void *db1, void *dW2, void *db2,
+                          Carver &cv, cudaStream_t st) {
+    FfnBwdWs w(cv, D);
+    const int32_t n = (int32_t)D.n;
+    MOE_TRY(launch_segment_colsum(dys, D.act, offsets, n, D.R, (int32_t)D.d, db2, w.colsum, w.tile_prefix, st));
+    SimtGemm g = base_gemm(D);  // dW2[e] = hid_e^T . dys_e
+    g.A = hid; g.B = dys; g.C = dW2;
+    g.sa_i = 1; g.sa_k = D.h; g.sb_k = D.d; g.sb_j = 1; g.sc_i = D.d; g.sc_j = 1;
+    g.mode = 1; g.offsets = offsets; g.nseg = n; g.M = D.h; g.N = D.d; g.c_e = D.h * D.d;
+    MOE_TRY(launch_simt_gemm(g, w.tile_prefix, st));
+    g = base_gemm(D);  // dz = (dys . W2[e]^T) * [hid > 0]
+    g.A = dys; g.B = W2; g.C = w.dz; g.mask = hid;
+    g.sa_i = D.d; g.sa_k = 1; g.sb_k = 1; g.sb_j = D.d; g.sc_i = D.h; g.sc_j = 1;
+    g.mode = 0; g.offsets = offsets; g.nseg = n; g.M = D.R; g.N = D.h; g.K = D.d; g.b_e = D.h * D.d;
+    MOE_TRY(launch_simt_gemm(g, w.tile_prefix, st));
+    MOE_TRY(launch_segment_colsum(w.dz, D.act, offsets, n, D.R, (int32_t)D.h, db1, w.colsum, w.tile_prefix, st));
+    g = base_gemm(D);  // dW1[e] = xs_e^T . dz_e
+    g.A = xs; g.B = w.dz; g.C = dW1;
+    g.sa_i = 1; g.sa_k = D.d; g.sb_k = D.h; g.sb_j = 1; g.sc_i = D.h; g.sc_j = 1;
+    g.mode = 1; g.offsets = offsets; g.nseg = n; g.M = D.d; g.N = D.h; g.c_e = D.d * D.h;
+    MOE_TRY(launch_simt_gemm(g, w.tile_prefix, st));
+    g = base_gemm(D);  // dxs = dz . W1[e]^T
+    g.A = w.dz; g.B = W1; g.C = dxs;
+    g.sa_i = D.h; g.sa_k = 1; g.sb_k = 1; g.sb_j = D.h; g.sc_i = D.d; g.sc_j = 1;
+    g.mode = 0; g.offsets = offsets; g.nseg = n; g.M = D.R; g.N = D.d; g.K = D.h; g.b_e = D.d * D.h;
+    return launch_simt_gemm(g, w.tile_prefix, st);
+}
+
+int32_t do_losses_bwd(const moe_config *c, const Dims &D, const float *importance, const float *load,
+                      const int32_t *topk_idx, float *dgates, float *dload, Carver &cv, cudaStream_t st) {
+    LossesBwdWs w(cv, D);
+    if (D.hier) return MOE_ERR_UNSUPPORTED;
+    return launch_losses_bwd_flat(importance, load, (int32_t)D.n, topk_idx, D.R, c->w_importance, c->w_load, dgates,
+                                  dload, w.dimp, st);
+}
+
+// dW = x^T . dlogit [d, n];  dX (+)= dlogit . W^T [T, d]
+int32_t gate_weight_grads(const Dims &D, const void *x, const float *dlogit, const float *W, int64_t n,
+                          float *dW, float *dX, bool accumulate, cudaStream_t st) {
+    SimtGemm g;
+    memset(&g, 0, sizeof(g));
+    g.a_row_div = 1;
+    g.ta = D.act == MOE_BF16 ? G_BF16 : G_F32; g.tb = G_F32; g.tc = G_F32;
+    g.A = x; g.B = dlogit; g.C = dW;
+    g.sa_i = 1; g.sa_k = D.d; g.sb_k = n; g.sb_j = 1; g.sc_i = n; g.sc_j = 1;
+    g.mode = 1; g.offsets = nullptr; g.nseg = 1; g.M = D.d; g.N = n; g.K = D.T;
+    MOE_TRY(launch_simt_gemm(g, nullptr, st));
+    memset(&g, 0, sizeof(g));
+    g.a_row_div = 1;
+    g.ta = g.tb = g.tc = G_F32;
+    g.A = dlogit; g.B = W; g.C = dX; g.accumulate = accumulate ? 1 : 0;
+    g.sa_i = n; g.sa_k = 1; g.sb_k = 1; g.sb_j = n; g.sc_i = D.d; g.sc_j = 1;
+    g.mode = 0; g.offsets = nullptr; g.nseg = 1; g.M = D.T; g.N = D.d; g.K = n;
+    return launch_simt_gemm(g, nullptr, st);
+}
+
+int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const float *Wg, const float *Wnoise,
+                    const float *noise, const float *clean, const float *raw_noise, const int32_t *topk_idx,
+                    const float *gates, const float *kth_vals, const int32_t *kth_idx, float *dgates,
+                    const float *dload, float *dWg, float *dWnoise, float *dX_gate, Carver &cv, cudaStream_t st) {
+    GateBwdWs w(cv, D);
+    if (D.hier) return MOE_ERR_UNSUPPORTED;
+    MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates, dload,
+                                    nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, st));
+    MOE_TRY(gate_weight_grads(D, x, w.dclean, Wg, D.n, dWg, dX_gate, false, st));
+    return gate_weight_grads(D, x, w.draw, Wnoise, D.n, dWnoise, dX_gate, true, st);
+}
+
+}  // namespace
+
+// ============================================================================ exported
+extern "C" {
+
+const char *moe_status_string(int32_t s) {
+    switch (s) {
+        case MOE_OK: return "ok";
+        case MOE_ERR_INVALID_ARG: return "invalid argument";
+        case MOE_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MOE_ERR_WORKSPACE: return "workspace too small";
+        case MOE_ERR_CUDA: return "CUDA error";
+        case MOE_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int32_t moe_validate(const moe_config *cfg) { return check_config(cfg); }
+
+int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *out) {
+    MOE_TRY(check_config(cfg));
+    if (!out) return MOE_ERR_INVALID_ARG;
+    const Dims D = dims_of(cfg);
+    out->R = D.R; out->gate_cols = D.gate_cols; out->logits_elems = D.logits; out->gates_elems = D.gates;
+    out->kth_elems = D.kth; out->wg_elems = D.wg; out->load_elems = D.load; out->dload_elems = D.dload;
+    const int64_t s_gate = measure([&](Carver &cv) { GateWs w(cv, D); (void)w; });
+    const int64_t s_disp = measure([&](Carver &cv) { DispatchWs w(cv, D); (void)w; });
+    const int64_t s_ffn = measure([&](Carver &cv) { FfnWs w(cv, D, cfg); (void)w; });
+    const int64_t s_loss = measure([&](Carver &cv) { LossesWs w(cv, D); (void)w; });
+    const int64_t s_fbwd = measure([&](Carver &cv) { FfnBwdWs w(cv, D); (void)w; });
+    const int64_t s_lbwd = measure([&](Carver &cv) { LossesBwdWs w(cv, D); (void)w; });
+    const int64_t s_gbwd = measure([&](Carver &cv) { GateBwdWs w(cv, D); (void)w; });
+    int64_t fwd = s_gate;
+    if (s_disp > fwd) fwd = s_disp;
+    if (s_ffn > fwd) fwd = s_ffn;
+    if (s_loss > fwd) fwd = s_loss;
+    int64_t stage_bwd = s_fbwd;
+    if (s_lbwd > stage_bwd) stage_bwd = s_lbwd;
+    if (s_gbwd > stage_bwd) stage_bwd = s_gbwd;
+    out->ws_bytes = fwd > stage_bwd ? fwd : stage_bwd;
+    out->ws_fwd_bytes = fwd;
+    out->ws_bwd_bytes = measure([&](Carver &cv) { BwdWs w(cv, D); (void)w; }) + stage_bwd;
+    Ctx ctx(nullptr, D);
+    out->ctx_bytes = ctx.bytes;
+    return MOE_OK;
+}
+
+int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *out) {
+    MOE_TRY(check_config(cfg));
+    if (!out) return MOE_ERR_INVALID_ARG;
+    Ctx ctx(nullptr, dims_of(cfg));
+    *out = ctx.off;
+    return MOE_OK;
+}
+
+int32_t moe_check_status(const void *ws, void *stream) {
+    if (!ws) return MOE_ERR_INVALID_ARG;
+    MOE_CUDA(cudaStreamSynchronize(as_stream(stream)));
+    int32_t word = 0;
+    MOE_CUDA(cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost));
+    return word == 0 ? MOE_OK : MOE_ERR_TIMEOUT;
+}
+
+int32_t moe_gate(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
+                 int32_t *topk_idx, float *gates, float *clean, float *raw_noise, float *kth_vals,
+                 int32_t *kth_idx, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(x, Wg, Wnoise, noise, topk_idx, gates, clean, raw_noise, kth_vals, kth_idx, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    return do_gate(cfg, D, x, Wg, Wnoise, noise, topk_idx, gates, clean, raw_noise, kth_vals, kth_idx, cv,
+                   as_stream(stream));
+}
+
+int32_t moe_dispatch(const moe_config *cfg, const void *x, const int32_t *topk_idx, void *xs, int32_t *perm,
+                     int32_t *inv_perm, int32_t *counts, int32_t *offsets, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(x, topk_idx, xs, perm, inv_perm, counts, offsets, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    return do_dispatch(D, x, topk_idx, xs, perm, inv_perm, counts, offsets, cv, as_stream(stream));
+}
+
+int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
+                       const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws,
+                       void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(xs, offsets, W1, b1, W2, b2, hid, ys, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return do_expert_ffn(cfg, D, xs, offsets, W1, b1, W2, b2, hid, ys, ws, cv, as_stream(stream));
+}
+
+int32_t moe_combine(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm, void *y,
+                    void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(ys, gates, inv_perm, y);
+    return launch_combine(ys, cfg->act, gates, inv_perm, cfg->T, cfg->k, cfg->d, y, as_stream(stream));
+}
+
+int32_t moe_losses(const moe_config *cfg, const int32_t *topk_idx, const float *gates, const float *clean,
+                   const float *raw_noise, const float *kth_vals, float *importance, float *load, float *losses,
+                   void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(topk_idx, gates, clean, raw_noise, kth_vals, importance, load, losses, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    return do_losses(cfg, D, topk_idx, gates, clean, raw_noise, kth_vals, importance, load, losses, cv,
+                     as_stream(stream));
+}
+
+int32_t moe_combine_bwd(const moe_config *cfg, const void *dY, const void *ys, const float *gates,
+                        const int32_t *inv_perm, float *dgates, void *dys, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(dY, ys, gates, inv_perm, dgates, dys);
+    return launch_combine_bwd(dY, ys, cfg->act, gates, inv_perm, cfg->T, cfg->k, cfg->d, dgates, dys,
+                              as_stream(stream));
+}
+
+int32_t moe_expert_ffn_bwd(const moe_config *cfg, const void *xs, const void *hid, const void *dys,
+                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1,
+                           void *db1, void *dW2, void *db2, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return do_expert_ffn_bwd(D, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, cv, as_stream(stream));
+}
+
+int32_t moe_dispatch_bwd(const moe_config *cfg, const void *dxs, const int32_t *inv_perm, float *dX_expert,
+                         void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(dxs, inv_perm, dX_expert);
+    return launch_dispatch_bwd(dxs, cfg->act, inv_perm, cfg->T, cfg->k, cfg->d, nullptr, dX_expert, nullptr,
+                               as_stream(stream));
+}
+
+int32_t moe_losses_bwd(const moe_config *cfg, const float *importance, const float *load,
+                       const int32_t *topk_idx, float *dgates, float *dload, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(importance, load, topk_idx, dgates, dload, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    return do_losses_bwd(cfg, D, importance, load, topk_idx, dgates, dload, cv, as_stream(stream));
+}
+
+int32_t moe_gate_bwd(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise,
+                     const float *noise, const float *clean, const float *raw_noise, const int32_t *topk_idx,
+                     const float *gates, const float *kth_vals, const int32_t *kth_idx, float *dgates,
+                     const float *dload, float *dWg, float *dWnoise, float *dX_gate, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(x, Wg, Wnoise, noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates, dload, dWg,
+                 dWnoise, dX_gate, ws);
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    return do_gate_bwd(cfg, D, x, Wg, Wnoise, noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates,
+                       dload, dWg, dWnoise, dX_gate, cv, as_stream(stream));
+}
+
+int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
+                    const void *W1, const void *b1, const void *W2, const void *b2, void *y, float *losses,
+                    float *importance, float *load, int32_t *counts, void *ctx, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(x, Wg, Wnoise, noise, W1, b1, W2, b2, y, losses, importance, load, counts, ctx, ws);
+    const Dims D = dims_of(cfg);
+    cudaStream_t st = as_stream(stream);
+    Ctx C(ctx, D);
+    MOE_TRY(reset_status(ws, st));
+    auto fresh = [&]() { Carver cv(ws); cv.take_bytes(kWsHeader); return cv; };
+    { Carver cv = fresh();
+      MOE_TRY(do_gate(cfg, D, x, Wg, Wnoise, noise, C.topk_idx, C.gates, C.clean, C.raw_noise, C.kth_vals,
+                      C.kth_idx, cv, st)); }
+    { Carver cv = fresh();
+      MOE_TRY(do_dispatch(D, x, C.topk_idx, C.xs, C.perm, C.inv_perm, C.counts, C.offsets, cv, st)); }
+    { Carver cv = fresh();
+      MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st)); }
+    MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st));
+    { Carver cv = fresh();
+      MOE_TRY(do_losses(cfg, D, C.topk_idx, C.gates, C.clean, C.raw_noise, C.kth_vals, C.importance, C.load,
+                        C.losses, cv, st)); }
+    MOE_CUDA(cudaMemcpyAsync(losses, C.losses, 2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    MOE_CUDA(cudaMemcpyAsync(importance, C.importance, D.n * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    MOE_CUDA(cudaMemcpyAsync(load, C.load, D.load * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    MOE_CUDA(cudaMemcpyAsync(counts, C.counts, D.n * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    return MOE_OK;
+}
+
+int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const float *Wg, const float *Wnoise,
+                     const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                     const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
+                     void *db2, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2, ws);
+    const Dims D = dims_of(cfg);
+    cudaStream_t st = as_stream(stream);
+    Ctx C(const_cast<void *>(ctx), D);
+    MOE_TRY(reset_status(ws, st));
+    Carver base(ws);
+    base.take_bytes(kWsHeader);
+    BwdWs B(base, D);
+    auto fresh = [&]() { return base; };  // stage scratch starts after the tensors that live across stages
+    MOE_TRY(launch_combine_bwd(dY, C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dgates,
+                               B.dys, st));
+    { Carver cv = fresh();
+      MOE_TRY(do_expert_ffn_bwd(D, C.xs, C.hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, cv, st)); }
+    { Carver cv = fresh();
+      MOE_TRY(do_losses_bwd(cfg, D, C.importance, C.load, C.topk_idx, B.dgates, B.dload, cv, st)); }
+    { Carver cv = fresh();
+      MOE_TRY(do_gate_bwd(cfg, D, x, Wg, Wnoise, noise, C.clean, C.raw_noise, C.topk_idx, C.gates, C.kth_vals,
+                          C.kth_idx, B.dgates, B.dload, dWg, dWnoise, B.dX_gate, cv, st)); }
+    return launch_dispatch_bwd(B.dxs, D.act, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dX_gate, nullptr, dX,
+                               st);
+}
+
+}  // extern "C"

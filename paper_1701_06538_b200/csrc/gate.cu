@@ -1,0 +1,306 @@
+// Noisy top-k gating (Section 2.1, Eq. 3-5): projection, noisy logits, KeepTopK, masked softmax.
+#include <math_constants.h>
+
+#include "moe_internal.cuh"
+
+namespace moe {
+
+// ------------------------------------------------------------------------------------------
+// Projection  clean = x.W_g,  raw = x.W_noise   (the two products of Eq. 4)
+//
+// The routing must be reproducible bit for bit, so every output is ONE chain of fused
+// multiply-adds over the input features in ascending order, starting from +0. A register-tiled
+// SIMT kernel keeps that order by construction (each accumulator sees k = 0, 1, 2, ...); a
+// tensor-core MMA would not. The kernel is therefore bound by the FP32 pipes, not by HBM.
+//
+// Tile 128 rows x BN virtual columns (the columns of [W_g | W_noise] side by side), BK = 16,
+// 256 threads, 8 x (BN/16) accumulators per thread.
+// ------------------------------------------------------------------------------------------
+constexpr int PBM = 128;
+constexpr int PBK = 16;
+
+struct ProjArgs {
+    const void *x;
+    const float *W0, *W1;
+    float *out0, *out1;
+    const int32_t *offsets;      // grouped only
+    const int32_t *perm;         // grouped only
+    const int32_t *tile_prefix;  // grouped only
+    int64_t M;
+    int32_t d, n0, nseg, kdiv;
+};
+
+template <typename XT, int BN>
+__global__ void __launch_bounds__(256) proj_kernel(ProjArgs a) {
+    constexpr int TN = BN / 16;  // 8 or 4 columns per thread
+    __shared__ __align__(16) float As[PBK][PBM];
+    __shared__ __align__(16) float Bs[PBK][BN];
+    __shared__ int32_t row_tok[PBM];  // source token of each tile row (-1: none)
+    __shared__ int32_t row_out[PBM];  // output row of each tile row
+
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int32_t n0 = a.n0, d = a.d;
+    const int32_t ncols = 2 * n0;
+    const int32_t j0 = blockIdx.y * BN;
+
+    // which rows does this tile cover?
+    const float *W0 = a.W0, *W1 = a.W1;
+    int64_t r0, r_end;
+    if (a.offsets == nullptr) {
+        r0 = (int64_t)blockIdx.x * PBM;
+        r_end = a.M;
+    } else {
+        const int32_t b = blockIdx.x;
+        if (b >= a.tile_prefix[a.nseg]) return;
+        int lo = 0, hi = a.nseg;  // last e with tile_prefix[e] <= b
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (a.tile_prefix[mid] <= b) lo = mid; else hi = mid;
+        }
+        r0 = a.offsets[lo] + (int64_t)(b - a.tile_prefix[lo]) * PBM;
+        r_end = a.offsets[lo + 1];
+        W0 += (int64_t)lo * d * n0;
+        W1 += (int64_t)lo * d * n0;
+    }
+    if (tid < PBM) {
+        int64_t r = r0 + tid;
+        int32_t tok = -1, orow = -1;
+        if (r < r_end) {
+            if (a.perm) { orow = a.perm[r]; tok = orow / a.kdiv; }
+            else { orow = (int32_t)r; tok = (int32_t)r; }
+        }
+        row_tok[tid] = tok;
+        row_out[tid] = orow;
+    }
+    __syncthreads();
+
+    float acc[8][TN];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+
+    // global -> register staging. A: thread loads 8 consecutive k of row (tid & 127).
+    const int a_row = tid & 127, a_half = tid >> 7;
+    const int32_t a_tok = row_tok[a_row];
+    const XT *xrow = a_tok >= 0 ? reinterpret_cast<const XT *>(a.x) + (int64_t)a_tok * d : nullptr;
+    float ra[8], rb[TN];
+
+    auto load_tiles = [&](int k0) {
+        const int kb = k0 + a_half * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ra[i] = 0.0f;
+        if (xrow) {
+            if (kb + 8 <= d) {
+                if constexpr (sizeof(XT) == 2) {
+                    uint4 v = *reinterpret_cast<const uint4 *>(xrow + kb);
+                    const bf16 *h = reinterpret_cast<const bf16 *>(&v);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) ra[i] = __bfloat162float(h[i]);
+                } else {
+                    float4 v0 = *reinterpret_cast<const float4 *>(xrow + kb);
+                    float4 v1 = *reinterpret_cast<const float4 *>(xrow + kb + 4);
+                    ra[0] = v0.x; ra[1] = v0.y; ra[2] = v0.z; ra[3] = v0.w;
+                    ra[4] = v1.x; ra[5] = v1.y; ra[6] = v1.z; ra[7] = v1.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (kb + i < d) ra[i] = to_f32(xrow[kb + i]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < TN; ++i) {
+            const int e = tid + i * 256;
+            const int kk = e / BN, j = j0 + (e % BN);
+            float v = 0.0f;
+            if (k0 + kk < d && j < ncols)
+                v = j < n0 ? W0[(int64_t)(k0 + kk) * n0 + j] : W1[(int64_t)(k0 + kk) * n0 + (j - n0)];
+            rb[i] = v;
+        }
+    };
+    auto store_tiles = [&]() {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) As[a_half * 8 + i][a_row] = ra[i];
+#pragma unroll
+        for (int i = 0; i < TN; ++i) {
+            const int e = tid + i * 256;
+            Bs[e / BN][e % BN] = rb[i];
+        }
+    };
+
+    load_tiles(0);
+    for (int k0 = 0; k0 < d; k0 += PBK) {
+        store_tiles();
+        __syncthreads();
+        if (k0 + PBK < d) load_tiles(k0 + PBK);
+#pragma unroll
+        for (int kk = 0; kk < PBK; ++kk) {
+            float av[8], bv[TN];
+            *reinterpret_cast<float4 *>(&av[0]) = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
+            *reinterpret_cast<float4 *>(&av[4]) = *reinterpret_cast<const float4 *>(&As[kk][64 + ty * 4]);
+            *reinterpret_cast<float4 *>(&bv[0]) = *reinterpret_cast<const float4 *>(&Bs[kk][tx * 4]);
+            if constexpr (TN == 8)
+                *reinterpret_cast<float4 *>(&bv[4]) = *reinterpret_cast<const float4 *>(&Bs[kk][64 + tx * 4]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int lr = (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+        const int32_t orow = row_out[lr];
+        if (orow < 0) continue;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int col = j0 + (j < 4 ? tx * 4 + j : 64 + tx * 4 + (j - 4));
+            if (col < n0) a.out0[(int64_t)orow * n0 + col] = acc[i][j];
+            else if (col < ncols) a.out1[(int64_t)orow * n0 + (col - n0)] = acc[i][j];
+        }
+    }
+}
+
+int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int32_t n0, const float *W0,
+                          const float *W1, float *out0, float *out1, const int32_t *offsets, int32_t nseg,
+                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st) {
+    if (M == 0) return MOE_OK;
+    ProjArgs a;
+    a.x = x; a.W0 = W0; a.W1 = W1; a.out0 = out0; a.out1 = out1;
+    a.offsets = offsets; a.perm = perm; a.tile_prefix = tile_prefix;
+    a.M = M; a.d = d; a.n0 = n0; a.nseg = nseg; a.kdiv = kdiv;
+    int64_t tiles_m = cdiv(M, PBM);
+    if (offsets) {
+        MOE_TRY(launch_tile_prefix(offsets, nseg, PBM, tile_prefix, st));
+        tiles_m += nseg;
+    }
+    const int32_t ncols = 2 * n0;
+    const bool wide = ncols > 64;
+    dim3 grid((unsigned)tiles_m, (unsigned)cdiv(ncols, wide ? 128 : 64));
+    if (act == MOE_BF16) {
+        if (wide) proj_kernel<bf16, 128><<<grid, 256, 0, st>>>(a);
+        else proj_kernel<bf16, 64><<<grid, 256, 0, st>>>(a);
+    } else {
+        if (wide) proj_kernel<float, 128><<<grid, 256, 0, st>>>(a);
+        else proj_kernel<float, 64><<<grid, 256, 0, st>>>(a);
+    }
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Noisy logits H = clean + noise * softplus(raw) (Eq. 4), KeepTopK (Eq. 5) and the softmax over
+// the kept entries (Eq. 3). One warp per row. Each lane keeps the k+1 best of its columns in a
+// sorted register list (value descending, then index ascending); k+1 rounds of a warp arg-max
+// over the list heads then produce the global order. Lowest index wins ties everywhere.
+// softplus is evaluated in double and rounded once, H by one fused multiply-add.
+// ------------------------------------------------------------------------------------------
+constexpr int KL = MOE_MAX_K + 1;
+
+__global__ void __launch_bounds__(256) gate_select_kernel(const float *__restrict__ clean,
+                                                          const float *__restrict__ raw,
+                                                          const float *__restrict__ noise, int64_t rows, int32_t n,
+                                                          int32_t k, int32_t *__restrict__ idx,
+                                                          float *__restrict__ gates, float *__restrict__ kth_vals,
+                                                          int32_t *__restrict__ kth_idx) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    float lv[KL];
+    int32_t li[KL];
+#pragma unroll
+    for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; }
+    const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
+    for (int32_t j = lane; j < n; j += 32) {
+        const double rd = (double)r[j];
+        const float sigma = (float)(fmax(rd, 0.0) + log1p(exp(-fabs(rd))));
+        float v = fmaf(e[j], sigma, c[j]);
+        int32_t id = j;
+        bool shifting = false;
+#pragma unroll
+        for (int s = 0; s < KL; ++s) {
+            if (shifting || v > lv[s]) {
+                float tv = lv[s]; int32_t ti = li[s];
+                lv[s] = v; li[s] = id; v = tv; id = ti;
+                shifting = true;
+            }
+        }
+    }
+    const int rounds = (k < n) ? k + 1 : k;
+    float myv = -CUDART_INF_F;
+    int32_t myi = -1;
+    float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
+    int32_t i_k = -1, i_k1 = -1;
+    for (int s = 0; s < rounds; ++s) {
+        float hv = lv[0];
+        int32_t hi = li[0];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, hv, off);
+            int32_t oi = __shfl_xor_sync(0xffffffffu, hi, off);
+            if (ov > hv || (ov == hv && oi < hi)) { hv = ov; hi = oi; }
+        }
+        if (li[0] == hi) {  // this lane held the winner: pop it
+#pragma unroll
+            for (int q = 0; q < KL - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; }
+            lv[KL - 1] = -CUDART_INF_F;
+            li[KL - 1] = INT32_MAX;
+        }
+        if (s < k && lane == s) { myv = hv; myi = hi; }
+        if (s == k - 1) { v_k = hv; i_k = hi; }
+        if (s == k) { v_k1 = hv; i_k1 = hi; }
+    }
+    // softmax over the k kept logits, denominator summed in slot order
+    const float m = __shfl_sync(0xffffffffu, myv, 0);
+    const float ex = lane < k ? expf(myv - m) : 0.0f;
+    float den = 0.0f;
+    for (int s = 0; s < k; ++s) den += __shfl_sync(0xffffffffu, ex, s);
+    if (lane < k) {
+        idx[row * k + lane] = myi;
+        gates[row * k + lane] = ex / den;
+    }
+    if (lane == 0) {
+        kth_vals[row * 2 + 0] = v_k;
+        kth_vals[row * 2 + 1] = v_k1;
+        kth_idx[row * 2 + 0] = i_k;
+        kth_idx[row * 2 + 1] = i_k1;
+    }
+}
+
+int32_t launch_gate_select(const float *clean, const float *raw, const float *noise, int64_t rows, int32_t n,
+                           int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
+                           cudaStream_t st) {
+    if (rows == 0) return MOE_OK;
+    gate_select_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates,
+                                                                  kth_vals, kth_idx);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// Hierarchical gate (Eq. 12): flat expert id i*b + j and product gate, slots primary-major.
+__global__ void hier_merge_kernel(int64_t total, int32_t k1, int32_t k2, int32_t b, const int32_t *idx_p,
+                                  const float *g_p, const int32_t *idx_s, const float *g_s, int32_t *topk_idx,
+                                  float *gates) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // over T*k1*k2
+    if (i >= total) return;
+    const int64_t p1 = i / k2;  // t*k1 + s1
+    topk_idx[i] = idx_p[p1] * b + idx_s[i];
+    gates[i] = g_p[p1] * g_s[i];
+}
+
+int32_t launch_hier_merge(int64_t T, int32_t k1, int32_t k2, int32_t b, const int32_t *idx_p, const float *g_p,
+                          const int32_t *idx_s, const float *g_s, int32_t *topk_idx, float *gates,
+                          cudaStream_t st) {
+    const int64_t total = T * k1 * k2;
+    if (total == 0) return MOE_OK;
+    hier_merge_kernel<<<(unsigned)cdiv(total, 256), 256, 0, st>>>(total, k1, k2, b, idx_p, g_p, idx_s, g_s,
+                                                                    topk_idx, gates);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+}  // namespace moe

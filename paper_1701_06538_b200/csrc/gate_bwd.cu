@@ -1,0 +1,94 @@
+// Back-propagation through the gating network (Section 2.1, "Training the Gating Network"):
+// exact derivative of Eq. 3-5 and of the load estimator Eq. 9-10 w.r.t. the clean logits
+// c = x.W_g and the raw noise logits r = x.W_noise.
+#include <math_constants.h>
+
+#include "moe_internal.cuh"
+
+namespace moe {
+
+// One warp per row. With sigma = softplus(r), z = (c - thr)/sigma, q_j = dLoad_j * phi(z_j)/sigma_j:
+//   softmax over the kept slots:  dH[idx_s] += g_s (dg_s - sum_s' g_s' dg_s')
+//   load estimator:               dc_j += q_j ; dsigma_j += -z_j q_j ;
+//                                 the threshold is another entry's noisy logit:
+//                                 dH[j_(k+1)] -= sum_{kept j} q_j ; dH[j_k] -= sum_{other j} q_j
+//   H = c + eps * sigma:          dc += dH ; dsigma += eps * dH ; dr = dsigma * sigmoid(r)
+__global__ void __launch_bounds__(256) gate_logit_grads_kernel(
+    const float *__restrict__ noise, const float *__restrict__ clean, const float *__restrict__ raw,
+    const int32_t *__restrict__ idx, const float *__restrict__ gates, const float *__restrict__ kth_vals,
+    const int32_t *__restrict__ kth_idx, const float *__restrict__ dgates, const float *__restrict__ dload,
+    const int32_t *__restrict__ dload_row_group, int64_t rows, int32_t n, int32_t k, float *__restrict__ dclean,
+    float *__restrict__ draw) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    int32_t sel_idx[MOE_MAX_K];
+    float sel_dh[MOE_MAX_K];
+    float inner = 0.0f;
+#pragma unroll
+    for (int s = 0; s < MOE_MAX_K; ++s) {
+        sel_idx[s] = s < k ? idx[row * k + s] : -1;
+        if (s < k) inner = fmaf(gates[row * k + s], dgates[row * k + s], inner);
+    }
+#pragma unroll
+    for (int s = 0; s < MOE_MAX_K; ++s)
+        sel_dh[s] = s < k ? gates[row * k + s] * (dgates[row * k + s] - inner) : 0.0f;
+    const float thr_unsel = kth_vals[row * 2 + 0], thr_sel = kth_vals[row * 2 + 1];
+    const int32_t j_k = kth_idx[row * 2 + 0], j_k1 = kth_idx[row * 2 + 1];
+    const float *dl = dload + (dload_row_group ? (int64_t)dload_row_group[row] * n : 0);
+    const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
+
+    auto load_terms = [&](int32_t j, bool &sel, float &dh_soft, float &q, float &zq) {
+        sel = false;
+        dh_soft = 0.0f;
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s)
+            if (sel_idx[s] == j) { sel = true; dh_soft = sel_dh[s]; }
+        const float rj = r[j];
+        const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
+        const float z = (c[j] - (sel ? thr_sel : thr_unsel)) / sigma;
+        if (isfinite(z)) {
+            q = dl[j] * (expf(-0.5f * z * z) * 0.39894228040143267794f) / sigma;
+            zq = z * q;
+        } else {
+            q = 0.0f;
+            zq = 0.0f;
+        }
+    };
+
+    float q_sel = 0.0f, q_uns = 0.0f;
+    for (int32_t j = lane; j < n; j += 32) {
+        bool sel; float dh, q, zq;
+        load_terms(j, sel, dh, q, zq);
+        if (sel) q_sel += q; else q_uns += q;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        q_sel += __shfl_xor_sync(0xffffffffu, q_sel, off);
+        q_uns += __shfl_xor_sync(0xffffffffu, q_uns, off);
+    }
+    for (int32_t j = lane; j < n; j += 32) {
+        bool sel; float dh, q, zq;
+        load_terms(j, sel, dh, q, zq);
+        if (j == j_k1) dh -= q_sel;
+        if (j == j_k && k < n) dh -= q_uns;
+        const float rj = r[j];
+        const float dsigma = fmaf(e[j], dh, -zq);
+        dclean[row * n + j] = q + dh;
+        draw[row * n + j] = dsigma / (1.0f + expf(-rj));
+    }
+}
+
+int32_t launch_gate_logit_grads(const float *noise, const float *clean, const float *raw, const int32_t *idx,
+                                const float *gates, const float *kth_vals, const int32_t *kth_idx,
+                                const float *dgates, const float *dload, const int32_t *dload_row_group,
+                                int64_t rows, int32_t n, int32_t k, float *dclean, float *draw, cudaStream_t st) {
+    if (rows == 0) return MOE_OK;
+    gate_logit_grads_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals,
+                                                                       kth_idx, dgates, dload, dload_row_group,
+                                                                       rows, n, k, dclean, draw);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+}  // namespace moe

@@ -1,0 +1,155 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "moe.h"
+
+#define MOE_TRY(expr)                                \
+    do {                                             \
+        int32_t st_ = (expr);                        \
+        if (st_ != MOE_OK) return st_;               \
+    } while (0)
+
+#define MOE_CUDA(expr)                               \
+    do {                                             \
+        if ((expr) != cudaSuccess) return MOE_ERR_CUDA; \
+    } while (0)
+
+#define MOE_LAUNCHED()                                           \
+    do {                                                         \
+        if (cudaPeekAtLastError() != cudaSuccess) return MOE_ERR_CUDA; \
+    } while (0)
+
+namespace moe {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+static inline size_t act_bytes(int32_t act) { return act == MOE_BF16 ? 2 : 4; }
+static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline int64_t imin(int64_t a, int64_t b) { return a < b ? a : b; }
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// Carves 256-byte aligned pieces out of a workspace. With base == nullptr it only measures,
+// so the size queries and the calls that use the workspace run the same code.
+struct Carver {
+    char *base;
+    size_t off;
+    explicit Carver(void *b) : base(static_cast<char *>(b)), off(0) {}
+    template <typename T> T *take(int64_t count) {
+        size_t bytes = (static_cast<size_t>(count < 0 ? 0 : count) * sizeof(T) + 255) & ~size_t(255);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += bytes;
+        return p;
+    }
+    void *take_bytes(int64_t bytes) { return take<char>(bytes); }
+};
+
+// Every workspace begins with a 256-byte header; word 0 is the status word of bounded waits.
+static const int64_t kWsHeader = 256;
+
+// ----------------------------------------------------------------------------- gating (gate.cu)
+// Projection clean = rows.W0, raw = rows.W1 with the fixed fused-multiply-add chain.
+// Ungrouped: offsets == nullptr, rows are tokens 0..M-1, outputs [M, n0].
+// Grouped (secondary gates): sorted row r belongs to segment e (offsets[e] <= r < offsets[e+1]),
+// reads token perm[r] / kdiv, uses W0 + e*d*n0, and writes output row perm[r].
+int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int32_t n0, const float *W0,
+                          const float *W1, float *out0, float *out1, const int32_t *offsets, int32_t nseg,
+                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st);
+// Noisy logits, top-k, masked softmax for `rows` rows of n columns.
+int32_t launch_gate_select(const float *clean, const float *raw, const float *noise, int64_t rows, int32_t n,
+                           int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
+                           cudaStream_t st);
+int32_t launch_hier_merge(int64_t T, int32_t k1, int32_t k2, int32_t b, const int32_t *idx_p, const float *g_p,
+                          const int32_t *idx_s, const float *g_s, int32_t *topk_idx, float *gates,
+                          cudaStream_t st);
+
+// ----------------------------------------------------------------------------- routing (route.cu)
+int64_t dispatch_ws_elems(int64_t R, int32_t n);  // int32 elements of scratch
+int32_t launch_dispatch_index(const int32_t *topk_idx, int64_t R, int32_t n, int32_t *perm, int32_t *inv_perm,
+                              int32_t *counts, int32_t *offsets, int32_t *scratch, cudaStream_t st);
+int32_t launch_dispatch_rows(const void *x, int32_t act, int64_t T, int32_t k, int32_t d, const int32_t *inv_perm,
+                             void *xs, cudaStream_t st);
+int32_t launch_combine(const void *ys, int32_t act, const float *gates, const int32_t *inv_perm, int64_t T,
+                       int32_t k, int32_t d, void *y, cudaStream_t st);
+int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const float *gates,
+                           const int32_t *inv_perm, int64_t T, int32_t k, int32_t d, float *dgates, void *dys,
+                           cudaStream_t st);
+// out_f32 = sum_s dxs[inv_perm[t*k+s]] (+ add_f32 if given); written as float or, if out_act
+// is given instead, rounded to the act type.
+int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_perm, int64_t T, int32_t k,
+                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st);
+// tile_prefix[e] = sum_{e' < e} ceil(count_e' / bm), e = 0..n
+int32_t launch_tile_prefix(const int32_t *offsets, int32_t n, int32_t bm, int32_t *tile_prefix, cudaStream_t st);
+
+// ----------------------------------------------------------------------------- losses (losses.cu)
+int64_t losses_ws_floats(int64_t rows, int32_t n);
+// Partial column sums over rows of the gate mass (importance) and of P(x, i) (load).
+// flat / primary level: seg == nullptr. Secondary level: rows are slots p, grouped through
+// perm/offsets (sorted row r -> slot perm[r]); sums are per segment: load_out [nseg, n].
+int32_t launch_level_sums(const int32_t *idx, const float *gates, const float *clean, const float *raw,
+                          const float *kth_vals, int64_t rows, int32_t n, int32_t k, float *importance_out,
+                          float *load_out, float *scratch, cudaStream_t st);
+int32_t launch_cv2(const float *importance, int32_t n_imp, const float *load, int32_t n_load, float w_imp,
+                   float w_load, float *losses, cudaStream_t st);
+int32_t launch_losses_bwd_flat(const float *importance, const float *load, int32_t n, const int32_t *topk_idx,
+                               int64_t R, float w_imp, float w_load, float *dgates, float *dload, float *dimp_tmp,
+                               cudaStream_t st);
+
+// ----------------------------------------------------------------------------- gate backward (gate_bwd.cu)
+// dclean, draw [rows, n] from the saved gate tensors; dload_row_stride = 0 broadcasts dload [n].
+int32_t launch_gate_logit_grads(const float *noise, const float *clean, const float *raw, const int32_t *idx,
+                                const float *gates, const float *kth_vals, const int32_t *kth_idx,
+                                const float *dgates, const float *dload, const int32_t *dload_row_group,
+                                int64_t rows, int32_t n, int32_t k, float *dclean, float *draw, cudaStream_t st);
+
+// ----------------------------------------------------------------------------- SIMT grouped GEMM (gemm_simt.cu)
+enum GemmType { G_F32 = 0, G_BF16 = 1 };
+struct SimtGemm {
+    // C(i,j) = epilogue( sum_kk A(i,kk) * B(kk,j) ), element strides in elements.
+    const void *A, *B;
+    void *C;
+    int32_t ta, tb, tc;  // GemmType of A, B, C
+    int64_t sa_i, sa_k, sb_k, sb_j, sc_i, sc_j;
+    // mode 0: output rows follow the segments (M_e = count_e, K fixed); A, C advance by rows,
+    //         B by expert (b_e). mode 1: contraction over the segment rows (K_e = count_e);
+    //         A, B advance by rows (their k index), C by expert (c_e).
+    int32_t mode;
+    const int32_t *offsets;  // nullptr: a single problem of M x N x K
+    int32_t nseg;
+    int64_t M, N, K;
+    int64_t b_e, c_e;
+    const void *bias;  // [nseg, N] of type tc, or nullptr
+    int32_t relu;      // 1: max(.,0)
+    const void *mask;  // mode 0: same shape/type as C; result multiplied by [mask > 0]
+    int32_t accumulate;  // 1: C += (float C only)
+    // optional row gathers through a permutation: mode 0: A row i reads row a_row_index[i] / a_row_div
+    // and C row i is written at c_row_index[i]; mode 1: the contraction index r reads A row
+    // a_row_index[r] / a_row_div and B row b_row_index[r].
+    const int32_t *a_row_index;
+    int32_t a_row_div;
+    const int32_t *b_row_index;
+    const int32_t *c_row_index;
+};
+int32_t launch_simt_gemm(const SimtGemm &g, int32_t *tile_prefix, cudaStream_t st);
+// out[e, j] = sum over the rows of segment e of in[r, j]   (out, in of the act type)
+int64_t colsum_ws_floats(int64_t R, int32_t n, int32_t N);
+int32_t launch_segment_colsum(const void *in, int32_t act, const int32_t *offsets, int32_t nseg, int64_t R,
+                              int32_t N, void *out, float *scratch, int32_t *tile_prefix, cudaStream_t st);
+
+// ----------------------------------------------------------------------------- tensor-core experts (ffn_tc.cu)
+bool tc_ffn_supported(const moe_config &c);
+int64_t tc_ffn_ws_bytes(const moe_config &c);
+int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
+                      const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
+                      cudaStream_t st);
+
+}  // namespace moe

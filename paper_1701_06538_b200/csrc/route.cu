@@ -1,0 +1,428 @@
+// Routing: dispatch of token rows into contiguous per-expert segments (Section 3.1), the
+// gate-weighted combine (Eq. 1) and their adjoints. All of it is HBM streaming: rows are moved
+// with 16-byte vector accesses, every token row is read once and written k times (dispatch) or
+// gathered k times and written once (combine).
+#include "moe_internal.cuh"
+
+namespace moe {
+
+// ------------------------------------------------------------------------------------------
+// Stable counting sort of the slots p = 0..R-1 by expert id, with no ordering race:
+//   1. each chunk of CH consecutive slots builds a histogram              (dispatch_hist)
+//   2. per expert, exclusive scan of the chunk histograms -> chunk bases,
+//      totals -> counts                                                   (dispatch_scan_chunks)
+//   3. exclusive scan of counts -> offsets                                (dispatch_scan_experts)
+//   4. one warp per chunk walks its slots in order, 32 at a time; equal experts inside a group
+//      of 32 are ranked with match_any, across groups with a shared-memory cursor per expert
+//                                                                          (dispatch_rank)
+// Integer atomics only (order-independent results); the permutation is unique and bit-exact.
+// ------------------------------------------------------------------------------------------
+constexpr int CH = 1024;  // slots per chunk
+
+int64_t dispatch_ws_elems(int64_t R, int32_t n) { return cdiv(R, CH) * (int64_t)n + 64; }
+
+__global__ void __launch_bounds__(256) dispatch_hist_kernel(const int32_t *__restrict__ topk_idx, int64_t R,
+                                                            int32_t n, int32_t *__restrict__ chunk_hist) {
+    extern __shared__ int32_t sh[];
+    for (int e = threadIdx.x; e < n; e += blockDim.x) sh[e] = 0;
+    __syncthreads();
+    const int64_t p0 = (int64_t)blockIdx.x * CH;
+    for (int i = threadIdx.x; i < CH; i += blockDim.x) {
+        const int64_t p = p0 + i;
+        if (p < R) {
+            const int32_t e = topk_idx[p];
+            if ((uint32_t)e < (uint32_t)n) atomicAdd(&sh[e], 1);
+        }
+    }
+    __syncthreads();
+    int32_t *out = chunk_hist + (int64_t)blockIdx.x * n;
+    for (int e = threadIdx.x; e < n; e += blockDim.x) out[e] = sh[e];
+}
+
+// block = 32 experts x 32 chunk lanes; lane cl owns a contiguous run of chunks
+__global__ void __launch_bounds__(1024) dispatch_scan_chunks_kernel(int32_t *__restrict__ chunk_hist,
+                                                                    int32_t nchunks, int32_t n,
+                                                                    int32_t *__restrict__ counts) {
+    __shared__ int32_t part[32][33];
+    const int el = threadIdx.x & 31, cl = threadIdx.x >> 5;
+    const int32_t e = blockIdx.x * 32 + el;
+    const int32_t per = (nchunks + 31) / 32;
+    const int32_t c0 = cl * per, c1 = min(c0 + per, nchunks);
+    int32_t sum = 0;
+    if (e < n)
+        for (int32_t c = c0; c < c1; ++c) sum += chunk_hist[(int64_t)c * n + e];
+    part[cl][el] = sum;
+    __syncthreads();
+    if (cl == 0) {
+        int32_t run = 0;
+        for (int q = 0; q < 32; ++q) { int32_t v = part[q][el]; part[q][el] = run; run += v; }
+        if (e < n) counts[e] = run;
+    }
+    __syncthreads();
+    if (e < n) {
+        int32_t run = part[cl][el];
+        for (int32_t c = c0; c < c1; ++c) {
+            const int64_t at = (int64_t)c * n + e;
+            const int32_t v = chunk_hist[at];
+            chunk_hist[at] = run;
+            run += v;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024) dispatch_scan_experts_kernel(const int32_t *__restrict__ counts, int32_t n,
+                                                                     int32_t *__restrict__ offsets) {
+    __shared__ int32_t warp_sum[32];
+    __shared__ int32_t carry;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < n; base += 1024) {
+        const int32_t e = base + threadIdx.x;
+        const int32_t v = e < n ? counts[e] : 0;
+        int32_t inc = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            int32_t o = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += o;
+        }
+        if (lane == 31) warp_sum[w] = inc;
+        __syncthreads();
+        if (w == 0) {
+            int32_t s = warp_sum[lane], si = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                int32_t o = __shfl_up_sync(0xffffffffu, si, off);
+                if (lane >= off) si += o;
+            }
+            warp_sum[lane] = si - s;  // exclusive
+        }
+        __syncthreads();
+        const int32_t excl = carry + warp_sum[w] + inc - v;
+        if (e < n) offsets[e] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) offsets[n] = carry;
+}
+
+__global__ void __launch_bounds__(32) dispatch_rank_kernel(const int32_t *__restrict__ topk_idx, int64_t R,
+                                                           int32_t n, const int32_t *__restrict__ chunk_base,
+                                                           const int32_t *__restrict__ offsets,
+                                                           int32_t *__restrict__ perm,
+                                                           int32_t *__restrict__ inv_perm) {
+    extern __shared__ int32_t cursor[];  // next sorted row of each expert for this chunk
+    const int lane = threadIdx.x;
+    const int32_t *base = chunk_base + (int64_t)blockIdx.x * n;
+    for (int e = lane; e < n; e += 32) cursor[e] = offsets[e] + base[e];
+    __syncwarp();
+    const int64_t p0 = (int64_t)blockIdx.x * CH;
+    for (int i = 0; i < CH; i += 32) {
+        const int64_t p = p0 + i + lane;
+        const bool live = p < R;
+        int32_t e = live ? topk_idx[p] : -1;
+        if ((uint32_t)e >= (uint32_t)n) e = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        const int rank = __popc(peers & ((1u << lane) - 1u));
+        const int leader = __ffs(peers) - 1;
+        int32_t start = 0;
+        if (e >= 0 && lane == leader) {
+            start = cursor[e];
+            cursor[e] = start + __popc(peers);
+        }
+        start = __shfl_sync(0xffffffffu, start, leader);
+        if (e >= 0) {
+            const int32_t r = start + rank;
+            perm[r] = (int32_t)p;
+            inv_perm[p] = r;
+        }
+        __syncwarp();
+    }
+}
+
+int32_t launch_dispatch_index(const int32_t *topk_idx, int64_t R, int32_t n, int32_t *perm, int32_t *inv_perm,
+                              int32_t *counts, int32_t *offsets, int32_t *scratch, cudaStream_t st) {
+    const int32_t nchunks = (int32_t)cdiv(R, CH);
+    if (nchunks == 0) {
+        MOE_CUDA(cudaMemsetAsync(counts, 0, sizeof(int32_t) * n, st));
+        MOE_CUDA(cudaMemsetAsync(offsets, 0, sizeof(int32_t) * (n + 1), st));
+        return MOE_OK;
+    }
+    dispatch_hist_kernel<<<nchunks, 256, n * sizeof(int32_t), st>>>(topk_idx, R, n, scratch);
+    MOE_LAUNCHED();
+    dispatch_scan_chunks_kernel<<<(unsigned)cdiv(n, 32), 1024, 0, st>>>(scratch, nchunks, n, counts);
+    MOE_LAUNCHED();
+    dispatch_scan_experts_kernel<<<1, 1024, 0, st>>>(counts, n, offsets);
+    MOE_LAUNCHED();
+    dispatch_rank_kernel<<<nchunks, 32, n * sizeof(int32_t), st>>>(topk_idx, R, n, scratch, offsets, perm, inv_perm);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// tile_prefix[e] = number of bm-row tiles of the segments before e (tile_prefix[n] = total)
+__global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t *__restrict__ offsets, int32_t n,
+                                                           int32_t bm, int32_t *__restrict__ tile_prefix) {
+    __shared__ int32_t warp_sum[32];
+    __shared__ int32_t carry;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < n; base += 1024) {
+        const int32_t e = base + threadIdx.x;
+        const int32_t v = e < n ? (offsets[e + 1] - offsets[e] + bm - 1) / bm : 0;
+        int32_t inc = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            int32_t o = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += o;
+        }
+        if (lane == 31) warp_sum[w] = inc;
+        __syncthreads();
+        if (w == 0) {
+            int32_t s = warp_sum[lane], si = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                int32_t o = __shfl_up_sync(0xffffffffu, si, off);
+                if (lane >= off) si += o;
+            }
+            warp_sum[lane] = si - s;
+        }
+        __syncthreads();
+        const int32_t excl = carry + warp_sum[w] + inc - v;
+        if (e < n) tile_prefix[e] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) tile_prefix[n] = carry;
+}
+
+int32_t launch_tile_prefix(const int32_t *offsets, int32_t n, int32_t bm, int32_t *tile_prefix, cudaStream_t st) {
+    tile_prefix_kernel<<<1, 1024, 0, st>>>(offsets, n, bm, tile_prefix);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Row movers. VEC = one 16-byte vector (8 bf16 or 4 float). One warp per token.
+// ------------------------------------------------------------------------------------------
+template <typename XT> struct Vec16 {
+    static constexpr int N = 16 / sizeof(XT);
+    uint4 raw;
+    __device__ __forceinline__ float get(int i) const { return to_f32(reinterpret_cast<const XT *>(&raw)[i]); }
+    __device__ __forceinline__ void set(int i, float v) { reinterpret_cast<XT *>(&raw)[i] = from_f32<XT>(v); }
+};
+
+// xs[inv_perm[t*k+s]] = x[t] for every slot s: x is read once, written k times
+template <typename XT>
+__global__ void __launch_bounds__(256) dispatch_rows_kernel(const XT *__restrict__ x, int64_t T, int32_t k,
+                                                            int32_t d, const int32_t *__restrict__ inv_perm,
+                                                            XT *__restrict__ xs) {
+    constexpr int VN = 16 / sizeof(XT);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int nvec = d / VN;
+    for (int64_t t = warp; t < T; t += nwarps) {
+        int32_t rows[MOE_MAX_K];
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) rows[s] = s < k ? inv_perm[t * k + s] : 0;
+        const uint4 *src = reinterpret_cast<const uint4 *>(x + t * d);
+        for (int v = lane; v < nvec; v += 32) {
+            const uint4 val = src[v];
+#pragma unroll
+            for (int s = 0; s < MOE_MAX_K; ++s)
+                if (s < k) reinterpret_cast<uint4 *>(xs + (int64_t)rows[s] * d)[v] = val;
+        }
+    }
+}
+
+int32_t launch_dispatch_rows(const void *x, int32_t act, int64_t T, int32_t k, int32_t d, const int32_t *inv_perm,
+                             void *xs, cudaStream_t st) {
+    if (T == 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
+    if (act == MOE_BF16)
+        dispatch_rows_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)x, T, k, d, inv_perm, (bf16 *)xs);
+    else
+        dispatch_rows_kernel<float><<<grid, 256, 0, st>>>((const float *)x, T, k, d, inv_perm, (float *)xs);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]]   (Eq. 1), float sum in slot order
+template <typename XT>
+__global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys, const float *__restrict__ gates,
+                                                      const int32_t *__restrict__ inv_perm, int64_t T, int32_t k,
+                                                      int32_t d, XT *__restrict__ y) {
+    constexpr int VN = 16 / sizeof(XT);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int nvec = d / VN;
+    for (int64_t t = warp; t < T; t += nwarps) {
+        int32_t rows[MOE_MAX_K];
+        float g[MOE_MAX_K];
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) {
+            rows[s] = s < k ? inv_perm[t * k + s] : 0;
+            g[s] = s < k ? gates[t * k + s] : 0.0f;
+        }
+        for (int v = lane; v < nvec; v += 32) {
+            float acc[VN];
+#pragma unroll
+            for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
+#pragma unroll
+            for (int s = 0; s < MOE_MAX_K; ++s) {
+                if (s < k) {
+                    Vec16<XT> in;
+                    in.raw = reinterpret_cast<const uint4 *>(ys + (int64_t)rows[s] * d)[v];
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) acc[i] = fmaf(g[s], in.get(i), acc[i]);
+                }
+            }
+            Vec16<XT> out;
+#pragma unroll
+            for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
+            reinterpret_cast<uint4 *>(y + t * d)[v] = out.raw;
+        }
+    }
+}
+
+int32_t launch_combine(const void *ys, int32_t act, const float *gates, const int32_t *inv_perm, int64_t T,
+                       int32_t k, int32_t d, void *y, cudaStream_t st) {
+    if (T == 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
+    if (act == MOE_BF16)
+        combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)ys, gates, inv_perm, T, k, d, (bf16 *)y);
+    else
+        combine_kernel<float><<<grid, 256, 0, st>>>((const float *)ys, gates, inv_perm, T, k, d, (float *)y);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// dgates[t,s] = <dY[t], ys[row]>,  dys[row] = gates[t,s] * dY[t]
+template <typename XT>
+__global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__ dY, const XT *__restrict__ ys,
+                                                          const float *__restrict__ gates,
+                                                          const int32_t *__restrict__ inv_perm, int64_t T,
+                                                          int32_t k, int32_t d, float *__restrict__ dgates,
+                                                          XT *__restrict__ dys) {
+    constexpr int VN = 16 / sizeof(XT);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int nvec = d / VN;
+    for (int64_t t = warp; t < T; t += nwarps) {
+        int32_t rows[MOE_MAX_K];
+        float g[MOE_MAX_K], dot[MOE_MAX_K];
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) {
+            rows[s] = s < k ? inv_perm[t * k + s] : 0;
+            g[s] = s < k ? gates[t * k + s] : 0.0f;
+            dot[s] = 0.0f;
+        }
+        for (int v = lane; v < nvec; v += 32) {
+            Vec16<XT> dy;
+            dy.raw = reinterpret_cast<const uint4 *>(dY + t * d)[v];
+#pragma unroll
+            for (int s = 0; s < MOE_MAX_K; ++s) {
+                if (s < k) {
+                    Vec16<XT> in, out;
+                    in.raw = reinterpret_cast<const uint4 *>(ys + (int64_t)rows[s] * d)[v];
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) {
+                        dot[s] = fmaf(dy.get(i), in.get(i), dot[s]);
+                        out.set(i, g[s] * dy.get(i));
+                    }
+                    reinterpret_cast<uint4 *>(dys + (int64_t)rows[s] * d)[v] = out.raw;
+                }
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) {
+            if (s < k) {
+                float v = dot[s];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+                if (lane == 0) dgates[t * k + s] = v;
+            }
+        }
+    }
+}
+
+int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const float *gates,
+                           const int32_t *inv_perm, int64_t T, int32_t k, int32_t d, float *dgates, void *dys,
+                           cudaStream_t st) {
+    if (T == 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
+    if (act == MOE_BF16)
+        combine_bwd_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)dY, (const bf16 *)ys, gates, inv_perm, T, k,
+                                                        d, dgates, (bf16 *)dys);
+    else
+        combine_bwd_kernel<float><<<grid, 256, 0, st>>>((const float *)dY, (const float *)ys, gates, inv_perm, T,
+                                                         k, d, dgates, (float *)dys);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// out[t] = sum_s dxs[inv_perm[t*k+s]] (+ add[t]); float output, or rounded to the act type
+template <typename XT>
+__global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict__ dxs,
+                                                           const int32_t *__restrict__ inv_perm, int64_t T,
+                                                           int32_t k, int32_t d, const float *__restrict__ add,
+                                                           float *__restrict__ out_f32, XT *__restrict__ out_act) {
+    constexpr int VN = 16 / sizeof(XT);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int nvec = d / VN;
+    for (int64_t t = warp; t < T; t += nwarps) {
+        int32_t rows[MOE_MAX_K];
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) rows[s] = s < k ? inv_perm[t * k + s] : 0;
+        for (int v = lane; v < nvec; v += 32) {
+            float acc[VN];
+#pragma unroll
+            for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
+#pragma unroll
+            for (int s = 0; s < MOE_MAX_K; ++s) {
+                if (s < k) {
+                    Vec16<XT> in;
+                    in.raw = reinterpret_cast<const uint4 *>(dxs + (int64_t)rows[s] * d)[v];
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) acc[i] += in.get(i);
+                }
+            }
+            if (add) {
+#pragma unroll
+                for (int i = 0; i < VN; ++i) acc[i] += add[t * d + (int64_t)v * VN + i];
+            }
+            if (out_act) {
+                Vec16<XT> out;
+#pragma unroll
+                for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
+                reinterpret_cast<uint4 *>(out_act + t * d)[v] = out.raw;
+            } else {
+#pragma unroll
+                for (int i = 0; i < VN; ++i) out_f32[t * d + (int64_t)v * VN + i] = acc[i];
+            }
+        }
+    }
+}
+
+int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_perm, int64_t T, int32_t k,
+                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st) {
+    if (T == 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
+    if (act == MOE_BF16)
+        dispatch_bwd_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)dxs, inv_perm, T, k, d, add_f32, out_f32,
+                                                         (bf16 *)out_act);
+    else
+        dispatch_bwd_kernel<float><<<grid, 256, 0, st>>>((const float *)dxs, inv_perm, T, k, d, add_f32, out_f32,
+                                                          (float *)out_act);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+}  // namespace moe

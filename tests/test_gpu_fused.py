@@ -1,0 +1,79 @@
+"""End-to-end parity of moe_forward / moe_backward against the CPU oracle on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1701_06538_b200 import binding as B
+from paper_1701_06538_b200 import synth
+
+from helpers import (TOL_F32, act_empty, assert_close, cat_parts, cfg_of, device_inputs, f32, host, i32, oracle_run,
+                     small_workload, tol_act)
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    small_workload("fused-ragged-f32", T=333, d=36, h=52, n=7, k=3, seed=11),
+    small_workload("fused-bf16", T=1500, d=128, h=256, n=24, k=4, act="bf16", seed=12),
+    small_workload("fused-empty-experts-bf16", T=200, d=64, h=128, n=150, k=2, act="bf16", seed=13),
+    synth.CONFIGS["c1"],
+    synth.CONFIGS["c2"],
+]
+
+
+def run_fused(w, I):
+    cfg = cfg_of(w)
+    S = B.moe_query_sizes(cfg)
+    D = device_inputs(w, I)
+    ctx = B.empty_bytes(S.ctx_bytes)
+    ws = B.empty_bytes(max(S.ws_fwd_bytes, S.ws_bwd_bytes))
+    ws.fill_(0xFF)  # the library must not rely on a zeroed workspace
+    y, losses, imp, load, counts = act_empty(w, w.T, w.d), f32(2), f32(w.n), f32(S.load_elems), i32(w.n)
+    B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], y, losses, imp,
+                  load, counts, ctx, ws)
+    assert B.moe_check_status(ws) == 0
+    dX = act_empty(w, w.T, w.d)
+    dWg, dWn = f32(S.wg_elems), f32(S.wg_elems)
+    dW1, db1 = act_empty(w, w.n, w.d, w.h), act_empty(w, w.n, w.h)
+    dW2, db2 = act_empty(w, w.n, w.h, w.d), act_empty(w, w.n, w.d)
+    B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], ctx,
+                   dX, dWg, dWn, dW1, db1, dW2, db2, ws)
+    assert B.moe_check_status(ws) == 0
+    V = B.ctx_views(cfg, ctx)
+    return dict(y=y, losses=losses, importance=imp, load=load, counts=counts, dX=dX, dWg=dWg, dWnoise=dWn, dW1=dW1,
+                db1=db1, dW2=dW2, db2=db2, ctx=V)
+
+
+@pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
+def test_fused_forward_backward(w):
+    I = synth.make_all(w)
+    F, Bk = oracle_run(w, I)
+    G = run_fused(w, I)
+    V = G["ctx"]
+    # routing: bit-exact
+    assert (host(V["topk_idx"]) == F.G.idx).all()
+    assert (host(V["perm"]) == F.D.perm).all() and (host(V["inv_perm"]) == F.D.inv_perm).all()
+    assert (host(G["counts"]) == F.D.counts).all() and (host(V["offsets"]) == F.D.offsets).all()
+    assert (host(V["kth_idx"]) == F.G.kth_idx).all()
+    # gating floats
+    assert_close(host(V["gates"]), cat_parts(F.G.gates), TOL_F32, "gates")
+    assert_close(host(G["importance"]), F.LS.importance, TOL_F32, "importance")
+    assert_close(host(G["load"]), F.LS.load, TOL_F32, "load")
+    assert_close(host(G["losses"]), F.LS.losses, dict(max=2e-4, mean=2e-4), "losses")
+    # expert side
+    tol = tol_act(w)
+    assert_close(host(V["hid"]), F.hid, tol, "hid")
+    assert_close(host(V["ys"]), F.ys, tol, "ys")
+    assert_close(host(G["y"]), F.y, tol, "y")
+    for name in ("dW1", "db1", "dW2", "db2", "dX"):
+        assert_close(host(G[name]), getattr(Bk, name), tol, name)
+    # gate gradients inherit the expert-side error through dgates
+    assert_close(host(G["dWg"]), cat_parts(Bk.dWg), tol, "dWg")
+    assert_close(host(G["dWnoise"]), cat_parts(Bk.dWnoise), tol, "dWnoise")
+
+
+def test_fused_is_deterministic():
+    w = small_workload("det-bf16", T=700, d=64, h=128, n=16, k=2, act="bf16", seed=14)
+    I = synth.make_all(w)
+    a, b = run_fused(w, I), run_fused(w, I)
+    for name in ("y", "losses", "importance", "load", "dX", "dWg", "dWnoise", "dW1", "db1", "dW2", "db2"):
+        assert torch.equal(a[name], b[name]), name

@@ -1,0 +1,179 @@
+"""Stage-by-stage parity of the CUDA library against the CPU oracle, through the C ABI.
+
+Each stage gets the ORACLE's upstream tensors as inputs, so one kernel is tested at a time:
+indices and permutations bit-exact, fp32 gating tensors within 1e-5, expert-side tensors within
+1e-5 (fp32 layer) or 2e-2 max / 1e-2 mean (bf16 layer), in the rms-floored relative metric of
+helpers.rel_err.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_1701_06538_b200 import binding as B
+from paper_1701_06538_b200 import synth
+
+from helpers import (TOL_F32, act_empty, assert_close, cfg_of, dev, dev_act, device_inputs, f32, host, i32,
+                     oracle_run, prec_of, small_workload, tol_act)
+
+pytestmark = pytest.mark.gpu
+
+FLAT = [
+    small_workload("ragged-f32", T=333, d=36, h=52, n=7, k=3),
+    small_workload("k1-f32", T=130, d=16, h=24, n=5, k=1, seed=2),
+    small_workload("k-eq-n-f32", T=65, d=8, h=8, n=4, k=4, seed=3),
+    small_workload("many-experts-f32", T=257, d=32, h=16, n=300, k=4, seed=4),   # most experts empty
+    small_workload("wide-n-bf16", T=1200, d=128, h=192, n=70, k=2, act="bf16", seed=5),
+    small_workload("k8-bf16", T=515, d=64, h=64, n=33, k=8, act="bf16", seed=6),
+    small_workload("one-expert-f32", T=100, d=12, h=20, n=1, k=1, seed=7),
+    synth.CONFIGS["c1"],
+]
+
+
+@pytest.fixture(scope="module", params=FLAT, ids=lambda w: w.name)
+def case(request):
+    w = request.param
+    I = synth.make_all(w)
+    F, Bk = oracle_run(w, I)
+    return w, I, F, Bk, device_inputs(w, I), cfg_of(w)
+
+
+def ws_for(cfg):
+    S = B.moe_query_sizes(cfg)
+    return B.empty_bytes(S.ws_bytes), S
+
+
+def test_gate(case):
+    w, I, F, _, D, cfg = case
+    ws, S = ws_for(cfg)
+    idx, gates = i32(w.T, w.k), f32(w.T, w.k)
+    clean, raw = f32(w.T, w.n), f32(w.T, w.n)
+    kv, ki = f32(w.T, 2), i32(w.T, 2)
+    B.moe_gate(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], idx, gates, clean, raw, kv, ki, ws)
+    assert (host(clean) == F.G.clean).all(), "clean logits must be bit-exact (fixed fma chain)"
+    assert (host(raw) == F.G.raw).all()
+    assert (host(idx) == F.G.idx).all(), "routing must be bit-exact"
+    assert (host(ki) == F.G.kth_idx).all()
+    assert (host(kv) == F.G.kth_val).all()
+    assert_close(host(gates), F.G.gates, TOL_F32, "gates")
+    assert np.abs(host(gates).sum(axis=1) - 1).max() < 1e-6
+
+
+def test_gate_with_ties_prefers_lowest_index():
+    w = small_workload("ties", T=64, d=8, h=8, n=40, k=3)
+    cfg = cfg_of(w)
+    ws, _ = ws_for(cfg)
+    x = torch.zeros(w.T, w.d, device="cuda")          # all logits equal: 0 + noise * ln 2
+    Wz = torch.zeros(w.d, w.n, device="cuda")
+    noise = torch.zeros(w.T, w.n, device="cuda")
+    noise[:, 7] = 1.0
+    noise[:, 35] = 1.0                                  # two-way tie at the top, 38-way tie below
+    idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
+    kv, ki = f32(w.T, 2), i32(w.T, 2)
+    B.moe_gate(cfg, x, Wz, Wz, noise, idx, gates, clean, raw, kv, ki, ws)
+    assert (host(idx) == np.array([7, 35, 0])).all()
+    assert (host(ki) == np.array([0, 1])).all()
+    G = O.gate(host(x), host(Wz), host(Wz), host(noise), w.k, "f32")
+    assert (G.idx == host(idx)).all() and (G.kth_idx == host(ki)).all()
+
+
+def test_dispatch(case):
+    w, I, F, _, D, cfg = case
+    ws, S = ws_for(cfg)
+    xs, perm, inv = act_empty(w, S.R, w.d), i32(S.R), i32(S.R)
+    counts, offsets = i32(w.n), i32(w.n + 1)
+    B.moe_dispatch(cfg, D["x"], dev(F.G.idx), xs, perm, inv, counts, offsets, ws)
+    assert (host(counts) == F.D.counts).all() and (host(offsets) == F.D.offsets).all()
+    assert (host(perm) == F.D.perm).all() and (host(inv) == F.D.inv_perm).all()
+    assert (host(xs) == np.asarray(F.D.xs, np.float32)).all(), "dispatched rows are exact copies"
+
+
+def test_expert_ffn(case):
+    w, I, F, _, D, cfg = case
+    ws, S = ws_for(cfg)
+    hid, ys = act_empty(w, S.R, w.h), act_empty(w, S.R, w.d)
+    B.moe_expert_ffn(cfg, dev_act(F.D.xs, w), dev(F.D.offsets), D["W1"], D["b1"], D["W2"], D["b2"], hid, ys, ws)
+    assert B.moe_check_status(ws) == 0
+    assert_close(host(hid), F.hid, tol_act(w), "hid")
+    assert_close(host(ys), F.ys, tol_act(w), "ys")
+
+
+def test_combine(case):
+    w, I, F, _, D, cfg = case
+    y = act_empty(w, w.T, w.d)
+    B.moe_combine(cfg, dev_act(F.ys, w), dev(F.G.gates), dev(F.D.inv_perm), y)
+    assert_close(host(y), F.y, tol_act(w), "y")
+
+
+def test_losses(case):
+    w, I, F, _, D, cfg = case
+    ws, S = ws_for(cfg)
+    imp, load, L = f32(w.n), f32(S.load_elems), f32(2)
+    B.moe_losses(cfg, dev(F.G.idx), dev(F.G.gates), dev(F.G.clean), dev(F.G.raw), dev(F.G.kth_val), imp, load, L, ws)
+    assert_close(host(imp), F.LS.importance, TOL_F32, "importance")
+    assert_close(host(load), F.LS.load, TOL_F32, "load")
+    assert_close(host(L), F.LS.losses, dict(max=2e-4, mean=2e-4), "losses")  # CV^2 amplifies by ~mean/std
+
+
+def test_combine_bwd(case):
+    w, I, F, Bk, D, cfg = case
+    S = B.moe_query_sizes(cfg)
+    dg, dys = f32(w.T, w.k), act_empty(w, S.R, w.d)
+    B.moe_combine_bwd(cfg, D["dY"], dev_act(F.ys, w), dev(F.G.gates), dev(F.D.inv_perm), dg, dys)
+    assert_close(host(dg), Bk.dgates, tol_act(w) if w.act == "bf16" else TOL_F32, "dgates")
+    assert_close(host(dys), Bk.dys, tol_act(w), "dys")
+
+
+def test_expert_ffn_bwd(case):
+    w, I, F, Bk, D, cfg = case
+    ws, S = ws_for(cfg)
+    dxs = act_empty(w, S.R, w.d)
+    dW1, db1 = act_empty(w, w.n, w.d, w.h), act_empty(w, w.n, w.h)
+    dW2, db2 = act_empty(w, w.n, w.h, w.d), act_empty(w, w.n, w.d)
+    B.moe_expert_ffn_bwd(cfg, dev_act(F.D.xs, w), dev_act(F.hid, w), dev_act(Bk.dys, w), dev(F.D.offsets), D["W1"],
+                         D["W2"], dxs, dW1, db1, dW2, db2, ws)
+    assert B.moe_check_status(ws) == 0
+    tol = tol_act(w)
+    for name, got, want in (("dxs", dxs, Bk.dxs), ("dW1", dW1, Bk.dW1), ("db1", db1, Bk.db1), ("dW2", dW2, Bk.dW2),
+                            ("db2", db2, Bk.db2)):
+        assert_close(host(got), want, tol, name)
+    empty = np.nonzero(F.D.counts == 0)[0]
+    if empty.size:
+        assert float(host(dW1)[empty].__abs__().max()) == 0.0 and float(host(db2)[empty].__abs__().max()) == 0.0
+
+
+def test_dispatch_bwd(case):
+    w, I, F, Bk, D, cfg = case
+    out = f32(w.T, w.d)
+    B.moe_dispatch_bwd(cfg, dev_act(Bk.dxs, w), dev(F.D.inv_perm), out)
+    assert_close(host(out), Bk.dX_expert, TOL_F32, "dX_expert")
+
+
+def test_losses_bwd_and_gate_bwd(case):
+    w, I, F, Bk, D, cfg = case
+    ws, S = ws_for(cfg)
+    prec = prec_of(w)
+    dg_want, dload_want = O.losses_bwd(F.LS.importance, F.LS.load, F.G.idx, Bk.dgates, w.w_importance, w.w_load, prec)
+    dg, dload = dev(np.asarray(Bk.dgates, np.float32)), f32(S.dload_elems)
+    B.moe_losses_bwd(cfg, dev(F.LS.importance), dev(F.LS.load), dev(F.G.idx), dg, dload, ws)
+    assert_close(host(dg), dg_want, TOL_F32, "dgates+importance")
+    assert_close(host(dload), dload_want, dict(max=1e-4, mean=1e-4), "dload")
+    GB = O.gate_bwd(I["x"], I["Wg"], I["Wnoise"], I["noise"], F.G.clean, F.G.raw, F.G.idx, F.G.gates, F.G.kth_val,
+                    F.G.kth_idx, dg_want, dload_want, prec)
+    dWg, dWn, dXg = f32(w.d, w.n), f32(w.d, w.n), f32(w.T, w.d)
+    B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], dev(F.G.clean), dev(F.G.raw), dev(F.G.idx),
+                   dev(F.G.gates), dev(F.G.kth_val), dev(F.G.kth_idx), dev(dg_want), dev(dload_want), dWg, dWn, dXg,
+                   ws)
+    assert_close(host(dWg), GB.dWg, TOL_F32, "dWg")
+    assert_close(host(dWn), GB.dWnoise, TOL_F32, "dWnoise")
+    assert_close(host(dXg), GB.dX_gate, TOL_F32, "dX_gate")
+
+
+def test_empty_batch():
+    w = small_workload("empty", T=0, d=16, h=16, n=4, k=2)
+    cfg = cfg_of(w)
+    ws, S = ws_for(cfg)
+    counts, offsets = i32(w.n), i32(w.n + 1)
+    B.moe_dispatch(cfg, act_empty(w, 1, w.d), i32(1), act_empty(w, 1, w.d), i32(1), i32(1), counts, offsets, ws)
+    torch.cuda.synchronize()
+    assert host(counts).sum() == 0 and host(offsets).sum() == 0
