@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE layer hot path: one step = moe_forward + moe_backward (both balancing
+losses included) over one synthetic batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c5] [--impl ours|reference]
+
+N > 1 is launched by torchrun (one rank per GPU); the layer has no exchange step on one GPU per
+replica, so ranks run independent replicas ("weak" scaling, no data-path collective); timing is the
+max over ranks. Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import concurrent.futures
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_1701_06538_b200 import synth  # noqa: E402
+
+METRIC = "moe_layer_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 2 ** 20
+# FP32 FMA peak of a B200 at its maximum SM clock: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                p = json.load(f)
+            return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arm
+def sample_workload(w, Ts):
+    return synth.Workload(**{**w.__dict__, "T": min(Ts, w.T), "name": f"{w.name}[first {min(Ts, w.T)} tokens]"})
+
+
+def oracle_step(ws, I):
+    """One forward+backward of the CPU oracle (test infrastructure) on host arrays."""
+    from oracle import moe_oracle as O
+    prec = "bf16" if ws.act == "bf16" else "f32"
+    F = O.forward(I["x"], I["Wg"], I["Wnoise"], I["noise"], I["W1"], I["b1"], I["W2"], I["b2"], ws.k,
+                  ws.w_importance, ws.w_load, prec, hier=ws.hier)
+    O.backward(I["dY"], I["x"], I["Wg"], I["Wnoise"], I["noise"], I["W1"], I["b1"], I["W2"], I["b2"], F,
+               ws.w_importance, ws.w_load, prec, hier=ws.hier)
+
+
+def host_inputs_sample(w, Ts, experts=None):
+    """Inputs of the first Ts tokens of workload w (the streams are per tensor, so rows [0, Ts) of the
+    full tensors are drawn by drawing the full x / noise / dY; expert weights are per expert)."""
+    ws = sample_workload(w, Ts)
+    x, dY = synth.make_x(w)[:ws.T], synth.make_dY(w)[:ws.T]
+    Wg, Wn, noise = synth.make_gate(w)
+    noise = tuple(p[:ws.T] for p in noise) if isinstance(noise, tuple) else noise[:ws.T]
+    W1, b1, W2, b2 = experts if experts is not None else synth.make_experts(w)
+    return ws, dict(x=x, dY=dY, Wg=Wg, Wnoise=Wn, noise=noise, W1=W1, b1=b1, W2=W2, b2=b2)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_sample_tokens(w):
+    # about 10-30 s of oracle work per forward+backward on the host cores
+    per_token_flop = 12.0 * w.k * w.d * w.h + 12.0 * w.d * (w.n if w.a == 0 else w.a + w.k1 * w.b)
+    return int(max(256, min(w.T, 2 ** int(np.log2(2.0e12 / per_token_flop)))))
+
+
+def run_reference(args, w):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    Ts = cpu_sample_tokens(w)
+    ws, I = host_inputs_sample(w, Ts)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(ws, I)
+    times = []
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        oracle_step(ws, I)
+        times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = ws.T * args.steps / total
+    cores = blas_threads()
+    sample = f"first {ws.T} of {w.T} tokens of {w.name}, all {w.n} experts resident, forward+backward per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def workload_config(w):
+    esz = 2 if w.act == "bf16" else 4
+    resident = w.T * w.d * esz * 2 + w.R * (2 * w.d + w.h) * esz + 2 * w.n * w.d * w.h * esz
+    return {"workload": w.name, "T": w.T, "d_model": w.d, "hidden": w.h, "experts": w.n, "k": w.k,
+            "hierarchical": [w.a, w.k1, w.b, w.k2] if w.a else None, "act": w.act, "gating": "f32",
+            "l2": "inputs larger than L2" if resident > 2 * L2_BYTES else "L2 flushed between timed steps",
+            "parallelism": "replicas (one per GPU, no collective)"}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.path = tempfile.mktemp(prefix="clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(gpu_index)], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "power_w_max": max(power), "samples": len(sm)}
+
+
+def build_device_state(w, keep_host_experts):
+    """Device tensors of the workload. Expert weights are drawn per expert on host threads and moved
+    expert by expert, so the host never holds more than a few experts unless the CPU baseline needs them."""
+    from paper_1701_06538_b200 import binding as B
+    adt = torch.bfloat16 if w.act == "bf16" else torch.float32
+    cfg = B.make_config(w.T, w.d, w.h, w.n, w.k, w.act, w.w_importance, w.w_load, w.a, w.k1, w.b, w.k2)
+    S = B.moe_query_sizes(cfg)
+
+    def cat(parts):
+        if isinstance(parts, tuple):
+            return np.concatenate([p.reshape(-1) for p in parts])
+        return parts.reshape(-1)
+
+    host = {"x": synth.make_x(w), "dY": synth.make_dY(w)}
+    Wg, Wn, noise = synth.make_gate(w)
+    host.update(Wg=Wg, Wnoise=Wn, noise=noise)
+    D = {"x": torch.from_numpy(host["x"]).to(adt).cuda(), "dY": torch.from_numpy(host["dY"]).to(adt).cuda(),
+         "Wg": torch.from_numpy(cat(Wg)).cuda(), "Wnoise": torch.from_numpy(cat(Wn)).cuda(),
+         "noise": torch.from_numpy(cat(noise)).cuda()}
+    D["W1"] = torch.empty(w.n, w.d, w.h, dtype=adt, device="cuda")
+    D["W2"] = torch.empty(w.n, w.h, w.d, dtype=adt, device="cuda")
+    D["b1"] = torch.empty(w.n, w.h, dtype=adt, device="cuda")
+    D["b2"] = torch.empty(w.n, w.d, dtype=adt, device="cuda")
+    if keep_host_experts:
+        host["W1"] = np.empty((w.n, w.d, w.h), np.float32); host["W2"] = np.empty((w.n, w.h, w.d), np.float32)
+        host["b1"] = np.empty((w.n, w.h), np.float32); host["b2"] = np.empty((w.n, w.d), np.float32)
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        for e, (W1, b1, W2, b2) in enumerate(pool.map(lambda e: synth.make_expert(w, e), range(w.n))):
+            D["W1"][e].copy_(torch.from_numpy(W1)); D["W2"][e].copy_(torch.from_numpy(W2))
+            D["b1"][e].copy_(torch.from_numpy(b1)); D["b2"][e].copy_(torch.from_numpy(b2))
+            if keep_host_experts:
+                host["W1"][e], host["b1"][e], host["W2"][e], host["b2"][e] = W1, b1, W2, b2
+    e = lambda *s, dt=torch.float32: torch.empty(*s, dtype=dt, device="cuda")
+    D.update(y=e(w.T, w.d, dt=adt), losses=e(2), importance=e(w.n), load=e(S.load_elems),
+             counts=e(w.n, dt=torch.int32), dX=e(w.T, w.d, dt=adt), dWg=e(S.wg_elems), dWnoise=e(S.wg_elems),
+             dW1=e(w.n, w.d, w.h, dt=adt), db1=e(w.n, w.h, dt=adt), dW2=e(w.n, w.h, w.d, dt=adt),
+             db2=e(w.n, w.d, dt=adt), ctx=B.empty_bytes(S.ctx_bytes),
+             ws=B.empty_bytes(max(S.ws_fwd_bytes, S.ws_bwd_bytes)))
+    return cfg, S, D, host
+
+
+def run_ours(args, w):
+    from paper_1701_06538_b200 import binding as B
+    rank, local_rank, world = dist_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks, peak_kind = load_peaks()
+    want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+    cfg, S, D, host = build_device_state(w, keep_host_experts=want_cpu)
+
+    def fwd():
+        B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], D["y"],
+                      D["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+
+    def bwd():
+        B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
+                       D["ctx"], D["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"], D["db2"], D["ws"])
+
+    small = "flushed" in workload_config(w)["l2"]
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if small else None
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    def timed(step_fn, K):
+        """K steps, each between its own pair of events on the launching stream; returns per-step ms."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        barrier()
+        for a, b in ev:
+            if flush_buf is not None:
+                flush_buf.fill_(1)
+            a.record()
+            step_fn()
+            b.record()
+        barrier()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    def step():
+        fwd()
+        bwd()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert B.moe_check_status(D["ws"]) == 0
+    sampler = ClockSampler(local_rank)
+    l0 = B.moe_debug_launch_count()
+    ms = timed(step, args.steps)
+    launches = B.moe_debug_launch_count() - l0
+
+    # end to end: pinned host inputs in, results out, every step
+    hx, hdY = torch.from_numpy(host["x"]).to(D["x"].dtype).pin_memory(), torch.from_numpy(host["dY"]).to(D["x"].dtype).pin_memory()
+    hnoise = D["noise"].cpu().pin_memory()
+    hy, hdX, hl = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory(), torch.empty(2).pin_memory()
+
+    def step_e2e():
+        D["x"].copy_(hx, non_blocking=True); D["noise"].copy_(hnoise, non_blocking=True)
+        D["dY"].copy_(hdY, non_blocking=True)
+        fwd()
+        bwd()
+        hy.copy_(D["y"], non_blocking=True); hdX.copy_(D["dX"], non_blocking=True)
+        hl.copy_(D["losses"], non_blocking=True)
+
+    step_e2e()
+    ms_e2e = timed(step_e2e, args.steps)
+    clocks = sampler.stop()
+    h2d = hx.numel() * hx.element_size() * 2 + hnoise.numel() * 4
+    d2h = hy.numel() * hy.element_size() * 2 + 8
+
+    total_ms, total_e2e = sum(ms), sum(ms_e2e)
+    if world > 1:
+        t = torch.tensor([total_ms, total_e2e], device="cuda", dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms, total_e2e = t.tolist()
+    value = world * w.T * args.steps / (total_ms / 1e3)
+    value_e2e = world * w.T * args.steps / (total_e2e / 1e3)
+
+    stages = stage_timings(B, cfg, S, D, w, timed, max(3, min(args.steps, 10)), peaks)
+    gemm_flop = 12.0 * w.R * w.d * w.h
+    gemm_ms = stages["expert_ffn"]["ms"] + stages["expert_ffn_bwd"]["ms"]
+    achieved = gemm_flop / (gemm_ms / 1e3) / 1e12
+    if w.act == "bf16":
+        roof = {"bound": "tensor", "kernel": "expert grouped GEMMs (moe_expert_ffn + moe_expert_ffn_bwd)",
+                "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                "peak_kind": f"{peak_kind} sustained bf16 (kernels timed back to back inside a long loop)",
+                "frac_of_nominal_2250": achieved / 2250.0}
+    else:
+        roof = {"bound": "alu", "kernel": "expert grouped GEMMs, fp32 SIMT", "achieved": achieved,
+                "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
+                "peak_kind": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.act == "bf16" else "f32",
+           "data": "synthetic", "config": workload_config(w), "clocks": clocks,
+           "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                   "ms_per_step": total_e2e / args.steps},
+           "gpu_launches": launches, "roofline": roof, "stages": stages,
+           "balance": balance_metrics(D)}
+    if want_cpu:
+        Ts = cpu_sample_tokens(w)
+        wsamp, I = host_inputs_sample(w, Ts, experts=(host["W1"], host["b1"], host["W2"], host["b2"]))
+        t0 = time.perf_counter()
+        oracle_step(wsamp, I)
+        sec = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": wsamp.T / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                               "sample": f"first {wsamp.T} of {w.T} tokens, all {w.n} experts, one forward+backward "
+                                         f"({sec:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def balance_metrics(D):
+    """The balance metrics of the paper's loss-ablation table, for the realised routing."""
+    imp, load, counts = D["importance"].double(), D["load"][:D["importance"].numel()].double(), D["counts"].double()
+    cv = lambda v: float(v.std(unbiased=False) / v.mean())
+    return {"cv_importance": cv(imp), "cv_load": cv(load), "max_over_mean_load": float(load.max() / load.mean()),
+            "max_over_min_count": float(counts.max() / counts.min().clamp(min=1)),
+            "max_over_mean_count": float(counts.max() / counts.mean())}
+
+
+def stage_timings(B, cfg, S, D, w, timed, K, peaks):
+    """Each stage call alone, K launches between events, on the tensors the fused forward saved."""
+    V = B.ctx_views(cfg, D["ctx"])
+    T, d, h, n, k, R = w.T, w.d, w.h, w.n, w.k, w.R
+    esz = 2 if w.act == "bf16" else 4
+    adt = D["x"].dtype
+    e = lambda *s, dt=torch.float32: torch.empty(*s, dtype=dt, device="cuda")
+    ws = D["ws"]
+    dgates, dys, dxs = e(S.gates_elems), e(R, d, dt=adt), e(R, d, dt=adt)
+    dload, dXe, dXg = e(S.dload_elems), e(T, d), e(T, d)
+    gate_cols = S.gate_cols
+    calls = {
+        "gate": (lambda: B.moe_gate(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], V["topk_idx"], V["gates"],
+                                    V["clean"], V["raw_noise"], V["kth_vals"], V["kth_idx"], ws),
+                 4.0 * T * d * gate_cols, T * d * esz + 3 * 4 * T * gate_cols + 8 * R + 16 * T),
+        "dispatch": (lambda: B.moe_dispatch(cfg, D["x"], V["topk_idx"], V["xs"], V["perm"], V["inv_perm"],
+                                            V["counts"], V["offsets"], ws), 0.0, (1 + k) * T * d * esz + 12 * R),
+        "expert_ffn": (lambda: B.moe_expert_ffn(cfg, V["xs"], V["offsets"], D["W1"], D["b1"], D["W2"], D["b2"],
+                                                V["hid"], V["ys"], ws),
+                       4.0 * R * d * h, (2 * R * d + 2 * R * h) * esz + 2 * n * d * h * esz),
+        "combine": (lambda: B.moe_combine(cfg, V["ys"], V["gates"], V["inv_perm"], D["y"]), 0.0,
+                    (k + 1) * T * d * esz + 8 * R),
+        "losses": (lambda: B.moe_losses(cfg, V["topk_idx"], V["gates"], V["clean"], V["raw_noise"], V["kth_vals"],
+                                        D["importance"], D["load"], D["losses"], ws), 0.0, 2 * 4 * T * gate_cols + 16 * R),
+        "combine_bwd": (lambda: B.moe_combine_bwd(cfg, D["dY"], V["ys"], V["gates"], V["inv_perm"], dgates, dys), 0.0,
+                        (1 + 2 * k) * T * d * esz + 12 * R),
+        "expert_ffn_bwd": (lambda: B.moe_expert_ffn_bwd(cfg, V["xs"], V["hid"], dys, V["offsets"], D["W1"], D["W2"],
+                                                        dxs, D["dW1"], D["db1"], D["dW2"], D["db2"], ws),
+                           8.0 * R * d * h, (4 * R * d + 3 * R * h) * esz + 4 * n * d * h * esz),
+        "losses_bwd": (lambda: B.moe_losses_bwd(cfg, D["importance"], D["load"], V["topk_idx"], dgates, dload, ws),
+                       0.0, 12 * R),
+        "gate_bwd": (lambda: B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], V["clean"], V["raw_noise"],
+                                            V["topk_idx"], V["gates"], V["kth_vals"], V["kth_idx"], dgates, dload,
+                                            D["dWg"], D["dWnoise"], dXg, ws),
+                     8.0 * T * d * gate_cols, T * d * (esz + 4) + 5 * 4 * T * gate_cols),
+        "dispatch_bwd": (lambda: B.moe_dispatch_bwd(cfg, dxs, V["inv_perm"], dXe), 0.0, k * T * d * esz + T * d * 4),
+    }
+    out = {}
+    for name, (fn, flop, byts) in calls.items():
+        fn()
+        ms = statistics.mean(timed(fn, K))
+        rec = {"ms": ms, "GB/s": byts / ms / 1e6, "hbm_frac": byts / ms / 1e6 / peaks["hbm_gbs"]}
+        if flop:
+            rec["TFLOP/s"] = flop / ms / 1e9
+        out[name] = rec
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c5", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--tokens", type=int, default=0, help="override T (smaller captures under a profiler)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.CONFIGS[args.config]
+    if args.tokens:
+        w = w.scaled(args.tokens)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -98,6 +98,10 @@ int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *host_out);
 int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *host_out);
 const char *moe_status_string(int32_t status);
 
+/* Diagnostics only: number of kernels this library has launched in this process so far
+ * (a host-side counter; the one piece of process-wide state the library keeps). */
+int64_t moe_debug_launch_count(void);
+
 /* Synchronises `stream`, then reads the status word the kernels of the last call that used
  * `ws` left there. MOE_OK, or MOE_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel
  * gave up (its outputs are then undefined; the context stays usable). */

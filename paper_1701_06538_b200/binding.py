@@ -19,7 +19,7 @@ MOE_F32, MOE_BF16 = 0, 1
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED", 3: "MOE_ERR_WORKSPACE",
                 4: "MOE_ERR_CUDA", 5: "MOE_ERR_TIMEOUT"}
 
-EXPORTS = ["moe_validate", "moe_query_sizes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
+EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
            "moe_gate", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward"]
@@ -62,6 +62,7 @@ def lib():
         for name in EXPORTS:
             getattr(L, name).restype = ctypes.c_int32
         L.moe_status_string.restype = ctypes.c_char_p
+        L.moe_debug_launch_count.restype = ctypes.c_int64
         _lib = L
     return _lib
 
@@ -93,6 +94,10 @@ def _call(name, cfg, *tensors, stream=True):
     status = getattr(lib(), name)(*args)
     if status != 0:
         raise MoeError(name, status)
+
+
+def moe_debug_launch_count() -> int:
+    return int(lib().moe_debug_launch_count())
 
 
 def moe_validate(cfg) -> int:

@@ -3,7 +3,12 @@
 
 #include "moe_internal.cuh"
 
+#include <atomic>
+
 using namespace moe;
+
+static std::atomic<long long> g_launches{0};
+void moe::count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 namespace {
 
@@ -352,6 +357,8 @@ const char *moe_status_string(int32_t s) {
         default: return "unknown status";
     }
 }
+
+int64_t moe_debug_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 int32_t moe_validate(const moe_config *cfg) { return check_config(cfg); }
 

@@ -20,10 +20,13 @@
 
 #define MOE_LAUNCHED()                                           \
     do {                                                         \
+        ::moe::count_launch();                                   \
         if (cudaPeekAtLastError() != cudaSuccess) return MOE_ERR_CUDA; \
     } while (0)
 
 namespace moe {
+
+void count_launch();  // diagnostics: kernels launched by this library so far (api.cu)
 
 typedef __nv_bfloat16 bf16;
 

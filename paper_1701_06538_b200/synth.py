@@ -61,11 +61,11 @@ CONFIGS = {
     "c1": Workload("c1-tiny-f32", T=256, d=64, h=128, n=8, k=2, act="f32", seed=BASE_SEED + 0),
     "c2": Workload("c2-lm-flat-32", T=8192, d=512, h=1024, n=32, k=4, seed=BASE_SEED + 1),
     "c3": Workload("c3-flat-256-uneven", T=32768, d=512, h=1024, n=256, k=4, seed=BASE_SEED + 2,
-                   skew="normal", gamma=0.17),
+                   skew="normal", gamma=0.205),
     "c4": Workload("c4-hier-64x64", T=65536, d=512, h=1024, n=4096, k=4, a=64, k1=2, b=64, k2=2,
                    seed=BASE_SEED + 3),
     "c5": Workload("c5-wide-zipf-128", T=131072, d=1024, h=4096, n=128, k=2, seed=BASE_SEED + 4,
-                   skew="zipf", gamma=0.78),
+                   skew="zipf", gamma=0.79),
 }
 
 

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
     assert len(names) >= 17
     for name in names:
         assert hasattr(lib, name), name
-    assert sorted(B.EXPORTS) == [n for n in names]
+    assert sorted(B.EXPORTS) == names
 
 
 def test_struct_layouts_match_header():
