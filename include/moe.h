@@ -49,7 +49,7 @@ typedef enum {
     MOE_OK = 0,
     MOE_ERR_INVALID_ARG = 1, /* NULL pointer, misaligned pointer, inconsistent or non-positive size */
     MOE_ERR_UNSUPPORTED = 2, /* valid in the method but outside what this build implements          */
-    MOE_ERR_WORKSPACE = 3,   /* reserved: workspace too small (sizes are the caller's contract)     */
+    MOE_ERR_WORKSPACE = 3,   /* the problem does not fit a fixed-size scratch (moe_dispatch_noalloc)  */
     MOE_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                              */
     MOE_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see moe_check_status)           */
 } moe_status;
@@ -133,6 +133,26 @@ int32_t moe_gate(const moe_config *cfg, const void *x, const float *Wg, const fl
  *      row r; inv_perm [R] sorted row of slot p; xs [R,d] act, xs[r] = x[perm[r] / k]. */
 int32_t moe_dispatch(const moe_config *cfg, const void *x, const int32_t *topk_idx, void *xs, int32_t *perm,
                      int32_t *inv_perm, int32_t *counts, int32_t *offsets, void *ws, void *stream);
+
+/* Dispatch without a workspace. (The paper has no counterpart: this entry point exists for the
+ * integration, not for the method.) Same inputs, outputs and results as moe_dispatch, but it takes
+ * no `ws`: its scratch is a fixed array of MOE_NOALLOC_SCRATCH_INTS int32 (4 MiB + 256 B) inside
+ * the library's device image, held by every GPU that loads the library until the process exits.
+ * It is meant for callers that cannot obtain device memory of their own at the point of the call
+ * -- code running inside a host framework's memory plan or a real-time loop where cudaMalloc (a
+ * device-wide synchronising call) is forbidden, or plug-ins handed fixed input/output buffers and
+ * nothing else. The call itself allocates and frees nothing, on the device or through any library.
+ *  - Limit: ceil(T*k / 1024) * n + 64 <= MOE_NOALLOC_SCRATCH_INTS, else MOE_ERR_WORKSPACE is
+ *    returned and nothing is launched (e.g. T*k = 262144 rows with up to 4096 experts fit).
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call before starting any stream capture.
+ *  - All calls in the process share the array, which keeps whatever the last call left there
+ *    (the kernels overwrite every word before reading it, so nothing needs clearing). Two
+ *    calls that overlap on the GPU -- different streams, or different host threads -- race on
+ *    it: serialise them. */
+#define MOE_NOALLOC_SCRATCH_INTS ((1 << 20) + 64)
+int32_t moe_dispatch_noalloc(const moe_config *cfg, const void *x, const int32_t *topk_idx, void *xs,
+                             int32_t *perm, int32_t *inv_perm, int32_t *counts, int32_t *offsets, void *stream);
 
 /* Experts (Section 3.2, Appendix C): on the rows offsets[e] <= r < offsets[e+1],
  *   hid = relu(xs.W1[e] + b1[e]),  ys = hid.W2[e] + b2[e],

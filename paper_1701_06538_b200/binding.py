@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED",
                 4: "MOE_ERR_CUDA", 5: "MOE_ERR_TIMEOUT"}
 
 EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
-           "moe_gate", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
+           "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward"]
 
@@ -130,6 +130,12 @@ def moe_gate(cfg, x, Wg, Wnoise, noise, topk_idx, gates, clean, raw_noise, kth_v
 
 def moe_dispatch(cfg, x, topk_idx, xs, perm, inv_perm, counts, offsets, ws):
     _call("moe_dispatch", cfg, x, topk_idx, xs, perm, inv_perm, counts, offsets, ws)
+
+
+def moe_dispatch_noalloc(cfg, x, topk_idx, xs, perm, inv_perm, counts, offsets):
+    """moe_dispatch for callers that cannot provide a workspace: the scratch is a fixed array inside
+    the library (see include/moe.h for the size limit and the sharing rules)."""
+    _call("moe_dispatch_noalloc", cfg, x, topk_idx, xs, perm, inv_perm, counts, offsets)
 
 
 def moe_expert_ffn(cfg, xs, offsets, W1, b1, W2, b2, hid, ys, ws):
