@@ -272,11 +272,14 @@ int32_t do_losses(const moe_config *c, const Dims &D, const int32_t *topk_idx, c
     return launch_cv2(importance, (int32_t)D.n, load, (int32_t)D.n, c->w_importance, c->w_load, losses, st);
 }
 
-int32_t do_expert_ffn_bwd(const Dims &D, const void *xs, const void *hid, const void *dys, const int32_t *offsets,
-                          const void *W1, const void *W2, void *dxs, void *dW1, void *db1, void *dW2, void *db2,
-                          Carver &cv, cudaStream_t st) {
+int32_t do_expert_ffn_bwd(const moe_config *c, const Dims &D, const void *xs, const void *hid, const void *dys,
+                          const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
+                          void *dW2, void *db2, void *ws_base, Carver &cv, cudaStream_t st) {
     FfnBwdWs w(cv, D);
     const int32_t n = (int32_t)D.n;
+    if (tc_ffn_supported(*c))
+        return launch_tc_ffn_bwd(*c, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, w.dz, w.colsum,
+                                 w.tile_prefix, status_word(ws_base), st);
     MOE_TRY(launch_segment_colsum(dys, D.act, offsets, n, D.R, (int32_t)D.d, db2, w.colsum, w.tile_prefix, st));
     SimtGemm g = base_gemm(D);  // dW2[e] = hid_e^T . dys_e
     g.A = hid; g.B = dys; g.C = dW2;
@@ -476,7 +479,8 @@ int32_t moe_expert_ffn_bwd(const moe_config *cfg, const void *xs, const void *hi
     Carver cv(ws);
     cv.take_bytes(kWsHeader);
     MOE_TRY(reset_status(ws, as_stream(stream)));
-    return do_expert_ffn_bwd(D, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, cv, as_stream(stream));
+    return do_expert_ffn_bwd(cfg, D, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws, cv,
+                             as_stream(stream));
 }
 
 int32_t moe_dispatch_bwd(const moe_config *cfg, const void *dxs, const int32_t *inv_perm, float *dX_expert,
@@ -556,7 +560,8 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
     MOE_TRY(launch_combine_bwd(dY, C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dgates,
                                B.dys, st));
     { Carver cv = fresh();
-      MOE_TRY(do_expert_ffn_bwd(D, C.xs, C.hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, cv, st)); }
+      MOE_TRY(do_expert_ffn_bwd(cfg, D, C.xs, C.hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, ws, cv,
+                                st)); }
     { Carver cv = fresh();
       MOE_TRY(do_losses_bwd(cfg, D, C.importance, C.load, C.topk_idx, B.dgates, B.dload, cv, st)); }
     { Carver cv = fresh();

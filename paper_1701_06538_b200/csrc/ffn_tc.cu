@@ -1,12 +1,565 @@
-// Tensor-core expert kernels (tcgen05 / TMEM / TMA). Placeholder until the kernels land:
-// reports "not supported" so the SIMT grouped GEMM is used.
+// Expert feed-forward networks on the 5th-generation tensor cores (Section 3.2, Appendix C):
+// variable-size grouped GEMMs, bf16 operands, fp32 accumulation in tensor memory.
+//
+// One persistent kernel template, one CTA per SM, 128 x 256 output tiles, K blocks of 64:
+//   warp 0      TMA producer: one bulk tensor copy per operand per stage into 128-byte-swizzled
+//               shared memory, completion counted on an mbarrier (4 stages)
+//   warp 1      MMA issuer: tcgen05.mma (cta_group::1, kind::f16, M 128, N 256, K 16), accumulator
+//               in TMEM, double buffered (2 x 256 columns) so the epilogue of one tile overlaps
+//               the main loop of the next; tcgen05.commit releases the stage / publishes the tile
+//   warps 2-5   epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), bias / ReLU / ReLU
+//               mask, round to bf16, 64-byte row stores with a row guard for ragged segments
+//
+// Three operand arrangements (KIND):
+//   ROW_BMN  rows x K activations (K-major A) times a per-expert [K, N] weight (N contiguous,
+//            "MN-major" B): forward GEMMs  hid = relu(xs.W1 + b1),  ys = hid.W2 + b2
+//   ROW_BK   same A, per-expert weight read transposed ([N, K], K contiguous, K-major B):
+//            dz = (dys.W2^T) * [hid > 0],  dxs = dz.W1^T
+//   WGRAD    contraction over the rows of a segment, both operands MN-major:
+//            dW2 = hid^T.dys,  dW1 = xs^T.dz. The last K block of a segment is ragged: the rows
+//            past the segment end are zeroed in shared memory (A operand only: 0 x finite = 0).
+// Weights are addressed through one tensor map with the expert as a coordinate, segment bounds
+// are read on the device: no per-expert descriptors and no host synchronisation.
+//
+// Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the CTA records
+// MOE_ERR_TIMEOUT in the workspace status word, stops issuing work, drains and frees its TMEM.
+#include <cuda.h>
+
 #include "moe_internal.cuh"
 
 namespace moe {
-bool tc_ffn_supported(const moe_config &) { return false; }
-int64_t tc_ffn_ws_bytes(const moe_config &) { return 0; }
-int32_t launch_tc_ffn(const moe_config &, const void *, const int32_t *, const void *, const void *, const void *,
-                      const void *, void *, void *, void *, int32_t *, cudaStream_t) {
-    return MOE_ERR_UNSUPPORTED;
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;  // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;  // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int TMEM_COLS = 512;
+constexpr int NTHREADS = 192;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+enum Kind { ROW_BMN = 0, ROW_BK = 1, WGRAD = 2 };
+
+struct GemmParams {
+    const int32_t *offsets;      // [nseg + 1] segment bounds (rows)
+    const int32_t *tile_prefix;  // ROW_*: [nseg + 1] prefix of 128-row tiles
+    int32_t nseg;
+    int32_t M;  // WGRAD: rows of the per-expert output; ROW_*: unused
+    int32_t N;  // output columns
+    int32_t K;  // ROW_*: contraction length; WGRAD: unused (segment rows)
+    bf16 *out;  // ROW_*: [R, N]; WGRAD: [nseg, M, N]
+    const bf16 *bias;  // [nseg, N] or nullptr
+    const bf16 *mask;  // [R, N] or nullptr: result kept where mask > 0
+    int32_t relu;
+    int32_t *status;
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait. Returns false (and raises the CTA's abort flag + the status word) on expiry.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) {
+            *abort_flag = 1;
+            atomicExch(status, (int32_t)MOE_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1,
+                                            int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
+        "[%2];" ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle, descriptor version 1 at bit 46).
+// K-major: rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride byte offset).
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// MN-major: 64 contiguous MN elements (128 B) per K row; 8 K rows per 1024-B atom (stride byte
+// offset); the next 64 MN elements start BK * 128 B further (leading byte offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)((BK * 128) >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: D fp32, A/B bf16, majors, N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+struct Tile {
+    int32_t e;        // expert / segment
+    int32_t row0;     // ROW_*: first sorted row; WGRAD: first row of the segment
+    int32_t row_end;  // end of the segment
+    int32_t m0;       // WGRAD: first output row of the tile
+    int32_t n0;       // first output column
+    int32_t kblocks;  // number of K blocks
+};
+
+template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
+    const int32_t tiles_n = (p.N + BN - 1) / BN;
+    if (KIND == WGRAD) {
+        const int32_t tiles_m = (p.M + BM - 1) / BM;
+        const int64_t per_e = (int64_t)tiles_m * tiles_n;
+        if (id >= per_e * p.nseg) return false;
+        t.e = (int32_t)(id / per_e);
+        const int32_t rem = (int32_t)(id % per_e);
+        t.m0 = (rem / tiles_n) * BM;
+        t.n0 = (rem % tiles_n) * BN;
+        t.row0 = p.offsets[t.e];
+        t.row_end = p.offsets[t.e + 1];
+        t.kblocks = (t.row_end - t.row0 + BK - 1) / BK;
+        return true;
+    } else {
+        const int32_t total_m = p.tile_prefix[p.nseg];
+        if (id >= (int64_t)total_m * tiles_n) return false;
+        const int32_t mt = (int32_t)(id / tiles_n);
+        t.n0 = (int32_t)(id % tiles_n) * BN;
+        int lo = 0, hi = p.nseg;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.tile_prefix[mid] <= mt) lo = mid; else hi = mid;
+        }
+        t.e = lo;
+        t.row0 = p.offsets[lo] + (mt - p.tile_prefix[lo]) * BM;
+        t.row_end = p.offsets[lo + 1];
+        t.m0 = 0;
+        t.kblocks = p.K / BK;
+        return true;
+    }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(NTHREADS, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-B aligned for the 128-B swizzle
+    uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
+                Tile t;
+                if (!decode_tile<KIND>(p, id, t)) break;
+                for (int kb = 0; kb < t.kblocks && ok; ++kb) {
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + A_BYTES;
+                    mbar_expect_tx(full_bar(s), STAGE_BYTES);
+                    if (KIND == WGRAD) {
+                        const int r = t.row0 + kb * BK;
+                        tma_load_3d(a_dst, &tmA, full_bar(s), 0, r, t.m0 / 64);
+                        tma_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.n0 / 64);
+                    } else {
+                        tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, t.row0);
+                        if (KIND == ROW_BMN) tma_load_4d(b_dst, &tmB, full_bar(s), 0, kb * BK, t.n0 / 64, t.e);
+                        else tma_load_3d(b_dst, &tmB, full_bar(s), kb * BK, t.n0, t.e);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+            // drain: every copy this thread started must have landed before the CTA may exit
+            if (!ok)
+                for (int q = 0; q < STAGES; ++q) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(full_bar(q), 0) && !mbar_try_wait(full_bar(q), 1) &&
+                           global_ns() - t0 < WAIT_LIMIT_NS) {}
+                }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        constexpr uint32_t idesc = make_idesc(KIND == WGRAD ? 1 : 0, KIND == ROW_BK ? 0 : 1);
+        int s = 0, acc = 0;
+        uint32_t ph = 0, acc_ph = 0;
+        bool ok = true;
+        for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
+            Tile t;
+            if (!decode_tile<KIND>(p, id, t)) break;
+            if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
+            ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            for (int kb = 0; kb < t.kblocks; ++kb) {
+                ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_BYTES;
+                if (KIND == WGRAD && kb == t.kblocks - 1) {
+                    const int valid = t.row_end - (t.row0 + kb * BK);  // rows of this block inside the segment
+                    if (valid < BK) {
+                        // zero K rows [valid, BK) of A: 128-B lines, in both 64-column chunks
+                        const int lines = (BK - valid) * (BM / 64);
+                        for (int u = lane; u < lines * 8; u += 32) {
+                            const int line = u >> 3, part = u & 7;
+                            const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
+                            *reinterpret_cast<uint4 *>(smem + s * STAGE_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
+                                make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
+                if (lane == 0) {
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        uint64_t ad, bd;
+                        if (KIND == WGRAD) ad = desc_mnmajor(a_src + k * 16 * 128);
+                        else ad = desc_kmajor(a_src + k * 32);
+                        if (KIND == ROW_BK) bd = desc_kmajor(b_src + k * 32);
+                        else bd = desc_mnmajor(b_src + k * 16 * 128);
+                        tc_mma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(empty_bar(s));  // the stage may be refilled once these MMAs have read it
+                }
+                __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (ok && lane == 0) tc_commit(tfull_bar(acc));  // accumulator complete
+            __syncwarp();
+            if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter + 31 belong to this warp
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        bool ok = true;
+        for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
+            Tile t;
+            if (!decode_tile<KIND>(p, id, t)) break;
+            const int lrow = quarter * 32 + lane;
+            int64_t out_row;
+            bool row_ok;
+            bf16 *out = p.out;
+            if (KIND == WGRAD) {
+                out += (int64_t)t.e * p.M * p.N;
+                out_row = t.m0 + lrow;
+                row_ok = out_row < p.M;
+            } else {
+                out_row = (int64_t)t.row0 + lrow;
+                row_ok = out_row < t.row_end;
+            }
+            const bool have_acc = t.kblocks > 0;
+            if (have_acc) {
+                ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = t.n0 + c * 32;
+                if (col0 >= p.N) break;
+                uint32_t v[32];
+                if (have_acc) {
+                    tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
+                    tc_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                if (row_ok) {
+                    uint4 packed[4];
+                    uint4 bias_raw[4], mask_raw[4];
+                    if (p.bias) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
+                    }
+                    if (p.mask) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
+                    }
+                    const bf16 *bias_h = reinterpret_cast<const bf16 *>(bias_raw);
+                    const bf16 *mask_h = reinterpret_cast<const bf16 *>(mask_raw);
+                    __nv_bfloat162 *ph2 = reinterpret_cast<__nv_bfloat162 *>(packed);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+                        if (p.bias) { x0 += __bfloat162float(bias_h[j]); x1 += __bfloat162float(bias_h[j + 1]); }
+                        if (p.relu) { x0 = fmaxf(x0, 0.0f); x1 = fmaxf(x1, 0.0f); }
+                        if (p.mask) {
+                            if (!(__bfloat162float(mask_h[j]) > 0.0f)) x0 = 0.0f;
+                            if (!(__bfloat162float(mask_h[j + 1]) > 0.0f)) x1 = 0.0f;
+                        }
+                        ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
+                    }
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + out_row * p.N + col0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) dst[q] = packed[q];
+                }
+            }
+            if (have_acc) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// bf16 tensor map; dims innermost first, strides (bytes) for dims 1.., box per dim; 128-B swizzle
+int32_t make_map(CUtensorMap *tm, const void *base, int rank, const uint64_t *dims, const uint64_t *strides,
+                 const uint32_t *box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return MOE_ERR_CUDA;
+    cuuint64_t gdim[5], gstr[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides[i];
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gdim, gstr, bx,
+                    es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// rows x cols activations, K-major operand: box 64 (cols) x 128 (rows)
+int32_t map_rows_kmajor(CUtensorMap *tm, const void *p, int64_t rows, int64_t cols) {
+    const uint64_t dims[2] = {(uint64_t)cols, (uint64_t)rows}, str[1] = {(uint64_t)cols * 2};
+    const uint32_t box[2] = {64, BM};
+    return make_map(tm, p, 2, dims, str, box);
+}
+// rows x cols activations, MN-major operand (contraction over rows): dims (64, rows, cols/64)
+int32_t map_rows_mnmajor(CUtensorMap *tm, const void *p, int64_t rows, int64_t cols, int chunks) {
+    const uint64_t dims[3] = {64, (uint64_t)rows, (uint64_t)(cols / 64)}, str[2] = {(uint64_t)cols * 2, 128};
+    const uint32_t box[3] = {64, BK, (uint32_t)chunks};
+    return make_map(tm, p, 3, dims, str, box);
+}
+// per-expert weight [n, K, N] used as MN-major B: dims (64, K, N/64, n)
+int32_t map_weight_mnmajor(CUtensorMap *tm, const void *p, int64_t n, int64_t K, int64_t N) {
+    const uint64_t dims[4] = {64, (uint64_t)K, (uint64_t)(N / 64), (uint64_t)n};
+    const uint64_t str[3] = {(uint64_t)N * 2, 128, (uint64_t)K * N * 2};
+    const uint32_t box[4] = {64, BK, BN / 64, 1};
+    return make_map(tm, p, 4, dims, str, box);
+}
+// per-expert weight [n, N, K] used as K-major B: dims (K, N, n)
+int32_t map_weight_kmajor(CUtensorMap *tm, const void *p, int64_t n, int64_t N, int64_t K) {
+    const uint64_t dims[3] = {(uint64_t)K, (uint64_t)N, (uint64_t)n};
+    const uint64_t str[2] = {(uint64_t)K * 2, (uint64_t)N * K * 2};
+    const uint32_t box[3] = {64, BN, 1};
+    return make_map(tm, p, 3, dims, str, box);
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p,
+                                   int64_t max_tiles, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        MOE_CUDA(cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        configured = true;
+    }
+    if (max_tiles <= 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(max_tiles, sm_count());
+    grouped_gemm_kernel<KIND><<<grid, NTHREADS, SMEM_BYTES, st>>>(tmA, tmB, p);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+}  // namespace
+
+bool tc_ffn_supported(const moe_config &c) {
+    return c.act == MOE_BF16 && c.d % 64 == 0 && c.h % 64 == 0 && c.d >= 64 && c.h >= 64;
+}
+
+int64_t tc_ffn_ws_bytes(const moe_config &c) { return ((int64_t)(c.n + 1) * 4 + 255) & ~255ll; }
+
+// C[rows, N] = epilogue(A[rows, K] . B_e) over the segments; B_e = W[e] as [K, N] (transposed = false)
+// or as [N, K] read transposed (transposed = true).
+int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t *offsets, int32_t nseg, int64_t R,
+                    int32_t N, int32_t K, void *out, const void *bias, const void *mask, int relu,
+                    int32_t *tile_prefix, int32_t *status, cudaStream_t st) {
+    if (R == 0) return MOE_OK;
+    CUtensorMap tmA, tmB;
+    MOE_TRY(map_rows_kmajor(&tmA, A, R, K));
+    if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
+    else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
+    MOE_TRY(launch_tile_prefix(offsets, nseg, BM, tile_prefix, st));
+    GemmParams p;
+    p.offsets = offsets; p.tile_prefix = tile_prefix; p.nseg = nseg; p.M = 0; p.N = N; p.K = K;
+    p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
+    const int64_t max_tiles = (cdiv(R, BM) + nseg) * cdiv(N, BN);
+    return transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st);
+}
+
+// dW[e] [M, N] = A_e^T . B_e, contraction over the rows of segment e; A [R, M], B [R, N]
+int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int32_t nseg, int64_t R, int32_t M,
+                      int32_t N, void *out, int32_t *status, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, BM / 64));
+    MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, BN / 64));
+    GemmParams p;
+    p.offsets = offsets; p.tile_prefix = nullptr; p.nseg = nseg; p.M = M; p.N = N; p.K = 0;
+    p.out = (bf16 *)out; p.bias = nullptr; p.mask = nullptr; p.relu = 0; p.status = status;
+    return launch<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, BM) * cdiv(N, BN), st);
+}
+
+int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
+                      const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
+                      cudaStream_t st) {
+    const int64_t R = (int64_t)c.T * c.k;
+    int32_t *tile_prefix = static_cast<int32_t *>(ws);
+    MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st));
+    return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st);
+}
+
+int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
+                          const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
+                          void *dW2, void *db2, void *dz, float *colsum, int32_t *tile_prefix, int32_t *status_word,
+                          cudaStream_t st) {
+    const int64_t R = (int64_t)c.T * c.k;
+    MOE_TRY(launch_segment_colsum(dys, c.act, offsets, c.n, R, c.d, db2, colsum, tile_prefix, st));
+    MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st));
+    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st));
+    MOE_TRY(launch_segment_colsum(dz, c.act, offsets, c.n, R, c.h, db1, colsum, tile_prefix, st));
+    MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st));
+    return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st);
+}
+
 }  // namespace moe

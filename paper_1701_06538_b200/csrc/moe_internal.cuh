@@ -155,4 +155,9 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
                       cudaStream_t st);
 
+int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
+                          const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
+                          void *dW2, void *db2, void *dz, float *colsum, int32_t *tile_prefix, int32_t *status_word,
+                          cudaStream_t st);
+
 }  // namespace moe
