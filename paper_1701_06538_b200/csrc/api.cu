@@ -142,10 +142,21 @@ struct LossesBwdWs {
 };
 
 struct GateBwdWs {
-    float *dclean, *draw;
+    float *dclean, *draw, *partials;
+    void *dsplit, *wsplit;
+    bool tc;
     GateBwdWs(Carver &cv, const Dims &D) {
-        dclean = cv.take<float>(D.logits);
-        draw = cv.take<float>(D.logits);
+        dclean = draw = partials = nullptr;
+        dsplit = wsplit = nullptr;
+        tc = !D.hier && tc_gate_bwd_supported(D.act, (int32_t)D.d, (int32_t)D.n);
+        if (tc) {
+            dsplit = cv.take<bf16>(D.T * 6 * D.n);
+            wsplit = cv.take<bf16>(D.d * 6 * D.n);
+            partials = cv.take<float>(tc_gate_bwd_partials(D.T, (int32_t)D.d, (int32_t)D.n));
+        } else {
+            dclean = cv.take<float>(D.logits);
+            draw = cv.take<float>(D.logits);
+        }
     }
 };
 
@@ -335,11 +346,15 @@ int32_t gate_weight_grads(const Dims &D, const void *x, const float *dlogit, con
 int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const float *Wg, const float *Wnoise,
                     const float *noise, const float *clean, const float *raw_noise, const int32_t *topk_idx,
                     const float *gates, const float *kth_vals, const int32_t *kth_idx, float *dgates,
-                    const float *dload, float *dWg, float *dWnoise, float *dX_gate, Carver &cv, cudaStream_t st) {
+                    const float *dload, float *dWg, float *dWnoise, float *dX_gate, void *ws_base, Carver &cv,
+                    cudaStream_t st) {
     GateBwdWs w(cv, D);
     if (D.hier) return MOE_ERR_UNSUPPORTED;
     MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates, dload,
-                                    nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, st));
+                                    nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, w.dsplit, st));
+    if (w.tc)
+        return launch_tc_gate_bwd(x, D.T, (int32_t)D.d, (int32_t)D.n, Wg, Wnoise, w.dsplit, w.wsplit, w.partials, dWg,
+                                  dWnoise, dX_gate, status_word(ws_base), st);
     MOE_TRY(gate_weight_grads(D, x, w.dclean, Wg, D.n, dWg, dX_gate, false, st));
     return gate_weight_grads(D, x, w.draw, Wnoise, D.n, dWnoise, dX_gate, true, st);
 }
@@ -511,8 +526,9 @@ int32_t moe_gate_bwd(const moe_config *cfg, const void *x, const float *Wg, cons
     const Dims D = dims_of(cfg);
     Carver cv(ws);
     cv.take_bytes(kWsHeader);
+    MOE_TRY(reset_status(ws, as_stream(stream)));
     return do_gate_bwd(cfg, D, x, Wg, Wnoise, noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates,
-                       dload, dWg, dWnoise, dX_gate, cv, as_stream(stream));
+                       dload, dWg, dWnoise, dX_gate, ws, cv, as_stream(stream));
 }
 
 int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
@@ -566,7 +582,7 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
       MOE_TRY(do_losses_bwd(cfg, D, C.importance, C.load, C.topk_idx, B.dgates, B.dload, cv, st)); }
     { Carver cv = fresh();
       MOE_TRY(do_gate_bwd(cfg, D, x, Wg, Wnoise, noise, C.clean, C.raw_noise, C.topk_idx, C.gates, C.kth_vals,
-                          C.kth_idx, B.dgates, B.dload, dWg, dWnoise, B.dX_gate, cv, st)); }
+                          C.kth_idx, B.dgates, B.dload, dWg, dWnoise, B.dX_gate, ws, cv, st)); }
     return launch_dispatch_bwd(B.dxs, D.act, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dX_gate, nullptr, dX,
                                st);
 }

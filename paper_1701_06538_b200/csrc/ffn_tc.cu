@@ -24,6 +24,7 @@
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the CTA records
 // MOE_ERR_TIMEOUT in the workspace status word, stops issuing work, drains and frees its TMEM.
 #include <cuda.h>
+#include <string.h>
 
 #include "moe_internal.cuh"
 
@@ -42,18 +43,30 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Kind { ROW_BMN = 0, ROW_BK = 1, WGRAD = 2 };
 
+constexpr int MAX_TERMS = 8;
+
 struct GemmParams {
-    const int32_t *offsets;      // [nseg + 1] segment bounds (rows)
-    const int32_t *tile_prefix;  // ROW_*: [nseg + 1] prefix of 128-row tiles
+    const int32_t *offsets;      // [nseg + 1] segment bounds (rows); nullptr = uniform segments
+    const int32_t *tile_prefix;  // ROW_* with offsets: [nseg + 1] prefix of 128-row tiles
     int32_t nseg;
-    int32_t M;  // WGRAD: rows of the per-expert output; ROW_*: unused
+    int32_t M;  // WGRAD: rows of the per-segment output; ROW_*: unused
     int32_t N;  // output columns
-    int32_t K;  // ROW_*: contraction length; WGRAD: unused (segment rows)
+    int32_t K;  // ROW_*: contraction length of one term; WGRAD: unused (segment rows)
     bf16 *out;  // ROW_*: [R, N]; WGRAD: [nseg, M, N]
+    float *out_f32;    // if set, results are written here as float instead of `out`
     const bf16 *bias;  // [nseg, N] or nullptr
     const bf16 *mask;  // [R, N] or nullptr: result kept where mask > 0
     int32_t relu;
     int32_t *status;
+    // uniform segments (offsets == nullptr): ROW_*: one segment of R rows. WGRAD: segment s covers
+    // rows [c * rows_per_seg, min(R, (c+1) * rows_per_seg)) with c = s % segs_per_term, and reads the
+    // B columns shifted by (s / segs_per_term) * b_term_chunks chunks of 64 (split-precision terms).
+    int64_t R;
+    int32_t rows_per_seg, segs_per_term, b_term_chunks;
+    // ROW_*: the contraction is the concatenation of nterms pieces of length K; piece i reads A
+    // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
+    int32_t nterms;
+    int32_t a_term_col[MAX_TERMS], b_term_col[MAX_TERMS];
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -171,6 +184,7 @@ struct Tile {
     int32_t m0;       // WGRAD: first output row of the tile
     int32_t n0;       // first output column
     int32_t kblocks;  // number of K blocks
+    int32_t b_chunk;  // WGRAD: first 64-column chunk of B
 };
 
 template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
@@ -183,15 +197,34 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
         const int32_t rem = (int32_t)(id % per_e);
         t.m0 = (rem / tiles_n) * BM;
         t.n0 = (rem % tiles_n) * BN;
-        t.row0 = p.offsets[t.e];
-        t.row_end = p.offsets[t.e + 1];
+        t.b_chunk = t.n0 / 64;
+        if (p.offsets) {
+            t.row0 = p.offsets[t.e];
+            t.row_end = p.offsets[t.e + 1];
+        } else {
+            const int64_t c = t.e % p.segs_per_term;
+            t.row0 = (int32_t)(c * p.rows_per_seg);
+            t.row_end = (int32_t)(((c + 1) * p.rows_per_seg < p.R) ? (c + 1) * p.rows_per_seg : p.R);
+            if (t.row_end < t.row0) t.row_end = t.row0;
+            t.b_chunk += (t.e / p.segs_per_term) * p.b_term_chunks;
+        }
         t.kblocks = (t.row_end - t.row0 + BK - 1) / BK;
         return true;
     } else {
+        t.m0 = 0;
+        t.b_chunk = 0;
+        t.kblocks = p.nterms * (p.K / BK);
+        t.n0 = (int32_t)(id % tiles_n) * BN;
+        const int32_t mt = (int32_t)(id / tiles_n);
+        if (!p.offsets) {
+            if ((int64_t)mt * BM >= p.R) return false;
+            t.e = 0;
+            t.row0 = mt * BM;
+            t.row_end = (int32_t)p.R;
+            return true;
+        }
         const int32_t total_m = p.tile_prefix[p.nseg];
         if (id >= (int64_t)total_m * tiles_n) return false;
-        const int32_t mt = (int32_t)(id / tiles_n);
-        t.n0 = (int32_t)(id % tiles_n) * BN;
         int lo = 0, hi = p.nseg;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -200,8 +233,6 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
         t.e = lo;
         t.row0 = p.offsets[lo] + (mt - p.tile_prefix[lo]) * BM;
         t.row_end = p.offsets[lo + 1];
-        t.m0 = 0;
-        t.kblocks = p.K / BK;
         return true;
     }
 }
@@ -259,11 +290,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (KIND == WGRAD) {
                         const int r = t.row0 + kb * BK;
                         tma_load_3d(a_dst, &tmA, full_bar(s), 0, r, t.m0 / 64);
-                        tma_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.n0 / 64);
+                        tma_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk);
                     } else {
-                        tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, t.row0);
-                        if (KIND == ROW_BMN) tma_load_4d(b_dst, &tmB, full_bar(s), 0, kb * BK, t.n0 / 64, t.e);
-                        else tma_load_3d(b_dst, &tmB, full_bar(s), kb * BK, t.n0, t.e);
+                        const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
+                        tma_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0);
+                        if (KIND == ROW_BMN) tma_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64, t.e);
+                        else tma_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0, t.e);
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -367,7 +399,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                if (row_ok) {
+                if (row_ok && p.out_f32) {
+                    float *dstf = p.out_f32 + (KIND == WGRAD ? (int64_t)t.e * p.M * p.N : 0) + out_row * p.N + col0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        reinterpret_cast<uint4 *>(dstf)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                } else if (row_ok) {
                     uint4 packed[4];
                     uint4 bias_raw[4], mask_raw[4];
                     if (p.bias) {
@@ -477,6 +514,14 @@ int32_t map_weight_kmajor(CUtensorMap *tm, const void *p, int64_t n, int64_t N, 
     return make_map(tm, p, 3, dims, str, box);
 }
 
+GemmParams default_params() {
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.nterms = 1;
+    p.segs_per_term = 1;
+    return p;
+}
+
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -521,8 +566,8 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
     else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
     MOE_TRY(launch_tile_prefix(offsets, nseg, BM, tile_prefix, st));
-    GemmParams p;
-    p.offsets = offsets; p.tile_prefix = tile_prefix; p.nseg = nseg; p.M = 0; p.N = N; p.K = K;
+    GemmParams p = default_params();
+    p.offsets = offsets; p.tile_prefix = tile_prefix; p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
     p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
     const int64_t max_tiles = (cdiv(R, BM) + nseg) * cdiv(N, BN);
     return transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st);
@@ -534,9 +579,9 @@ int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int3
     CUtensorMap tmA, tmB;
     MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, BM / 64));
     MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, BN / 64));
-    GemmParams p;
-    p.offsets = offsets; p.tile_prefix = nullptr; p.nseg = nseg; p.M = M; p.N = N; p.K = 0;
-    p.out = (bf16 *)out; p.bias = nullptr; p.mask = nullptr; p.relu = 0; p.status = status;
+    GemmParams p = default_params();
+    p.offsets = offsets; p.nseg = nseg; p.M = M; p.N = N; p.R = R;
+    p.out = (bf16 *)out; p.status = status;
     return launch<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, BM) * cdiv(N, BN), st);
 }
 
@@ -547,6 +592,102 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
     int32_t *tile_prefix = static_cast<int32_t *>(ws);
     MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st));
     return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st);
+}
+
+// ------------------------------------------------------------------------------------------
+// Gate backward contractions on the tensor cores (no bit-exactness is required there):
+//   dW = x^T . dlogit   and   dX_gate = dlogit . [W_g | W_noise]^T
+// with the float operands split into three bf16 terms (hi + mid + lo carries 24 mantissa bits), x being
+// bf16 already. dsplit is [T, 3 * n2] = (hi | mid | lo) of the [T, n2] logit gradients (n2 = 2n: clean
+// columns then raw-noise columns), wsplit is [d, 3 * n2] likewise for [W_g | W_noise].
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) split_weights_kernel(const float *__restrict__ Wg,
+                                                            const float *__restrict__ Wn, int32_t d, int32_t n,
+                                                            bf16 *__restrict__ wsplit) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t n2 = 2 * n;
+    if (i >= (int64_t)d * n2) return;
+    const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
+    const float v = j < n ? Wg[(int64_t)q * n + j] : Wn[(int64_t)q * n + (j - n)];
+    const bf16 hi = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(hi);
+    const bf16 mid = __float2bfloat16_rn(r1);
+    const bf16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    bf16 *row = wsplit + (int64_t)q * 3 * n2;
+    row[j] = hi; row[n2 + j] = mid; row[2 * n2 + j] = lo;
+}
+
+__global__ void __launch_bounds__(256) reduce_partials_kernel(const float *__restrict__ part, int32_t nparts,
+                                                              int32_t d, int32_t n, float *__restrict__ dWg,
+                                                              float *__restrict__ dWn) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t n2 = 2 * n;
+    const int64_t total = (int64_t)d * n2;
+    if (i >= total) return;
+    double s = 0.0;
+    for (int32_t c = 0; c < nparts; ++c) s += (double)part[(int64_t)c * total + i];
+    const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
+    if (j < n) dWg[(int64_t)q * n + j] = (float)s;
+    else dWn[(int64_t)q * n + (j - n)] = (float)s;
+}
+
+bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
+    return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0;
+}
+
+static void gate_bwd_split(int64_t T, int32_t d, int32_t n, int32_t *S, int32_t *rows_per_seg) {
+    const int64_t tiles = cdiv(d, BM) * cdiv(2 * n, BN);
+    int64_t s = (2 * 148) / (3 * tiles);
+    if (s > T / 256) s = T / 256;
+    if (s < 1) s = 1;
+    int64_t rps = cdiv(cdiv(T, s), 64) * 64;
+    if (rps < 64) rps = 64;
+    *rows_per_seg = (int32_t)rps;
+    *S = (int32_t)(T > 0 ? cdiv(T, rps) : 1);
+}
+
+int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n) {
+    int32_t S, rps;
+    gate_bwd_split(T, d, n, &S, &rps);
+    return (int64_t)3 * S * d * 2 * n;
+}
+
+int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
+                           const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
+                           float *dX_gate, int32_t *status, cudaStream_t st) {
+    const int32_t n2 = 2 * n;
+    if (T == 0) {
+        MOE_CUDA(cudaMemsetAsync(dWg, 0, sizeof(float) * d * n, st));
+        MOE_CUDA(cudaMemsetAsync(dWn, 0, sizeof(float) * d * n, st));
+        return MOE_OK;
+    }
+    split_weights_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
+    MOE_LAUNCHED();
+    int32_t S, rps;
+    gate_bwd_split(T, d, n, &S, &rps);
+    {   // dW partials: contraction over the tokens, split into S row ranges x 3 precision terms
+        CUtensorMap tmA, tmB;
+        MOE_TRY(map_rows_mnmajor(&tmA, x, T, d, BM / 64));
+        MOE_TRY(map_rows_mnmajor(&tmB, dsplit, T, 3 * n2, BN / 64));
+        GemmParams p = default_params();
+        p.nseg = 3 * S; p.M = d; p.N = n2; p.R = T; p.out_f32 = partials; p.status = status;
+        p.rows_per_seg = rps; p.segs_per_term = S; p.b_term_chunks = n2 / 64;
+        MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
+        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, 3 * S, d, n, dWg, dWn);
+        MOE_LAUNCHED();
+    }
+    {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
+        CUtensorMap tmA, tmB;
+        MOE_TRY(map_rows_kmajor(&tmA, dsplit, T, 3 * n2));
+        MOE_TRY(map_weight_kmajor(&tmB, wsplit, 1, d, 3 * n2));
+        GemmParams p = default_params();
+        p.nseg = 1; p.N = d; p.K = n2; p.R = T; p.out_f32 = dX_gate; p.status = status;
+        p.nterms = 6;
+        const int32_t at[6] = {2, 0, 1, 0, 1, 0}, bt[6] = {0, 2, 1, 1, 0, 0};  // smallest products first
+        for (int i = 0; i < 6; ++i) { p.a_term_col[i] = at[i] * n2; p.b_term_col[i] = bt[i] * n2; }
+        MOE_TRY(launch<ROW_BK>(tmA, tmB, p, cdiv(T, BM) * cdiv(d, BN), st));
+    }
+    return MOE_OK;
 }
 
 int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
