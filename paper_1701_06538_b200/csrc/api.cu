@@ -118,10 +118,43 @@ struct FfnWs {
     }
 };
 
+// index tensors of the hierarchical levels, rebuilt from topk_idx where a stage needs them
+struct HierIdxWs {
+    int32_t *idx_p, *idx_s, *perm_p, *inv_perm_p, *counts_p, *offsets_p, *scratch, *tile_prefix;
+    HierIdxWs(Carver &cv, const Dims &D) {
+        idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
+        if (!D.hier) return;
+        idx_p = cv.take<int32_t>(D.T * D.k1);
+        idx_s = cv.take<int32_t>(D.T * D.k);
+        perm_p = cv.take<int32_t>(D.T * D.k1);
+        inv_perm_p = cv.take<int32_t>(D.T * D.k1);
+        counts_p = cv.take<int32_t>(D.a);
+        offsets_p = cv.take<int32_t>(D.a + 1);
+        scratch = cv.take<int32_t>(dispatch_ws_elems(D.T * D.k1, (int32_t)D.a));
+        tile_prefix = cv.take<int32_t>(D.a + 1);
+    }
+    int32_t build(const Dims &D, const int32_t *topk_idx, cudaStream_t st) {
+        MOE_TRY(launch_hier_split_idx(topk_idx, D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.b, idx_p, idx_s, st));
+        return launch_dispatch_index(idx_p, D.T * D.k1, (int32_t)D.a, perm_p, inv_perm_p, counts_p, offsets_p, scratch,
+                                     st);
+    }
+};
+
 struct LossesWs {
-    float *scratch;
-    LossesWs(Carver &cv, const Dims &D) {
+    float *scratch, *grouped;
+    HierIdxWs H;
+    int32_t *perm_e, *inv_perm_e, *counts_e, *offsets_e, *scratch_e;  // by flat expert, if the caller has none
+    LossesWs(Carver &cv, const Dims &D) : H(cv, D) {
         scratch = cv.take<float>(losses_ws_floats(D.T, (int32_t)(D.hier ? D.a : D.n)));
+        grouped = nullptr;
+        perm_e = inv_perm_e = counts_e = offsets_e = scratch_e = nullptr;
+        if (!D.hier) return;
+        grouped = cv.take<float>(grouped_sums_ws_floats(D.T * D.k1, (int32_t)D.a, (int32_t)D.b));
+        perm_e = cv.take<int32_t>(D.R);
+        inv_perm_e = cv.take<int32_t>(D.R);
+        counts_e = cv.take<int32_t>(D.n);
+        offsets_e = cv.take<int32_t>(D.n + 1);
+        scratch_e = cv.take<int32_t>(dispatch_ws_elems(D.R, (int32_t)D.n));
     }
 };
 
@@ -137,17 +170,22 @@ struct FfnBwdWs {
 };
 
 struct LossesBwdWs {
-    float *dimp;
-    LossesBwdWs(Carver &cv, const Dims &D) { dimp = cv.take<float>(D.n); }
+    float *dimp, *dload_h;
+    LossesBwdWs(Carver &cv, const Dims &D) {
+        dimp = cv.take<float>(D.n);
+        dload_h = D.hier ? cv.take<float>(D.n) : nullptr;
+    }
 };
 
 struct GateBwdWs {
-    float *dclean, *draw, *partials;
+    float *dclean, *draw, *partials, *dX_sec;
     void *dsplit, *wsplit;
     bool tc;
-    GateBwdWs(Carver &cv, const Dims &D) {
-        dclean = draw = partials = nullptr;
+    HierIdxWs H;
+    GateBwdWs(Carver &cv, const Dims &D) : H(cv, D) {
+        dclean = draw = partials = dX_sec = nullptr;
         dsplit = wsplit = nullptr;
+        if (D.hier) dX_sec = cv.take<float>(D.T * D.k1 * D.d);
         tc = !D.hier && tc_gate_bwd_supported(D.act, (int32_t)D.d, (int32_t)D.n);
         if (tc) {
             dsplit = cv.take<bf16>(D.T * 6 * D.n);
@@ -275,12 +313,32 @@ int32_t do_expert_ffn(const moe_config *c, const Dims &D, const void *xs, const 
 
 int32_t do_losses(const moe_config *c, const Dims &D, const int32_t *topk_idx, const float *gates,
                   const float *clean, const float *raw_noise, const float *kth_vals, float *importance, float *load,
-                  float *losses, Carver &cv, cudaStream_t st) {
+                  float *losses, const int32_t *perm, const int32_t *offsets, Carver &cv, cudaStream_t st) {
     LossesWs w(cv, D);
-    if (D.hier) return MOE_ERR_UNSUPPORTED;
-    MOE_TRY(launch_level_sums(topk_idx, gates, clean, raw_noise, kth_vals, D.T, (int32_t)D.n, (int32_t)D.k,
-                              importance, load, w.scratch, st));
-    return launch_cv2(importance, (int32_t)D.n, load, (int32_t)D.n, c->w_importance, c->w_load, losses, st);
+    if (!D.hier) {
+        MOE_TRY(launch_level_sums(topk_idx, gates, clean, raw_noise, kth_vals, D.T, (int32_t)D.n, (int32_t)D.k,
+                                  importance, load, w.scratch, st));
+        return launch_cv2(importance, (int32_t)D.n, load, (int32_t)D.n, c->w_importance, c->w_load, losses, st);
+    }
+    // Eq. 13: Importance_H = batch sum of the product gates per expert (ordered sum over each expert's rows)
+    if (!perm) {
+        MOE_TRY(launch_dispatch_index(topk_idx, D.R, (int32_t)D.n, w.perm_e, w.inv_perm_e, w.counts_e, w.offsets_e,
+                                      w.scratch_e, st));
+        perm = w.perm_e;
+        offsets = w.offsets_e;
+    }
+    MOE_TRY(launch_segment_sum(gates, perm, offsets, (int32_t)D.n, importance, st));
+    // Eq. 14: Load_primary, the per-group Load_i over X^(i), |X^(i)|
+    MOE_TRY(w.H.build(D, topk_idx, st));
+    const int64_t ab = D.a * D.b, lp = D.T * D.a;
+    float *load_p = load + ab, *load_s = load_p + D.a;
+    MOE_TRY(launch_level_sums(w.H.idx_p, gates + D.T * D.k, clean, raw_noise, kth_vals, D.T, (int32_t)D.a,
+                              (int32_t)D.k1, nullptr, load_p, w.scratch, st));
+    MOE_TRY(launch_grouped_load(w.H.idx_s, clean + lp, raw_noise + lp, kth_vals + 2 * D.T, w.H.perm_p, w.H.offsets_p,
+                                (int32_t)D.a, D.T * D.k1, (int32_t)D.b, (int32_t)D.k2, load_s, w.grouped,
+                                w.H.tile_prefix, st));
+    MOE_TRY(launch_load_h(load, w.H.counts_p, (int32_t)D.a, (int32_t)D.b, st));
+    return launch_cv2(importance, (int32_t)ab, load, (int32_t)ab, c->w_importance, c->w_load, losses, st);
 }
 
 int32_t do_expert_ffn_bwd(const moe_config *c, const Dims &D, const void *xs, const void *hid, const void *dys,
@@ -318,9 +376,13 @@ int32_t do_expert_ffn_bwd(const moe_config *c, const Dims &D, const void *xs, co
 int32_t do_losses_bwd(const moe_config *c, const Dims &D, const float *importance, const float *load,
                       const int32_t *topk_idx, float *dgates, float *dload, Carver &cv, cudaStream_t st) {
     LossesBwdWs w(cv, D);
-    if (D.hier) return MOE_ERR_UNSUPPORTED;
-    return launch_losses_bwd_flat(importance, load, (int32_t)D.n, topk_idx, D.R, c->w_importance, c->w_load, dgates,
-                                  dload, w.dimp, st);
+    if (!D.hier)
+        return launch_losses_bwd_flat(importance, load, (int32_t)D.n, topk_idx, D.R, c->w_importance, c->w_load,
+                                      dgates, dload, w.dimp, st);
+    MOE_TRY(launch_cv2_grad(importance, (int32_t)D.n, c->w_importance, w.dimp, st));
+    MOE_TRY(launch_add_gathered(dgates, topk_idx, w.dimp, D.R, st));
+    MOE_TRY(launch_cv2_grad(load, (int32_t)D.n, c->w_load, w.dload_h, st));  // load[0 : a*b] is Load_H
+    return launch_load_h_bwd(load, w.dload_h, (int32_t)D.a, (int32_t)D.b, dload, st);
 }
 
 // dW = x^T . dlogit [d, n];  dX (+)= dlogit . W^T [T, d]
@@ -349,7 +411,45 @@ int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const flo
                     const float *dload, float *dWg, float *dWnoise, float *dX_gate, void *ws_base, Carver &cv,
                     cudaStream_t st) {
     GateBwdWs w(cv, D);
-    if (D.hier) return MOE_ERR_UNSUPPORTED;
+    if (D.hier) {
+        const int64_t P1 = D.T * D.k1, lp = D.T * D.a, wp = D.d * D.a;
+        const float *g_p = gates + D.T * D.k, *g_s = g_p + P1;
+        float *dg_p = dgates + D.T * D.k, *dg_s = dg_p + P1;
+        float *dc_p = w.dclean, *dr_p = w.draw, *dc_s = w.dclean + lp, *dr_s = w.draw + lp;
+        MOE_TRY(w.H.build(D, topk_idx, st));
+        MOE_TRY(launch_hier_gate_product_bwd(gates, dgates, D.T, (int32_t)D.k1, (int32_t)D.k2, st));
+        // primary gate (Eq. 12: G_primary), rows = tokens
+        MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, w.H.idx_p, g_p, kth_vals, kth_idx, dg_p, dload,
+                                        nullptr, D.T, (int32_t)D.a, (int32_t)D.k1, dc_p, dr_p, nullptr, st));
+        MOE_TRY(gate_weight_grads(D, x, dc_p, Wg, D.a, dWg, dX_gate, false, st));
+        MOE_TRY(gate_weight_grads(D, x, dr_p, Wnoise, D.a, dWnoise, dX_gate, true, st));
+        // secondary gates G_i, rows = slots (t, s1); dLoad_i of the row's group
+        MOE_TRY(launch_gate_logit_grads(noise + lp, clean + lp, raw_noise + lp, w.H.idx_s, g_s, kth_vals + 2 * D.T,
+                                        kth_idx + 2 * D.T, dg_s, dload + D.a, w.H.idx_p, P1, (int32_t)D.b,
+                                        (int32_t)D.k2, dc_s, dr_s, nullptr, st));
+        for (int part = 0; part < 2; ++part) {
+            const float *dl = part == 0 ? dc_s : dr_s;
+            const float *W = (part == 0 ? Wg : Wnoise) + wp;
+            float *dW = (part == 0 ? dWg : dWnoise) + wp;
+            SimtGemm g;  // dW_s[i] = sum over the slots of group i of x[token]^T . dlogit[slot]
+            memset(&g, 0, sizeof(g));
+            g.ta = D.act == MOE_BF16 ? G_BF16 : G_F32; g.tb = G_F32; g.tc = G_F32;
+            g.A = x; g.B = dl; g.C = dW;
+            g.sa_i = 1; g.sa_k = D.d; g.sb_k = D.b; g.sb_j = 1; g.sc_i = D.b; g.sc_j = 1;
+            g.mode = 1; g.offsets = w.H.offsets_p; g.nseg = (int32_t)D.a; g.M = D.d; g.N = D.b; g.c_e = D.d * D.b;
+            g.a_row_index = w.H.perm_p; g.a_row_div = (int32_t)D.k1; g.b_row_index = w.H.perm_p;
+            MOE_TRY(launch_simt_gemm(g, w.H.tile_prefix, st));
+            memset(&g, 0, sizeof(g));  // dX_sec[slot] (+)= dlogit[slot] . W_s[group]^T
+            g.ta = g.tb = g.tc = G_F32;
+            g.A = dl; g.B = W; g.C = w.dX_sec; g.accumulate = part;
+            g.sa_i = D.b; g.sa_k = 1; g.sb_k = 1; g.sb_j = D.b; g.sc_i = D.d; g.sc_j = 1;
+            g.mode = 0; g.offsets = w.H.offsets_p; g.nseg = (int32_t)D.a; g.M = P1; g.N = D.d; g.K = D.b;
+            g.b_e = D.d * D.b;
+            g.a_row_index = w.H.perm_p; g.a_row_div = 1; g.c_row_index = w.H.perm_p;
+            MOE_TRY(launch_simt_gemm(g, w.H.tile_prefix, st));
+        }
+        return launch_add_slot_rows(w.dX_sec, D.T, (int32_t)D.k1, (int32_t)D.d, dX_gate, st);
+    }
     MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates, dload,
                                     nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, w.dsplit, st));
     if (w.tc)
@@ -473,7 +573,7 @@ int32_t moe_losses(const moe_config *cfg, const int32_t *topk_idx, const float *
     const Dims D = dims_of(cfg);
     Carver cv(ws);
     cv.take_bytes(kWsHeader);
-    return do_losses(cfg, D, topk_idx, gates, clean, raw_noise, kth_vals, importance, load, losses, cv,
+    return do_losses(cfg, D, topk_idx, gates, clean, raw_noise, kth_vals, importance, load, losses, nullptr, nullptr, cv,
                      as_stream(stream));
 }
 
@@ -551,7 +651,7 @@ int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const
     MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st));
     { Carver cv = fresh();
       MOE_TRY(do_losses(cfg, D, C.topk_idx, C.gates, C.clean, C.raw_noise, C.kth_vals, C.importance, C.load,
-                        C.losses, cv, st)); }
+                        C.losses, C.perm, C.offsets, cv, st)); }
     MOE_CUDA(cudaMemcpyAsync(losses, C.losses, 2 * sizeof(float), cudaMemcpyDeviceToDevice, st));
     MOE_CUDA(cudaMemcpyAsync(importance, C.importance, D.n * sizeof(float), cudaMemcpyDeviceToDevice, st));
     MOE_CUDA(cudaMemcpyAsync(load, C.load, D.load * sizeof(float), cudaMemcpyDeviceToDevice, st));

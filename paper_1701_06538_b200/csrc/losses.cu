@@ -151,6 +151,19 @@ __global__ void add_gathered_kernel(float *dgates, const int32_t *topk_idx, cons
     if (p < R) dgates[p] += dimp[topk_idx[p]];
 }
 
+int32_t launch_cv2_grad(const float *v, int32_t m, float scale, float *out, cudaStream_t st) {
+    cv2_grad_kernel<<<1, 256, 0, st>>>(v, m, scale, out);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, cudaStream_t st) {
+    if (R == 0) return MOE_OK;
+    add_gathered_kernel<<<(unsigned)cdiv(R, 256), 256, 0, st>>>(dgates, topk_idx, dimp, R);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
 int32_t launch_losses_bwd_flat(const float *importance, const float *load, int32_t n, const int32_t *topk_idx,
                                int64_t R, float w_imp, float w_load, float *dgates, float *dload, float *dimp_tmp,
                                cudaStream_t st) {

@@ -107,6 +107,24 @@ int32_t launch_losses_bwd_flat(const float *importance, const float *load, int32
                                int64_t R, float w_imp, float w_load, float *dgates, float *dload, float *dimp_tmp,
                                cudaStream_t st);
 
+// ----------------------------------------------------------------------------- hierarchical pieces (hier.cu)
+int32_t launch_hier_split_idx(const int32_t *topk_idx, int64_t T, int32_t k1, int32_t k2, int32_t b, int32_t *idx_p,
+                              int32_t *idx_s, cudaStream_t st);
+int32_t launch_segment_sum(const float *vals, const int32_t *perm, const int32_t *offsets, int32_t nseg, float *out,
+                           cudaStream_t st);
+int64_t grouped_sums_ws_floats(int64_t rows, int32_t nseg, int32_t n);
+int32_t launch_grouped_load(const int32_t *idx_s, const float *clean, const float *raw, const float *kth_vals,
+                            const int32_t *perm, const int32_t *offsets, int32_t nseg, int64_t rows, int32_t n,
+                            int32_t k, float *out, float *scratch, int32_t *tile_prefix, cudaStream_t st);
+int32_t launch_load_h(float *load, const int32_t *counts_p, int32_t a, int32_t b, cudaStream_t st);
+int32_t launch_load_h_bwd(const float *load, const float *dload_h, int32_t a, int32_t b, float *dload,
+                          cudaStream_t st);
+int32_t launch_hier_gate_product_bwd(const float *gates, float *dgates, int64_t T, int32_t k1, int32_t k2,
+                                     cudaStream_t st);
+int32_t launch_add_slot_rows(const float *dX_sec, int64_t T, int32_t k1, int32_t d, float *dX_gate, cudaStream_t st);
+int32_t launch_cv2_grad(const float *v, int32_t m, float scale, float *out, cudaStream_t st);
+int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, cudaStream_t st);
+
 // ----------------------------------------------------------------------------- gate backward (gate_bwd.cu)
 // dclean, draw [rows, n] from the saved gate tensors; dload_row_stride = 0 broadcasts dload [n].
 int32_t launch_gate_logit_grads(const float *noise, const float *clean, const float *raw, const int32_t *idx,

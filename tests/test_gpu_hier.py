@@ -1,0 +1,113 @@
+"""Hierarchical mixture of experts (Appendix B): stage-wise and fused parity against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_1701_06538_b200 import binding as B
+from paper_1701_06538_b200 import synth
+
+from helpers import (TOL_F32, act_empty, assert_close, cat_parts, cfg_of, dev, dev_act, device_inputs, f32, host, i32,
+                     oracle_run, prec_of, small_workload, tol_act)
+
+pytestmark = pytest.mark.gpu
+
+HIER = [
+    small_workload("hier-f32", T=300, d=32, h=24, n=30, k=4, a=5, k1=2, b=6, k2=2, seed=31),
+    small_workload("hier-k1-eq-a-f32", T=150, d=16, h=16, n=12, k=3, a=1, k1=1, b=12, k2=3, seed=32),
+    small_workload("hier-bf16", T=1000, d=64, h=128, n=64, k=4, a=8, k1=2, b=8, k2=2, act="bf16", seed=33),
+    small_workload("hier-wide-bf16", T=777, d=128, h=64, n=96, k=6, a=3, k1=2, b=32, k2=3, act="bf16", seed=34),
+]
+
+
+def gate_tensors(G):
+    """Oracle gate state in the ABI's layouts (primary part then secondary part)."""
+    P, S = G.primary, G.secondary
+    return dict(topk_idx=G.idx, gates=cat_parts((G.gates, P.gates, S.gates)), clean=cat_parts((P.clean, S.clean)),
+                raw=cat_parts((P.raw, S.raw)), kth_vals=cat_parts((P.kth_val, S.kth_val)),
+                kth_idx=np.concatenate([P.kth_idx.reshape(-1), S.kth_idx.reshape(-1)]).astype(np.int32))
+
+
+@pytest.fixture(scope="module", params=HIER, ids=lambda w: w.name)
+def case(request):
+    w = request.param
+    I = synth.make_all(w)
+    F, Bk = oracle_run(w, I)
+    return w, I, F, Bk, device_inputs(w, I), cfg_of(w)
+
+
+def test_hier_gate(case):
+    w, I, F, _, D, cfg = case
+    S = B.moe_query_sizes(cfg)
+    ws = B.empty_bytes(S.ws_bytes)
+    idx, gates = i32(w.T, w.k), f32(S.gates_elems)
+    clean, raw = f32(S.logits_elems), f32(S.logits_elems)
+    kv, ki = f32(S.kth_elems), i32(S.kth_elems)
+    B.moe_gate(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], idx, gates, clean, raw, kv, ki, ws)
+    want = gate_tensors(F.G)
+    assert (host(idx) == want["topk_idx"]).all(), "hierarchical routing must be bit-exact"
+    assert (host(clean) == want["clean"]).all() and (host(raw) == want["raw"]).all()
+    assert (host(ki) == want["kth_idx"]).all() and (host(kv) == want["kth_vals"]).all()
+    assert_close(host(gates), want["gates"], TOL_F32, "gates")
+
+
+def test_hier_losses_and_backward_stages(case):
+    w, I, F, Bk, D, cfg = case
+    S = B.moe_query_sizes(cfg)
+    ws = B.empty_bytes(S.ws_bytes)
+    G = gate_tensors(F.G)
+    imp, load, L = f32(w.n), f32(S.load_elems), f32(2)
+    B.moe_losses(cfg, dev(G["topk_idx"]), dev(G["gates"]), dev(G["clean"]), dev(G["raw"]), dev(G["kth_vals"]), imp,
+                 load, L, ws)
+    ab = w.a * w.b
+    LS = F.LS
+    want_load = np.concatenate([np.asarray(LS.load, np.float64), LS.load_p, LS.load_s.reshape(-1), LS.cnt])
+    assert_close(host(imp), LS.importance, TOL_F32, "importance_H")
+    assert_close(host(load)[:ab], want_load[:ab], TOL_F32, "load_H")
+    assert_close(host(load)[ab:], want_load[ab:], TOL_F32, "load levels")
+    assert_close(host(L), LS.losses, dict(max=2e-4, mean=2e-4), "losses")
+    # losses backward + gate backward, fed with the oracle's upstream gradients
+    prec = prec_of(w)
+    dI = w.w_importance * O.cv_squared_grad(LS.importance)
+    dLH = (w.w_load * O.cv_squared_grad(LS.load)).reshape(w.a, w.b)
+    safe = np.where(LS.cnt > 0, LS.cnt, 1.0)
+    live = (LS.cnt > 0)[:, None]
+    want_dload = np.concatenate([np.where(live, dLH * LS.load_s / safe[:, None], 0).sum(1),
+                                 np.where(live, dLH * LS.load_p[:, None] / safe[:, None], 0).reshape(-1)])
+    dg = torch.zeros(S.gates_elems, device="cuda")
+    dg[:w.T * w.k] = dev(np.asarray(Bk.dgates, np.float32)).reshape(-1)
+    dload = f32(S.dload_elems)
+    B.moe_losses_bwd(cfg, imp, load, dev(G["topk_idx"]), dg, dload, ws)
+    assert_close(host(dg)[:w.T * w.k], (np.asarray(Bk.dgates, np.float64) + dI[F.G.idx]).reshape(-1), TOL_F32, "dgates")
+    assert_close(host(dload), want_dload, dict(max=2e-4, mean=2e-4), "dload")
+    GB = O.gate_h_bwd(I["x"], I["Wg"][0], I["Wnoise"][0], I["noise"][0], I["Wg"][1], I["Wnoise"][1], I["noise"][1], F.G,
+                      LS, Bk.dgates, w.w_importance, w.w_load, prec)
+    dWg, dWn, dXg = f32(S.wg_elems), f32(S.wg_elems), f32(w.T, w.d)
+    B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], dev(G["clean"]), dev(G["raw"]), dev(G["topk_idx"]),
+                   dev(G["gates"]), dev(G["kth_vals"]), dev(G["kth_idx"]), dg, dload, dWg, dWn, dXg, ws)
+    tol = dict(max=5e-5, mean=1e-5)  # dload carries the CV^2 amplification of the load error
+    assert_close(host(dWg), cat_parts((GB.dWg_p, GB.dWg_s)), tol, "dWg")
+    assert_close(host(dWn), cat_parts((GB.dWn_p, GB.dWn_s)), tol, "dWnoise")
+    assert_close(host(dXg), GB.dX_gate, tol, "dX_gate")
+
+
+def test_hier_fused(case):
+    from test_gpu_fused import run_fused
+    w, I, F, Bk, D, cfg = case
+    G = run_fused(w, I)
+    V = G["ctx"]
+    want = gate_tensors(F.G)
+    assert (host(V["topk_idx"]) == F.G.idx).all()
+    assert (host(V["perm"]) == F.D.perm).all() and (host(G["counts"]) == F.D.counts).all()
+    assert_close(host(V["gates"]), want["gates"], TOL_F32, "gates")
+    assert_close(host(G["importance"]), F.LS.importance, TOL_F32, "importance")
+    assert_close(host(G["load"])[:w.n], F.LS.load, TOL_F32, "load")
+    assert_close(host(G["losses"]), F.LS.losses, dict(max=2e-4, mean=2e-4), "losses")
+    tol = tol_act(w) if w.act == "bf16" else dict(max=5e-5, mean=1e-5)
+    assert_close(host(G["y"]), F.y, tol_act(w), "y")
+    hid = host(V["hid"])
+    if ((hid > 0) == (np.asarray(F.hid) > 0)).all():  # no ReLU decision within rounding of zero
+        for name in ("dW1", "db1", "dW2", "db2", "dX"):
+            assert_close(host(G[name]), getattr(Bk, name), tol, name)
+    assert_close(host(G["dWg"]), cat_parts(Bk.dWg), tol, "dWg")
+    assert_close(host(G["dWnoise"]), cat_parts(Bk.dWnoise), tol, "dWnoise")
