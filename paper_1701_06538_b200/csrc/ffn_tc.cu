@@ -63,6 +63,7 @@ struct GemmParams {
     // B columns shifted by (s / segs_per_term) * b_term_chunks chunks of 64 (split-precision terms).
     int64_t R;
     int32_t rows_per_seg, segs_per_term, b_term_chunks;
+    int32_t segs_term0, rows_per_seg0;  // if segs_term0 > 0: term 0 is cut into that many ranges of rows_per_seg0
     // ROW_*: the contraction is the concatenation of nterms pieces of length K; piece i reads A
     // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
     int32_t nterms;
@@ -202,11 +203,19 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
             t.row0 = p.offsets[t.e];
             t.row_end = p.offsets[t.e + 1];
         } else {
-            const int64_t c = t.e % p.segs_per_term;
-            t.row0 = (int32_t)(c * p.rows_per_seg);
-            t.row_end = (int32_t)(((c + 1) * p.rows_per_seg < p.R) ? (c + 1) * p.rows_per_seg : p.R);
+            int64_t c, rps;
+            int32_t term;
+            if (t.e < p.segs_term0) {  // term 0 may use its own (shorter) row ranges
+                c = t.e; rps = p.rows_per_seg0; term = 0;
+            } else {
+                const int32_t e2 = t.e - p.segs_term0;
+                c = e2 % p.segs_per_term; rps = p.rows_per_seg;
+                term = e2 / p.segs_per_term + (p.segs_term0 > 0 ? 1 : 0);
+            }
+            t.row0 = (int32_t)(c * rps);
+            t.row_end = (int32_t)(((c + 1) * rps < p.R) ? (c + 1) * rps : p.R);
             if (t.row_end < t.row0) t.row_end = t.row0;
-            t.b_chunk += (t.e / p.segs_per_term) * p.b_term_chunks;
+            t.b_chunk += term * p.b_term_chunks;
         }
         t.kblocks = (t.row_end - t.row0 + BK - 1) / BK;
         return true;
@@ -635,21 +644,20 @@ bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
     return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0;
 }
 
-static void gate_bwd_split(int64_t T, int32_t d, int32_t n, int32_t *S, int32_t *rows_per_seg) {
-    const int64_t tiles = cdiv(d, BM) * cdiv(2 * n, BN);
-    int64_t s = (2 * 148) / (3 * tiles);
-    if (s > T / 256) s = T / 256;
-    if (s < 1) s = 1;
-    int64_t rps = cdiv(cdiv(T, s), 64) * 64;
-    if (rps < 64) rps = 64;
-    *rows_per_seg = (int32_t)rps;
-    *S = (int32_t)(T > 0 ? cdiv(T, rps) : 1);
+// Row ranges of the partial sums of dW. Short on purpose for the leading (hi) term: an fp32 accumulator
+// loses low bits when a long run of same-sign terms is added (e.g. the gradient of a constant input
+// feature); 128 rows per partial keeps that below 1e-5 of the result, and the partials are added in double.
+// The mid and lo terms are 2^-8 and 2^-16 of the hi term and can use long ranges.
+constexpr int GB_ROWS_HI = 128, GB_ROWS_LO = 2048;
+static void gate_bwd_split(int64_t T, int32_t *S_hi, int32_t *S_lo) {
+    *S_hi = (int32_t)(T > 0 ? cdiv(T, GB_ROWS_HI) : 1);
+    *S_lo = (int32_t)(T > 0 ? cdiv(T, GB_ROWS_LO) : 1);
 }
 
 int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n) {
-    int32_t S, rps;
-    gate_bwd_split(T, d, n, &S, &rps);
-    return (int64_t)3 * S * d * 2 * n;
+    int32_t S_hi, S_lo;
+    gate_bwd_split(T, &S_hi, &S_lo);
+    return (int64_t)(S_hi + 2 * S_lo) * d * 2 * n;
 }
 
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
@@ -663,17 +671,18 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
     }
     split_weights_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
     MOE_LAUNCHED();
-    int32_t S, rps;
-    gate_bwd_split(T, d, n, &S, &rps);
-    {   // dW partials: contraction over the tokens, split into S row ranges x 3 precision terms
+    int32_t S_hi, S_lo;
+    gate_bwd_split(T, &S_hi, &S_lo);
+    {   // dW partials: contraction over the tokens, cut into row ranges, one set per precision term
         CUtensorMap tmA, tmB;
         MOE_TRY(map_rows_mnmajor(&tmA, x, T, d, BM / 64));
         MOE_TRY(map_rows_mnmajor(&tmB, dsplit, T, 3 * n2, BN / 64));
         GemmParams p = default_params();
-        p.nseg = 3 * S; p.M = d; p.N = n2; p.R = T; p.out_f32 = partials; p.status = status;
-        p.rows_per_seg = rps; p.segs_per_term = S; p.b_term_chunks = n2 / 64;
+        p.nseg = S_hi + 2 * S_lo; p.M = d; p.N = n2; p.R = T; p.out_f32 = partials; p.status = status;
+        p.segs_term0 = S_hi; p.rows_per_seg0 = GB_ROWS_HI;
+        p.rows_per_seg = GB_ROWS_LO; p.segs_per_term = S_lo; p.b_term_chunks = n2 / 64;
         MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
-        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, 3 * S, d, n, dWg, dWn);
+        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, S_hi + 2 * S_lo, d, n, dWg, dWn);
         MOE_LAUNCHED();
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction

@@ -1,0 +1,145 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times (fused calls).
+
+The oracle cannot run the expert GEMMs of these batches in reasonable time, so:
+  - everything integer (routing, order statistics, dispatch permutation, counts) and every gating
+    tensor (gates, Importance, Load, losses) is compared IN FULL: the oracle's gate and loss code
+    handles the whole batch;
+  - expert-side outputs are compared on samples the oracle computes one by one: y and dX of sampled
+    tokens (each token's experts are evaluated on that token alone, which is exact because the
+    experts act row by row), and the complete weight / bias gradients of two small experts
+    (every row of those experts is evaluated);
+  - the gate backward is compared in full through its stage call, fed with the oracle's gate state.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle import moe_oracle as O
+from paper_1701_06538_b200 import binding as B
+from paper_1701_06538_b200 import synth
+
+from helpers import TOL_BF16, TOL_F32, assert_close, cat_parts, f32, host
+from test_gpu_hier import gate_tensors
+
+pytestmark = pytest.mark.gpu
+
+N_TOKENS = 48
+
+
+def slice_gate(G, rows):
+    from types import SimpleNamespace as NS
+    return NS(**{k: getattr(G, k)[rows] for k in ("idx", "gates", "clean", "raw", "sigma", "H", "kth_val", "kth_idx")})
+
+
+@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+def test_full_size_fused(name):
+    w = synth.CONFIGS[name]
+    cfg, S, D, hostI = bench.build_device_state(w, keep_host_experts=False)
+    B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], D["y"],
+                  D["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+    B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], D["ctx"],
+                   D["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"], D["db2"], D["ws"])
+    assert B.moe_check_status(D["ws"]) == 0
+    V = B.ctx_views(cfg, D["ctx"])
+    x, dY = hostI["x"], hostI["dY"]
+    Wg, Wn, noise = hostI["Wg"], hostI["Wnoise"], hostI["noise"]
+    hier = w.hier
+    # ---------------- gating, in full
+    if hier is None:
+        G = O.gate(x, Wg, Wn, noise, w.k, "bf16")
+        LS = O.losses(G.idx, G.gates, G.clean, G.raw, G.kth_val, w.w_importance, w.w_load, "bf16")
+        want_gates, want_kidx = G.gates.reshape(-1), G.kth_idx.reshape(-1)
+    else:
+        G = O.gate_h(x, Wg[0], Wn[0], noise[0], Wg[1], Wn[1], noise[1], w.k1, w.k2, "bf16")
+        LS = O.losses_h(G, w.a, w.b, w.w_importance, w.w_load, "bf16")
+        GT = gate_tensors(G)
+        want_gates, want_kidx = GT["gates"], GT["kth_idx"]
+    Dp = O.dispatch(np.zeros((w.T, 1), np.float32), G.idx, w.n)
+    assert (host(V["topk_idx"]) == G.idx).all(), "routing must be bit-exact"
+    assert (host(V["kth_idx"]).reshape(-1) == want_kidx).all()
+    assert (host(D["counts"]) == Dp.counts).all() and (host(V["offsets"]) == Dp.offsets).all()
+    assert (host(V["perm"]) == Dp.perm).all() and (host(V["inv_perm"]) == Dp.inv_perm).all()
+    assert_close(host(V["gates"]), want_gates, TOL_F32, "gates")
+    assert_close(host(D["importance"]), LS.importance, TOL_F32, "importance")
+    assert_close(host(D["load"])[:w.n], LS.load, TOL_F32, "load")
+    assert_close(host(D["losses"]), LS.losses, dict(max=2e-4, mean=2e-4), "losses")
+    xs_rows = host(V["xs"][torch.from_numpy(np.arange(0, S.R, max(1, S.R // 97))).cuda()])
+    assert (xs_rows == x[Dp.perm[np.arange(0, S.R, max(1, S.R // 97))] // w.k]).all()
+
+    # ---------------- sampled tokens: y and dX
+    g = np.random.default_rng(7)
+    first_of_big, last_of_small = Dp.perm[Dp.offsets[np.argmax(Dp.counts)]] // w.k, Dp.perm[-1] // w.k
+    toks = np.unique(np.concatenate([g.choice(w.T, N_TOKENS, replace=False), [0, w.T - 1, first_of_big, last_of_small]]))
+    experts = np.unique(G.idx[toks])
+    local = {int(e): i for i, e in enumerate(experts)}
+    Wl = [synth.make_expert(w, int(e)) for e in experts]
+    W1, b1, W2, b2 = (np.stack([p[i] for p in Wl]) for i in range(4))
+    idx_l = np.vectorize(local.get)(G.idx[toks]).astype(np.int32)
+    Ds = O.dispatch(x[toks], idx_l, len(experts))
+    hid, ys = O.expert_ffn(Ds.xs, Ds.offsets, W1, b1, W2, b2, "bf16")
+    y = O.combine(ys, G.gates[toks], Ds.inv_perm, "bf16")
+    assert_close(host(D["y"])[toks], y, TOL_BF16, "y (sampled tokens)")
+    dg, dys = O.combine_bwd(dY[toks], ys, G.gates[toks], Ds.inv_perm, "bf16")
+    E = O.expert_ffn_bwd(Ds.xs, hid, dys, Ds.offsets, W1, W2, "bf16")
+    dX_exp = O.dispatch_bwd(E.dxs, Ds.inv_perm, len(toks), w.k, "bf16")
+    if hier is None:
+        dg2, dload = O.losses_bwd(LS.importance, LS.load, G.idx[toks], dg, w.w_importance, w.w_load, "bf16")
+        dc, dr = O.gate_logit_grads(noise[toks], G.clean[toks], G.raw[toks], G.idx[toks], G.gates[toks],
+                                    G.kth_val[toks], G.kth_idx[toks], dg2, dload, "bf16")
+        dXg = dc @ Wg.astype(np.float64).T + dr @ Wn.astype(np.float64).T
+    else:
+        from types import SimpleNamespace as NS
+        Gs = NS(idx=G.idx[toks], gates=G.gates[toks], primary=slice_gate(G.primary, toks),
+                secondary=slice_gate(G.secondary, toks))
+        GB = O.gate_h_bwd(x[toks], Wg[0], Wn[0], noise[0][toks], Wg[1], Wn[1], noise[1][toks], Gs, LS, dg,
+                          w.w_importance, w.w_load, "bf16")
+        dXg = np.asarray(GB.dX_gate, np.float64)
+    dX = O.store(np.asarray(dX_exp, np.float64) + dXg, "bf16", expert_side=True)
+    got_hid = host(V["hid"][torch.from_numpy(Dp.inv_perm.reshape(w.T, w.k)[toks].reshape(-1).astype(np.int64)).cuda()])
+    want_hid = np.asarray(hid)[Ds.inv_perm]
+    assert_close(got_hid, want_hid, TOL_BF16, "hid (sampled rows)")
+    clean_rows = ((got_hid > 0) == (want_hid > 0)).reshape(len(toks), -1).all(axis=1)  # no ReLU decision at rounding of 0
+    assert clean_rows.mean() > 0.5
+    assert_close(host(D["dX"])[toks][clean_rows], dX[clean_rows], TOL_BF16, "dX (sampled tokens)")
+
+    # ---------------- two small non-empty experts: their complete weight and bias gradients
+    order = np.argsort(Dp.counts, kind="stable")
+    small = [int(e) for e in order if Dp.counts[e] > 0][:2]
+    for e in small + [int(e) for e in order if Dp.counts[e] == 0][:1]:
+        got = {k2: host(D[k2][e]) for k2 in ("dW1", "db1", "dW2", "db2")}
+        if Dp.counts[e] == 0:
+            assert all(np.abs(v).max() == 0 for v in got.values()), "an expert without rows has zero gradients"
+            continue
+        slots = Dp.perm[Dp.offsets[e]:Dp.offsets[e + 1]]
+        t_e, s_e = slots // w.k, slots % w.k
+        We = synth.make_expert(w, e)
+        offs = np.array([0, len(slots)], np.int32)
+        hid_e, _ = O.expert_ffn(x[t_e], offs, We[0][None], We[1][None], We[2][None], We[3][None], "bf16")
+        dys_e = O.store(np.asarray(G.gates, np.float64)[t_e, s_e][:, None] * dY[t_e].astype(np.float64), "bf16", True)
+        Ee = O.expert_ffn_bwd(x[t_e], hid_e, dys_e, offs, We[0][None], We[2][None], "bf16")
+        got_hid_e = host(V["hid"][int(Dp.offsets[e]):int(Dp.offsets[e + 1])])
+        keep_cols = ((got_hid_e > 0) == (np.asarray(hid_e) > 0)).all(axis=0)
+        assert keep_cols.mean() > 0.9
+        assert_close(got["dW2"], Ee.dW2[0], TOL_BF16, f"dW2[{e}]")
+        assert_close(got["db2"], Ee.db2[0], TOL_BF16, f"db2[{e}]")
+        assert_close(got["dW1"][:, keep_cols], Ee.dW1[0][:, keep_cols], TOL_BF16, f"dW1[{e}]")
+        assert_close(got["db1"][keep_cols], Ee.db1[0][keep_cols], TOL_BF16, f"db1[{e}]")
+
+    # ---------------- gate backward in full, through its stage call, fed with the oracle's gate state
+    if hier is None:
+        gd = np.random.default_rng(8)
+        dgates = gd.standard_normal((w.T, w.k)).astype(np.float32)
+        dload = (gd.standard_normal(w.n) * 1e-3).astype(np.float32)
+        GBf = O.gate_bwd(x, Wg, Wn, noise, G.clean, G.raw, G.idx, G.gates, G.kth_val, G.kth_idx, dgates, dload, "bf16")
+        dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+        dWg, dWn, dXg_d = f32(w.d, w.n), f32(w.d, w.n), f32(w.T, w.d)
+        B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], dev(G.clean), dev(G.raw), dev(G.idx),
+                       dev(G.gates), dev(G.kth_val), dev(G.kth_idx), dev(dgates), dev(dload), dWg, dWn, dXg_d, D["ws"])
+        assert B.moe_check_status(D["ws"]) == 0
+        assert_close(host(dWg), GBf.dWg, TOL_F32, "dWg (full)")
+        assert_close(host(dWn), GBf.dWnoise, TOL_F32, "dWnoise (full)")
+        # The uneven-load workloads route a constant feature through W_g[0, :] with offsets up to ~4 while
+        # sum_j dclean_j ~ 0: that column of dX_gate is a cancelling sum, and fp32 accumulation (any order)
+        # leaves ~1e-5 of the result there; the mean error stays at the 1e-7 level.
+        assert_close(host(dXg_d), GBf.dX_gate, dict(max=5e-5, mean=1e-6), "dX_gate (full)")
