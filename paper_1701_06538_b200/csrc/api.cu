@@ -178,16 +178,25 @@ struct LossesBwdWs {
 };
 
 struct GateBwdWs {
-    float *dclean, *draw, *partials, *dX_sec;
-    void *dsplit, *wsplit;
-    bool tc;
+    float *dclean, *draw, *partials, *dX_sec, *partials_s;
+    void *dsplit, *wsplit, *dsplit_s, *wsplit_s, *xs_p;
+    bool tc, tc_hier;
     HierIdxWs H;
     GateBwdWs(Carver &cv, const Dims &D) : H(cv, D) {
-        dclean = draw = partials = dX_sec = nullptr;
-        dsplit = wsplit = nullptr;
+        dclean = draw = partials = dX_sec = partials_s = nullptr;
+        dsplit = wsplit = dsplit_s = wsplit_s = xs_p = nullptr;
         if (D.hier) dX_sec = cv.take<float>(D.T * D.k1 * D.d);
         tc = !D.hier && tc_gate_bwd_supported(D.act, (int32_t)D.d, (int32_t)D.n);
-        if (tc) {
+        tc_hier = D.hier && tc_hier_gate_bwd_supported(D.act, (int32_t)D.d, (int32_t)D.a, (int32_t)D.b);
+        if (tc_hier) {
+            dsplit = cv.take<bf16>(D.T * 6 * D.a);
+            wsplit = cv.take<bf16>(D.d * 6 * D.a);
+            partials = cv.take<float>(tc_gate_bwd_partials(D.T, (int32_t)D.d, (int32_t)D.a));
+            dsplit_s = cv.take<bf16>(D.T * D.k1 * 6 * D.b);
+            wsplit_s = cv.take<bf16>(D.a * D.d * 6 * D.b);
+            partials_s = cv.take<float>(3 * D.a * D.d * 2 * D.b);
+            xs_p = cv.take<bf16>(D.T * D.k1 * D.d);
+        } else if (tc) {
             dsplit = cv.take<bf16>(D.T * 6 * D.n);
             wsplit = cv.take<bf16>(D.d * 6 * D.n);
             partials = cv.take<float>(tc_gate_bwd_partials(D.T, (int32_t)D.d, (int32_t)D.n));
@@ -418,15 +427,34 @@ int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const flo
         float *dc_p = w.dclean, *dr_p = w.draw, *dc_s = w.dclean + lp, *dr_s = w.draw + lp;
         MOE_TRY(w.H.build(D, topk_idx, st));
         MOE_TRY(launch_hier_gate_product_bwd(gates, dgates, D.T, (int32_t)D.k1, (int32_t)D.k2, st));
+        if (w.tc_hier) {
+            // both levels on the tensor cores: split logit gradients (the secondary ones written in the
+            // order sorted by primary group), grouped products, then the slots' rows are added per token
+            MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, w.H.idx_p, g_p, kth_vals, kth_idx, dg_p, dload,
+                                            nullptr, D.T, (int32_t)D.a, (int32_t)D.k1, nullptr, nullptr, w.dsplit,
+                                            nullptr, st));
+            MOE_TRY(launch_tc_gate_bwd(x, D.T, (int32_t)D.d, (int32_t)D.a, Wg, Wnoise, w.dsplit, w.wsplit, w.partials,
+                                       dWg, dWnoise, dX_gate, status_word(ws_base), st));
+            MOE_TRY(launch_gate_logit_grads(noise + lp, clean + lp, raw_noise + lp, w.H.idx_s, g_s, kth_vals + 2 * D.T,
+                                            kth_idx + 2 * D.T, dg_s, dload + D.a, w.H.idx_p, P1, (int32_t)D.b,
+                                            (int32_t)D.k2, nullptr, nullptr, w.dsplit_s, w.H.inv_perm_p, st));
+            MOE_TRY(launch_dispatch_rows(x, D.act, D.T, (int32_t)D.k1, (int32_t)D.d, w.H.inv_perm_p, w.xs_p, st));
+            MOE_TRY(launch_tc_hier_secondary_bwd(w.xs_p, w.dsplit_s, w.wsplit_s, Wg + wp, Wnoise + wp, w.H.offsets_p,
+                                                 w.H.tile_prefix, (int32_t)D.a, P1, (int32_t)D.d, (int32_t)D.b,
+                                                 w.partials_s, dWg + wp, dWnoise + wp, w.dX_sec, status_word(ws_base),
+                                                 st));
+            return launch_dispatch_bwd(w.dX_sec, MOE_F32, w.H.inv_perm_p, D.T, (int32_t)D.k1, (int32_t)D.d, dX_gate,
+                                       dX_gate, nullptr, st);
+        }
         // primary gate (Eq. 12: G_primary), rows = tokens
         MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, w.H.idx_p, g_p, kth_vals, kth_idx, dg_p, dload,
-                                        nullptr, D.T, (int32_t)D.a, (int32_t)D.k1, dc_p, dr_p, nullptr, st));
+                                        nullptr, D.T, (int32_t)D.a, (int32_t)D.k1, dc_p, dr_p, nullptr, nullptr, st));
         MOE_TRY(gate_weight_grads(D, x, dc_p, Wg, D.a, dWg, dX_gate, false, st));
         MOE_TRY(gate_weight_grads(D, x, dr_p, Wnoise, D.a, dWnoise, dX_gate, true, st));
         // secondary gates G_i, rows = slots (t, s1); dLoad_i of the row's group
         MOE_TRY(launch_gate_logit_grads(noise + lp, clean + lp, raw_noise + lp, w.H.idx_s, g_s, kth_vals + 2 * D.T,
                                         kth_idx + 2 * D.T, dg_s, dload + D.a, w.H.idx_p, P1, (int32_t)D.b,
-                                        (int32_t)D.k2, dc_s, dr_s, nullptr, st));
+                                        (int32_t)D.k2, dc_s, dr_s, nullptr, nullptr, st));
         for (int part = 0; part < 2; ++part) {
             const float *dl = part == 0 ? dc_s : dr_s;
             const float *W = (part == 0 ? Wg : Wnoise) + wp;
@@ -451,7 +479,8 @@ int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const flo
         return launch_add_slot_rows(w.dX_sec, D.T, (int32_t)D.k1, (int32_t)D.d, dX_gate, st);
     }
     MOE_TRY(launch_gate_logit_grads(noise, clean, raw_noise, topk_idx, gates, kth_vals, kth_idx, dgates, dload,
-                                    nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, w.dsplit, st));
+                                    nullptr, D.T, (int32_t)D.n, (int32_t)D.k, w.dclean, w.draw, w.dsplit, nullptr,
+                                    st));
     if (w.tc)
         return launch_tc_gate_bwd(x, D.T, (int32_t)D.d, (int32_t)D.n, Wg, Wnoise, w.dsplit, w.wsplit, w.partials, dWg,
                                   dWnoise, dX_gate, status_word(ws_base), st);

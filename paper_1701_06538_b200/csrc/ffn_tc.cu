@@ -64,6 +64,7 @@ struct GemmParams {
     int64_t R;
     int32_t rows_per_seg, segs_per_term, b_term_chunks;
     int32_t segs_term0, rows_per_seg0;  // if segs_term0 > 0: term 0 is cut into that many ranges of rows_per_seg0
+    int32_t off_mod;                    // WGRAD with offsets: see decode_tile
     // ROW_*: the contraction is the concatenation of nterms pieces of length K; piece i reads A
     // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
     int32_t nterms;
@@ -199,9 +200,11 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
         t.m0 = (rem / tiles_n) * BM;
         t.n0 = (rem % tiles_n) * BN;
         t.b_chunk = t.n0 / 64;
-        if (p.offsets) {
-            t.row0 = p.offsets[t.e];
-            t.row_end = p.offsets[t.e + 1];
+        if (p.offsets) {  // with off_mod: segment s reads the rows of group s % off_mod, B term s / off_mod
+            const int32_t seg = p.off_mod > 0 ? t.e % p.off_mod : t.e;
+            t.row0 = p.offsets[seg];
+            t.row_end = p.offsets[seg + 1];
+            if (p.off_mod > 0) t.b_chunk += (t.e / p.off_mod) * p.b_term_chunks;
         } else {
             int64_t c, rps;
             int32_t term;
@@ -626,18 +629,20 @@ __global__ void __launch_bounds__(256) split_weights_kernel(const float *__restr
     row[j] = hi; row[n2 + j] = mid; row[2 * n2 + j] = lo;
 }
 
+// out (group g = blockIdx.y) = sum_c part[c * part_stride + g * d * 2n + .], split into the W_g and W_noise halves
 __global__ void __launch_bounds__(256) reduce_partials_kernel(const float *__restrict__ part, int32_t nparts,
-                                                              int32_t d, int32_t n, float *__restrict__ dWg,
-                                                              float *__restrict__ dWn) {
+                                                              int64_t part_stride, int32_t d, int32_t n,
+                                                              float *__restrict__ dWg, float *__restrict__ dWn) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int32_t n2 = 2 * n;
     const int64_t total = (int64_t)d * n2;
     if (i >= total) return;
+    const int64_t g = blockIdx.y;
     double s = 0.0;
-    for (int32_t c = 0; c < nparts; ++c) s += (double)part[(int64_t)c * total + i];
+    for (int32_t c = 0; c < nparts; ++c) s += (double)part[(int64_t)c * part_stride + g * total + i];
     const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
-    if (j < n) dWg[(int64_t)q * n + j] = (float)s;
-    else dWn[(int64_t)q * n + (j - n)] = (float)s;
+    if (j < n) dWg[(g * d + q) * n + j] = (float)s;
+    else dWn[(g * d + q) * n + (j - n)] = (float)s;
 }
 
 bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
@@ -682,7 +687,8 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
         p.segs_term0 = S_hi; p.rows_per_seg0 = GB_ROWS_HI;
         p.rows_per_seg = GB_ROWS_LO; p.segs_per_term = S_lo; p.b_term_chunks = n2 / 64;
         MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
-        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, S_hi + 2 * S_lo, d, n, dWg, dWn);
+        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, S_hi + 2 * S_lo, (int64_t)d * n2, d, n, dWg,
+                                                                                            dWn);
         MOE_LAUNCHED();
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
@@ -695,6 +701,47 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
         const int32_t at[6] = {2, 0, 1, 0, 1, 0}, bt[6] = {0, 2, 1, 1, 0, 0};  // smallest products first
         for (int i = 0; i < 6; ++i) { p.a_term_col[i] = at[i] * n2; p.b_term_col[i] = bt[i] * n2; }
         MOE_TRY(launch<ROW_BK>(tmA, tmB, p, cdiv(T, BM) * cdiv(d, BN), st));
+    }
+    return MOE_OK;
+}
+
+// Secondary gates of the hierarchical layer: the slots (t, s1) sorted by primary group are the rows.
+// xs_p [P1, d] token rows in sorted order, dsplit_s [P1, 3 * 2b] split logit gradients in sorted order.
+bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b) {
+    return act == MOE_BF16 && d % 64 == 0 && (2 * a) % 64 == 0 && (2 * b) % 64 == 0;
+}
+
+int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, void *wsplit_s, const float *Wg_s,
+                                     const float *Wn_s, const int32_t *offsets_p, int32_t *tile_prefix, int32_t a,
+                                     int64_t P1, int32_t d, int32_t b, float *partials, float *dWg_s, float *dWn_s,
+                                     float *dX_sec, int32_t *status, cudaStream_t st) {
+    const int32_t n2 = 2 * b;
+    split_weights_kernel<<<(unsigned)cdiv((int64_t)a * d * n2, 256), 256, 0, st>>>(Wg_s, Wn_s, a * d, b, (bf16 *)wsplit_s);
+    MOE_LAUNCHED();
+    {   // dW_s[i] = sum over the slots of group i of x[token]^T . dlogit[slot], one partial per precision term
+        CUtensorMap tmA, tmB;
+        MOE_TRY(map_rows_mnmajor(&tmA, xs_p, P1 > 0 ? P1 : 1, d, BM / 64));
+        MOE_TRY(map_rows_mnmajor(&tmB, dsplit_s, P1 > 0 ? P1 : 1, 3 * n2, BN / 64));
+        GemmParams p = default_params();
+        p.offsets = offsets_p; p.nseg = 3 * a; p.off_mod = a; p.b_term_chunks = n2 / 64;
+        p.M = d; p.N = n2; p.R = P1; p.out_f32 = partials; p.status = status;
+        MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
+        reduce_partials_kernel<<<dim3((unsigned)cdiv((int64_t)d * n2, 256), (unsigned)a), 256, 0, st>>>(
+            partials, 3, (int64_t)a * d * n2, d, b, dWg_s, dWn_s);
+        MOE_LAUNCHED();
+    }
+    if (P1 > 0) {   // dX_sec[row] = dlogit[row] . [W_g | W_noise][group]^T, six cross terms
+        CUtensorMap tmA, tmB;
+        MOE_TRY(map_rows_kmajor(&tmA, dsplit_s, P1, 3 * n2));
+        MOE_TRY(map_weight_kmajor(&tmB, wsplit_s, a, d, 3 * n2));
+        MOE_TRY(launch_tile_prefix(offsets_p, a, BM, tile_prefix, st));
+        GemmParams p = default_params();
+        p.offsets = offsets_p; p.tile_prefix = tile_prefix; p.nseg = a; p.N = d; p.K = n2; p.R = P1;
+        p.out_f32 = dX_sec; p.status = status;
+        p.nterms = 6;
+        const int32_t at[6] = {2, 0, 1, 0, 1, 0}, bt[6] = {0, 2, 1, 1, 0, 0};
+        for (int i = 0; i < 6; ++i) { p.a_term_col[i] = at[i] * n2; p.b_term_col[i] = bt[i] * n2; }
+        MOE_TRY(launch<ROW_BK>(tmA, tmB, p, (cdiv(P1, BM) + a) * cdiv(d, BN), st));
     }
     return MOE_OK;
 }

@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
     const int32_t *__restrict__ idx, const float *__restrict__ gates, const float *__restrict__ kth_vals,
     const int32_t *__restrict__ kth_idx, const float *__restrict__ dgates, const float *__restrict__ dload,
     const int32_t *__restrict__ dload_row_group, int64_t rows, int32_t n, int32_t k, float *__restrict__ dclean,
-    float *__restrict__ draw, bf16 *__restrict__ dsplit) {
+    float *__restrict__ draw, bf16 *__restrict__ dsplit, const int32_t *__restrict__ split_row_index) {
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -77,7 +77,8 @@ __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
         const float dc = q + dh, dr = dsigma / (1.0f + expf(-rj));
         if (dsplit) {
             // three-term bf16 split (hi | mid | lo), row layout [3][clean n | raw n], for the tensor-core products
-            bf16 *o = dsplit + row * (6 * (int64_t)n);
+            const int64_t orow = split_row_index ? split_row_index[row] : row;  // e.g. sorted by primary group
+            bf16 *o = dsplit + orow * (6 * (int64_t)n);
             float v = dc;
 #pragma unroll
             for (int term = 0; term < 3; ++term) {
@@ -103,11 +104,12 @@ int32_t launch_gate_logit_grads(const float *noise, const float *clean, const fl
                                 const float *gates, const float *kth_vals, const int32_t *kth_idx,
                                 const float *dgates, const float *dload, const int32_t *dload_row_group,
                                 int64_t rows, int32_t n, int32_t k, float *dclean, float *draw, void *dsplit,
-                                cudaStream_t st) {
+                                const int32_t *split_row_index, cudaStream_t st) {
     if (rows == 0) return MOE_OK;
     gate_logit_grads_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals,
                                                                        kth_idx, dgates, dload, dload_row_group,
-                                                                       rows, n, k, dclean, draw, (bf16 *)dsplit);
+                                                                       rows, n, k, dclean, draw, (bf16 *)dsplit,
+                                                                       split_row_index);
     MOE_LAUNCHED();
     return MOE_OK;
 }

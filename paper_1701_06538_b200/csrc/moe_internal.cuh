@@ -131,7 +131,7 @@ int32_t launch_gate_logit_grads(const float *noise, const float *clean, const fl
                                 const float *gates, const float *kth_vals, const int32_t *kth_idx,
                                 const float *dgates, const float *dload, const int32_t *dload_row_group,
                                 int64_t rows, int32_t n, int32_t k, float *dclean, float *draw, void *dsplit,
-                                cudaStream_t st);
+                                const int32_t *split_row_index, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- SIMT grouped GEMM (gemm_simt.cu)
 enum GemmType { G_F32 = 0, G_BF16 = 1 };
@@ -179,6 +179,11 @@ int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n);  // floats of par
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
                            float *dX_gate, int32_t *status, cudaStream_t st);
+bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b);
+int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, void *wsplit_s, const float *Wg_s,
+                                     const float *Wn_s, const int32_t *offsets_p, int32_t *tile_prefix, int32_t a,
+                                     int64_t P1, int32_t d, int32_t b, float *partials, float *dWg_s, float *dWn_s,
+                                     float *dX_sec, int32_t *status, cudaStream_t st);
 int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
                           void *dW2, void *db2, void *dz, float *colsum, int32_t *tile_prefix, int32_t *status_word,

@@ -370,8 +370,8 @@ int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const fl
 template <typename XT>
 __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict__ dxs,
                                                            const int32_t *__restrict__ inv_perm, int64_t T,
-                                                           int32_t k, int32_t d, const float *__restrict__ add,
-                                                           float *__restrict__ out_f32, XT *__restrict__ out_act) {
+                                                           int32_t k, int32_t d, const float *add,
+                                                           float *out_f32, XT *__restrict__ out_act) {
     constexpr int VN = 16 / sizeof(XT);
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);

@@ -17,6 +17,8 @@ HIER = [
     small_workload("hier-k1-eq-a-f32", T=150, d=16, h=16, n=12, k=3, a=1, k1=1, b=12, k2=3, seed=32),
     small_workload("hier-bf16", T=1000, d=64, h=128, n=64, k=4, a=8, k1=2, b=8, k2=2, act="bf16", seed=33),
     small_workload("hier-wide-bf16", T=777, d=128, h=64, n=96, k=6, a=3, k1=2, b=32, k2=3, act="bf16", seed=34),
+    # both gating levels wide enough for the tensor-core gate backward (2a and 2b multiples of 64)
+    small_workload("hier-tc-bf16", T=2100, d=64, h=64, n=1024, k=4, a=32, k1=2, b=32, k2=2, act="bf16", seed=35),
 ]
 
 
