@@ -7,7 +7,7 @@
 //   warp 1      MMA issuer: tcgen05.mma (cta_group::1, kind::f16, M 128, N 256, K 16), accumulator
 //               in TMEM, double buffered (2 x 256 columns) so the epilogue of one tile overlaps
 //               the main loop of the next; tcgen05.commit releases the stage / publishes the tile
-//   warps 2-5   epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), bias / ReLU / ReLU
+//   warps 2-9   epilogue: tcgen05.ld (32 lanes x 32 columns per instruction), bias / ReLU / ReLU
 //               mask, round to bf16, 64-byte row stores with a row guard for ragged segments
 //
 // Three operand arrangements (KIND):
@@ -24,6 +24,7 @@
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the CTA records
 // MOE_ERR_TIMEOUT in the workspace status word, stops issuing work, drains and frees its TMEM.
 #include <cuda.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "moe_internal.cuh"
@@ -36,9 +37,10 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;  // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;  // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_STAGE_BYTES = 8 * 4096;  // per epilogue warp: a 32 x 128 B slab for float output
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Kind { ROW_BMN = 0, ROW_BK = 1, WGRAD = 2 };
@@ -189,7 +191,8 @@ struct Tile {
     int32_t b_chunk;  // WGRAD: first 64-column chunk of B
 };
 
-template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
+template <int KIND, int TM = BM>
+__device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
     const int32_t tiles_n = (p.N + BN - 1) / BN;
     if (KIND == WGRAD) {
         const int32_t tiles_m = (p.M + BM - 1) / BM;
@@ -229,9 +232,9 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
         t.n0 = (int32_t)(id % tiles_n) * BN;
         const int32_t mt = (int32_t)(id / tiles_n);
         if (!p.offsets) {
-            if ((int64_t)mt * BM >= p.R) return false;
+            if ((int64_t)mt * TM >= p.R) return false;
             t.e = 0;
-            t.row0 = mt * BM;
+            t.row0 = mt * TM;
             t.row_end = (int32_t)p.R;
             return true;
         }
@@ -243,7 +246,7 @@ template <int KIND> __device__ __forceinline__ bool decode_tile(const GemmParams
             if (p.tile_prefix[mid] <= mt) lo = mid; else hi = mid;
         }
         t.e = lo;
-        t.row0 = p.offsets[lo] + (mt - p.tile_prefix[lo]) * BM;
+        t.row0 = p.offsets[lo] + (mt - p.tile_prefix[lo]) * TM;
         t.row_end = p.offsets[lo + 1];
         return true;
     }
@@ -268,7 +271,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
@@ -374,7 +377,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter + 31 belong to this warp
         int acc = 0;
         uint32_t acc_ph = 0;
@@ -382,25 +385,33 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
             Tile t;
             if (!decode_tile<KIND>(p, id, t)) break;
-            const int lrow = quarter * 32 + lane;
-            int64_t out_row;
-            bool row_ok;
-            bf16 *out = p.out;
-            if (KIND == WGRAD) {
-                out += (int64_t)t.e * p.M * p.N;
-                out_row = t.m0 + lrow;
-                row_ok = out_row < p.M;
-            } else {
-                out_row = (int64_t)t.row0 + lrow;
-                row_ok = out_row < t.row_end;
-            }
             const bool have_acc = t.kblocks > 0;
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
             }
-            for (int c = 0; c < BN / 32; ++c) {
+            // Two warps share each quarter of the accumulator's rows and take half of its columns each.
+            // A thread owns one row. bf16 results are stored straight from registers (64 B per thread and
+            // step); float results (128 B per row and step) go through a swizzled shared-memory slab so that
+            // the stores are whole 128-byte row segments: lane l moves piece l % 8 of row 4 * i + l / 8.
+            const int half = (warp - 2) >> 2;
+            uint8_t *stage_o = smem + STAGES * STAGE_BYTES + 256 + (warp - 2) * 4096;
+            int64_t tile_row0;   // first output row of this warp's 32 rows
+            int32_t rows_valid;  // how many of them exist
+            int64_t out_off = 0;
+            if (KIND == WGRAD) {
+                out_off = (int64_t)t.e * p.M * p.N;
+                tile_row0 = t.m0 + quarter * 32;
+                rows_valid = p.M - (int32_t)tile_row0;
+            } else {
+                tile_row0 = (int64_t)t.row0 + quarter * 32;
+                rows_valid = t.row_end - (int32_t)tile_row0;
+            }
+            const int my_piece = lane & 7, my_sub = lane >> 3;
+            const bool row_ok = lane < rows_valid;
+            const int64_t out_row = tile_row0 + lane;
+            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                 const int col0 = t.n0 + c * 32;
                 if (col0 >= p.N) break;
                 uint32_t v[32];
@@ -411,11 +422,20 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                if (row_ok && p.out_f32) {
-                    float *dstf = p.out_f32 + (KIND == WGRAD ? (int64_t)t.e * p.M * p.N : 0) + out_row * p.N + col0;
+                if (p.out_f32) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
-                        reinterpret_cast<uint4 *>(dstf)[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                        *reinterpret_cast<uint4 *>(stage_o + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = 4 * i + my_sub;
+                        if (row < rows_valid)
+                            *reinterpret_cast<uint4 *>(p.out_f32 + out_off + (tile_row0 + row) * p.N + col0 + my_piece * 4) =
+                                *reinterpret_cast<const uint4 *>(stage_o + row * 128 + ((my_piece ^ (row & 7)) << 4));
+                    }
+                    __syncwarp();
                 } else if (row_ok) {
                     uint4 packed[4];
                     uint4 bias_raw[4], mask_raw[4];
@@ -443,7 +463,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>(out + out_row * p.N + col0);
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) dst[q] = packed[q];
                 }
@@ -462,6 +482,259 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+    }
+}
+
+
+// ------------------------------------------------------------------------------------------
+// Two-CTA variant for the row GEMMs (ROW_BMN, ROW_BK): a cluster of two CTAs (an SM pair) works on a
+// 256 x 256 tile with tcgen05.mma cta_group::2 (M 256). Each CTA stages its own 128 rows of A and its
+// own 128 columns of B (32 KiB per stage instead of 48, six stages), the pair's tensor cores exchange
+// the B halves, and each CTA keeps the accumulator of its 128 rows in its own TMEM. The even CTA of
+// the pair issues the MMAs; the loads of both CTAs count on its "full" barrier; tcgen05.commit
+// releases a stage / publishes an accumulator in both CTAs at once; the odd CTA's epilogue warps
+// hand their accumulator buffer back with an arrive on the even CTA's barrier.
+// ------------------------------------------------------------------------------------------
+constexpr int STAGES2 = 6;
+constexpr int A2_BYTES = 128 * BK * 2, B2_BYTES = 128 * BK * 2, STAGE2_BYTES = A2_BYTES + B2_BYTES;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
+constexpr uint32_t PEER_BIT_MASK = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address of the pair
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at this shared-memory offset in the EVEN CTA of the pair
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_BIT_MASK) : "memory");
+}
+__device__ __forceinline__ void tc_commit2(uint32_t bar) {  // arrives at this offset in both CTAs of the pair
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma2_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// loads of the pair: both CTAs' transaction bytes are counted on the even CTA's barrier
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar & PEER_BIT_MASK), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1,
+                                             int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar & PEER_BIT_MASK), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1,
+                                             int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], "
+        "[%2];" ::"r"(dst), "l"(tm), "r"(bar & PEER_BIT_MASK), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__host__ __device__ constexpr uint32_t make_idesc2(int a_mn, int b_mn) {  // M 256, N 256
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(NTHREADS, 1)
+grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bars = base + STAGES2 * STAGE2_BYTES;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (STAGES2 + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + 2 + a); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES2 * STAGE2_BYTES + 8 * (2 * STAGES2 + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES2 * STAGE2_BYTES + 8 * (2 * STAGES2 + 4) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: issues the MMAs, owns the full / tempty barriers
+    const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers exist before anything is signalled across the pair
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int64_t id = cluster_id; ok; id += n_clusters) {
+                Tile t;
+                if (!decode_tile<KIND, 256>(p, id, t)) break;
+                for (int kb = 0; kb < t.kblocks && ok; ++kb) {
+                    ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    const uint32_t a_dst = base + s * STAGE2_BYTES, b_dst = a_dst + A2_BYTES;
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+                    const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
+                    tma2_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0 + 128 * (int)rank);
+                    if (KIND == ROW_BMN)
+                        tma2_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64 + 2 * (int)rank, t.e);
+                    else
+                        tma2_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0 + 128 * (int)rank, t.e);
+                    if (++s == STAGES2) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (even CTA only)
+        if (rank == 0) {
+            constexpr uint32_t idesc = make_idesc2(0, KIND == ROW_BK ? 0 : 1);
+            int s = 0, acc = 0;
+            uint32_t ph = 0, acc_ph = 0;
+            bool ok = true;
+            for (int64_t id = cluster_id; ok; id += n_clusters) {
+                Tile t;
+                if (!decode_tile<KIND, 256>(p, id, t)) break;
+                ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < t.kblocks; ++kb) {
+                    ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_src = base + s * STAGE2_BYTES, b_src = a_src + A2_BYTES;
+                    if (lane == 0) {
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k) {
+                            const uint64_t ad = desc_kmajor(a_src + k * 32);
+                            const uint64_t bd = KIND == ROW_BK ? desc_kmajor(b_src + k * 32) : desc_mnmajor(b_src + k * 16 * 128);
+                            tc_mma2_bf16(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        }
+                        tc_commit2(empty_bar(s));
+                    }
+                    __syncwarp();
+                    if (++s == STAGES2) { s = 0; ph ^= 1u; }
+                }
+                if (ok && lane == 0) tc_commit2(tfull_bar(acc));
+                __syncwarp();
+                if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        uint8_t *stage_o = smem + STAGES2 * STAGE2_BYTES + 256 + (warp - 2) * 4096;
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        bool ok = true;
+        for (int64_t id = cluster_id; ok; id += n_clusters) {
+            Tile t;
+            if (!decode_tile<KIND, 256>(p, id, t)) break;
+            ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const int64_t tile_row0 = (int64_t)t.row0 + 128 * (int)rank + quarter * 32;
+            const int32_t rows_valid = t.row_end - (int32_t)tile_row0;
+            const int my_piece = lane & 7, my_sub = lane >> 3;
+            const bool row_ok = lane < rows_valid;
+            const int64_t out_row = tile_row0 + lane;
+            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+                const int col0 = t.n0 + c * 32;
+                if (col0 >= p.N) break;
+                uint32_t v[32];
+                tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
+                tc_ld_wait();
+                if (p.out_f32) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<uint4 *>(stage_o + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                            make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = 4 * i + my_sub;
+                        if (row < rows_valid)
+                            *reinterpret_cast<uint4 *>(p.out_f32 + (tile_row0 + row) * p.N + col0 + my_piece * 4) =
+                                *reinterpret_cast<const uint4 *>(stage_o + row * 128 + ((my_piece ^ (row & 7)) << 4));
+                    }
+                    __syncwarp();
+                } else if (row_ok) {
+                    uint4 packed[4];
+                    uint4 bias_raw[4], mask_raw[4];
+                    if (p.bias) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
+                    }
+                    if (p.mask) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
+                    }
+                    const bf16 *bias_h = reinterpret_cast<const bf16 *>(bias_raw);
+                    const bf16 *mask_h = reinterpret_cast<const bf16 *>(mask_raw);
+                    __nv_bfloat162 *ph2 = reinterpret_cast<__nv_bfloat162 *>(packed);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
+                        if (p.bias) { x0 += __bfloat162float(bias_h[j]); x1 += __bfloat162float(bias_h[j + 1]); }
+                        if (p.relu) { x0 = fmaxf(x0, 0.0f); x1 = fmaxf(x1, 0.0f); }
+                        if (p.mask) {
+                            if (!(__bfloat162float(mask_h[j]) > 0.0f)) x0 = 0.0f;
+                            if (!(__bfloat162float(mask_h[j + 1]) > 0.0f)) x1 = 0.0f;
+                        }
+                        ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
+                    }
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_row * p.N + col0);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) dst[q] = packed[q];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the pair's MMAs read both CTAs' shared memory: leave together
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
                      : "memory");
     }
 }
@@ -534,6 +807,20 @@ GemmParams default_params() {
     return p;
 }
 
+// per-expert weight as B of the two-CTA kernel: each CTA of the pair loads 128 of the 256 columns
+int32_t map_weight_mnmajor_half(CUtensorMap *tm, const void *p, int64_t n, int64_t K, int64_t N) {
+    const uint64_t dims[4] = {64, (uint64_t)K, (uint64_t)(N / 64), (uint64_t)n};
+    const uint64_t str[3] = {(uint64_t)N * 2, 128, (uint64_t)K * N * 2};
+    const uint32_t box[4] = {64, BK, 2, 1};
+    return make_map(tm, p, 4, dims, str, box);
+}
+int32_t map_weight_kmajor_half(CUtensorMap *tm, const void *p, int64_t n, int64_t N, int64_t K) {
+    const uint64_t dims[3] = {(uint64_t)K, (uint64_t)N, (uint64_t)n};
+    const uint64_t str[2] = {(uint64_t)K * 2, (uint64_t)N * K * 2};
+    const uint32_t box[3] = {64, 128, 1};
+    return make_map(tm, p, 3, dims, str, box);
+}
+
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -559,6 +846,30 @@ template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tm
     return MOE_OK;
 }
 
+template <int KIND> int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p,
+                                    int64_t max_tiles, cudaStream_t st) {
+    static int max_clusters = 0;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM2_BYTES; cfg.stream = st;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    if (!max_clusters) {
+        MOE_CUDA(cudaFuncSetAttribute(grouped_gemm2_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+        cfg.gridDim = dim3(2 * (sm_count() / 2));
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, grouped_gemm2_kernel<KIND>, &cfg) != cudaSuccess || n <= 0) return MOE_ERR_CUDA;
+        max_clusters = n;
+    }
+    if (max_tiles <= 0) return MOE_OK;
+    cfg.gridDim = dim3(2 * (unsigned)imin(max_tiles, max_clusters));
+    MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND>, tmA, tmB, p));
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
 }  // namespace
 
 bool tc_ffn_supported(const moe_config &c) {
@@ -566,6 +877,13 @@ bool tc_ffn_supported(const moe_config &c) {
 }
 
 int64_t tc_ffn_ws_bytes(const moe_config &c) { return ((int64_t)(c.n + 1) * 4 + 255) & ~255ll; }
+
+// The 256-row tiles of the two-CTA kernel pay off when the average segment fills them.
+static bool use_two_cta(int64_t R, int32_t nseg) {
+    const char *env = getenv("MOE_TC_ONE_CTA");
+    if (env && env[0] == '1') return false;
+    return R / (nseg > 0 ? nseg : 1) >= 384;
+}
 
 // C[rows, N] = epilogue(A[rows, K] . B_e) over the segments; B_e = W[e] as [K, N] (transposed = false)
 // or as [N, K] read transposed (transposed = true).
@@ -575,12 +893,19 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     if (R == 0) return MOE_OK;
     CUtensorMap tmA, tmB;
     MOE_TRY(map_rows_kmajor(&tmA, A, R, K));
-    if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
-    else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
-    MOE_TRY(launch_tile_prefix(offsets, nseg, BM, tile_prefix, st));
     GemmParams p = default_params();
     p.offsets = offsets; p.tile_prefix = tile_prefix; p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
     p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
+    if (use_two_cta(R, nseg)) {  // segments long enough to fill 256-row tiles: SM pairs
+        if (transposed) MOE_TRY(map_weight_kmajor_half(&tmB, W, nseg, N, K));
+        else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
+        MOE_TRY(launch_tile_prefix(offsets, nseg, 256, tile_prefix, st));
+        const int64_t max_tiles2 = (cdiv(R, 256) + nseg) * cdiv(N, BN);
+        return transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st) : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st);
+    }
+    if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
+    else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
+    MOE_TRY(launch_tile_prefix(offsets, nseg, BM, tile_prefix, st));
     const int64_t max_tiles = (cdiv(R, BM) + nseg) * cdiv(N, BN);
     return transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st);
 }

@@ -26,6 +26,7 @@ FLAT = [
     small_workload("wide-n-bf16", T=1200, d=128, h=192, n=70, k=2, act="bf16", seed=5),
     small_workload("k8-bf16", T=515, d=64, h=64, n=33, k=8, act="bf16", seed=6),
     small_workload("one-expert-f32", T=100, d=12, h=20, n=1, k=1, seed=7),
+    small_workload("long-segments-bf16", T=3000, d=128, h=320, n=5, k=2, act="bf16", seed=8),  # 256-row tile pairs
     synth.CONFIGS["c1"],
 ]
 
