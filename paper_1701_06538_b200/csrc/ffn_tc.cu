@@ -94,6 +94,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// same, with cluster-scope acquire (the arrival comes from the other CTA of the pair)
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -195,12 +205,12 @@ template <int KIND, int TM = BM>
 __device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
     const int32_t tiles_n = (p.N + BN - 1) / BN;
     if (KIND == WGRAD) {
-        const int32_t tiles_m = (p.M + BM - 1) / BM;
+        const int32_t tiles_m = (p.M + TM - 1) / TM;
         const int64_t per_e = (int64_t)tiles_m * tiles_n;
         if (id >= per_e * p.nseg) return false;
         t.e = (int32_t)(id / per_e);
         const int32_t rem = (int32_t)(id % per_e);
-        t.m0 = (rem / tiles_n) * BM;
+        t.m0 = (rem / tiles_n) * TM;
         t.n0 = (rem % tiles_n) * BN;
         t.b_chunk = t.n0 / 64;
         if (p.offsets) {  // with off_mod: segment s reads the rows of group s % off_mod, B term s / off_mod
@@ -565,15 +575,22 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     auto empty_bar = [&](int s) { return bars + 8u * (STAGES2 + s); };
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + a); };
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + 2 + a); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES2 * STAGE2_BYTES + 8 * (2 * STAGES2 + 4));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES2 * STAGE2_BYTES + 8 * (2 * STAGES2 + 4) + 8);
+    // WGRAD only: afull = this CTA's own A tile has landed (it may need its ragged K tail zeroed before use);
+    // ready (even CTA) = the odd CTA's A tile is landed and fixed
+    auto afull_bar = [&](int s) { return bars + 8u * (2 * STAGES2 + 4 + s); };
+    auto ready_bar = [&](int s) { return bars + 8u * (3 * STAGES2 + 4 + s); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES2 * STAGE2_BYTES + 8 * (4 * STAGES2 + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES2 * STAGE2_BYTES + 8 * (4 * STAGES2 + 4) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0: issues the MMAs, owns the full / tempty barriers
     const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES2; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < STAGES2; ++s) {
+            mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
+            mbar_init(afull_bar(s), 1); mbar_init(ready_bar(s), 1);
+        }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -605,32 +622,71 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
                     const uint32_t a_dst = base + s * STAGE2_BYTES, b_dst = a_dst + A2_BYTES;
-                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
-                    const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
-                    tma2_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0 + 128 * (int)rank);
-                    if (KIND == ROW_BMN)
-                        tma2_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64 + 2 * (int)rank, t.e);
-                    else
-                        tma2_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0 + 128 * (int)rank, t.e);
+                    if (KIND == WGRAD) {
+                        const int r = t.row0 + kb * BK;
+                        if (t.row_end - r < BK) {  // ragged last block: A lands on this CTA's own barrier first
+                            if (rank == 0) mbar_expect_tx(full_bar(s), 2 * B2_BYTES);
+                            mbar_expect_tx(afull_bar(s), A2_BYTES);
+                            tma_load_3d(a_dst, &tmA, afull_bar(s), 0, r, t.m0 / 64 + 2 * (int)rank);
+                        } else {
+                            if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+                            tma2_load_3d(a_dst, &tmA, full_bar(s), 0, r, t.m0 / 64 + 2 * (int)rank);
+                        }
+                        tma2_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk + 2 * (int)rank);
+                    } else {
+                        if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
+                        const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
+                        tma2_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0 + 128 * (int)rank);
+                        if (KIND == ROW_BMN)
+                            tma2_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64 + 2 * (int)rank, t.e);
+                        else
+                            tma2_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0 + 128 * (int)rank, t.e);
+                    }
                     if (++s == STAGES2) { s = 0; ph ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
+        // WGRAD: both CTAs' warp 1 first fix the ragged K tail of their own A tile (rows of the last block
+        // that lie past the segment end are zeroed); the odd CTA then reports its tile ready.
+        auto zero_tail = [&](int s, int valid) {
+            const int lines = (BK - valid) * 2;
+            for (int u = lane; u < lines * 8; u += 32) {
+                const int line = u >> 3, part = u & 7;
+                const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
+                *reinterpret_cast<uint4 *>(smem + s * STAGE2_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
+                    make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+        };
         if (rank == 0) {
-            constexpr uint32_t idesc = make_idesc2(0, KIND == ROW_BK ? 0 : 1);
+            constexpr uint32_t idesc = make_idesc2(KIND == WGRAD ? 1 : 0, KIND == ROW_BK ? 0 : 1);
             int s = 0, acc = 0;
-            uint32_t ph = 0, acc_ph = 0;
+            uint32_t ph = 0, acc_ph = 0, tail_ph = 0;  // tail_ph: one phase bit per stage for afull / ready
             bool ok = true;
             for (int64_t id = cluster_id; ok; id += n_clusters) {
                 Tile t;
                 if (!decode_tile<KIND, 256>(p, id, t)) break;
+                if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
                 ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < t.kblocks; ++kb) {
+                    if (KIND == WGRAD) {
+                        const int valid = t.row_end - (t.row0 + kb * BK);
+                        if (valid < BK) {
+                            const uint32_t tp = (tail_ph >> s) & 1u;
+                            ok = mbar_wait(afull_bar(s), tp, abort_flag, p.status);
+                            if (!ok) break;
+                            zero_tail(s, valid);
+                            ok = mbar_wait(ready_bar(s), tp, abort_flag, p.status) && mbar_try_wait_cluster(ready_bar(s), tp);
+                            if (!ok) break;
+                            tail_ph ^= 1u << s;
+                        }
+                    }
                     ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
@@ -638,7 +694,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (lane == 0) {
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k) {
-                            const uint64_t ad = desc_kmajor(a_src + k * 32);
+                            const uint64_t ad = KIND == WGRAD ? desc_mnmajor(a_src + k * 16 * 128) : desc_kmajor(a_src + k * 32);
                             const uint64_t bd = KIND == ROW_BK ? desc_kmajor(b_src + k * 32) : desc_mnmajor(b_src + k * 16 * 128);
                             tc_mma2_bf16(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                         }
@@ -651,6 +707,26 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 __syncwarp();
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
+        } else if (KIND == WGRAD) {
+            int s = 0;
+            uint32_t tail_ph = 0;
+            bool ok = true;
+            for (int64_t id = cluster_id; ok; id += n_clusters) {
+                Tile t;
+                if (!decode_tile<KIND, 256>(p, id, t)) break;
+                for (int kb = 0; kb < t.kblocks; ++kb) {
+                    const int valid = t.row_end - (t.row0 + kb * BK);
+                    if (valid < BK) {
+                        ok = mbar_wait(afull_bar(s), (tail_ph >> s) & 1u, abort_flag, p.status);
+                        if (!ok) break;
+                        zero_tail(s, valid);
+                        if (lane == 0) mbar_arrive_leader(ready_bar(s));
+                        __syncwarp();
+                        tail_ph ^= 1u << s;
+                    }
+                    if (++s == STAGES2) s = 0;
+                }
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
@@ -662,11 +738,22 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         for (int64_t id = cluster_id; ok; id += n_clusters) {
             Tile t;
             if (!decode_tile<KIND, 256>(p, id, t)) break;
-            ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
-            const int64_t tile_row0 = (int64_t)t.row0 + 128 * (int)rank + quarter * 32;
-            const int32_t rows_valid = t.row_end - (int32_t)tile_row0;
+            const bool have_acc = t.kblocks > 0;
+            if (have_acc) {
+                ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            int64_t tile_row0, out_off = 0;
+            int32_t rows_valid;
+            if (KIND == WGRAD) {
+                out_off = (int64_t)t.e * p.M * p.N;
+                tile_row0 = t.m0 + 128 * (int)rank + quarter * 32;
+                rows_valid = p.M - (int32_t)tile_row0;
+            } else {
+                tile_row0 = (int64_t)t.row0 + 128 * (int)rank + quarter * 32;
+                rows_valid = t.row_end - (int32_t)tile_row0;
+            }
             const int my_piece = lane & 7, my_sub = lane >> 3;
             const bool row_ok = lane < rows_valid;
             const int64_t out_row = tile_row0 + lane;
@@ -674,8 +761,13 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 const int col0 = t.n0 + c * 32;
                 if (col0 >= p.N) break;
                 uint32_t v[32];
-                tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
-                tc_ld_wait();
+                if (have_acc) {
+                    tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
+                    tc_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
                 if (p.out_f32) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
@@ -686,7 +778,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     for (int i = 0; i < 8; ++i) {
                         const int row = 4 * i + my_sub;
                         if (row < rows_valid)
-                            *reinterpret_cast<uint4 *>(p.out_f32 + (tile_row0 + row) * p.N + col0 + my_piece * 4) =
+                            *reinterpret_cast<uint4 *>(p.out_f32 + out_off + (tile_row0 + row) * p.N + col0 + my_piece * 4) =
                                 *reinterpret_cast<const uint4 *>(stage_o + row * 128 + ((my_piece ^ (row & 7)) << 4));
                     }
                     __syncwarp();
@@ -717,15 +809,17 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         }
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_row * p.N + col0);
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) dst[q] = packed[q];
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
-            if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            if (have_acc) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
+                if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            }
         }
     }
 
@@ -914,11 +1008,16 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
 int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int32_t nseg, int64_t R, int32_t M,
                       int32_t N, void *out, int32_t *status, cudaStream_t st) {
     CUtensorMap tmA, tmB;
-    MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, BM / 64));
-    MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, BN / 64));
     GemmParams p = default_params();
     p.offsets = offsets; p.nseg = nseg; p.M = M; p.N = N; p.R = R;
     p.out = (bf16 *)out; p.status = status;
+    if (use_two_cta(R, nseg) && M >= 256) {  // SM pairs: 256 x 256 tiles, each CTA stages half of A and half of B
+        MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, 2));
+        MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, 2));
+        return launch2<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, 256) * cdiv(N, BN), st);
+    }
+    MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, BM / 64));
+    MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, BN / 64));
     return launch<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, BM) * cdiv(N, BN), st);
 }
 
