@@ -508,7 +508,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 // ------------------------------------------------------------------------------------------
 constexpr int STAGES2 = 6;
 constexpr int A2_BYTES = 128 * BK * 2, B2_BYTES = 128 * BK * 2, STAGE2_BYTES = A2_BYTES + B2_BYTES;
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
+constexpr int DATA2_BYTES = STAGES2 * STAGE2_BYTES + EPI_STAGE_BYTES;  // 224 KiB: 6 stages + float staging, or 5 stages + mask tile
+constexpr int SMEM2_BYTES = DATA2_BYTES + 1024 + 256;
 constexpr uint32_t PEER_BIT_MASK = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address of the pair
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -563,39 +564,46 @@ __host__ __device__ constexpr uint32_t make_idesc2(int a_mn, int b_mn) {  // M 2
            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
-template <int KIND>
+// MASKT: the ReLU mask of the dgrad GEMM is not read row by row from global memory by the epilogue but
+// fetched as a 128 x 256 tile by TMA (one stage fewer in exchange for the 64 KiB it occupies).
+template <int KIND, bool MASKT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                     const GemmParams p) {
+                     const __grid_constant__ CUtensorMap tmM, const GemmParams p) {
+    constexpr int NST = MASKT ? 5 : 6;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + STAGES2 * STAGE2_BYTES;
+    const uint32_t bars = base + DATA2_BYTES;  // [stages][float staging or mask tile] then the barriers
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES2 + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES2 + 2 + a); };
+    auto empty_bar = [&](int s) { return bars + 8u * (NST + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * NST + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * NST + 2 + a); };
     // WGRAD only: afull = this CTA's own A tile has landed (it may need its ragged K tail zeroed before use);
     // ready (even CTA) = the odd CTA's A tile is landed and fixed
-    auto afull_bar = [&](int s) { return bars + 8u * (2 * STAGES2 + 4 + s); };
-    auto ready_bar = [&](int s) { return bars + 8u * (3 * STAGES2 + 4 + s); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES2 * STAGE2_BYTES + 8 * (4 * STAGES2 + 4));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES2 * STAGE2_BYTES + 8 * (4 * STAGES2 + 4) + 8);
+    auto afull_bar = [&](int s) { return bars + 8u * (2 * NST + 4 + s); };
+    auto ready_bar = [&](int s) { return bars + 8u * (3 * NST + 4 + s); };
+    const uint32_t mfull_bar = bars + 8u * 28, mempty_bar = bars + 8u * 29;  // mask tile landed / read by all 8 epilogue warps
+    const uint32_t mask_smem = base + NST * STAGE2_BYTES;                     // 4 blocks of [128 rows][64 columns], 128-B swizzle
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + DATA2_BYTES + 240);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + DATA2_BYTES + 248);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0: issues the MMAs, owns the full / tempty barriers
     const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES2; ++s) {
+        for (int s = 0; s < NST; ++s) {
             mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
             mbar_init(afull_bar(s), 1); mbar_init(ready_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
+        mbar_init(mfull_bar, 1); mbar_init(mempty_bar, 8);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+        if (MASKT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmM) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
@@ -613,7 +621,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
             int s = 0;
-            uint32_t ph = 0;
+            uint32_t ph = 0, mask_ph = 0;
             bool ok = true;
             for (int64_t id = cluster_id; ok; id += n_clusters) {
                 Tile t;
@@ -642,7 +650,16 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         else
                             tma2_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0 + 128 * (int)rank, t.e);
                     }
-                    if (++s == STAGES2) { s = 0; ph ^= 1u; }
+                    if (++s == NST) { s = 0; ph ^= 1u; }
+                }
+                if (MASKT && ok) {  // this tile's mask rows, once the previous tile's have been read
+                    ok = mbar_wait(mempty_bar, mask_ph ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    const int nblk = min(4, (p.N - t.n0) / 64);
+                    mbar_expect_tx(mfull_bar, nblk * 16384);
+                    for (int b = 0; b < nblk; ++b)
+                        tma_load_2d(mask_smem + b * 16384, &tmM, mfull_bar, t.n0 + b * 64, t.row0 + 128 * (int)rank);
+                    mask_ph ^= 1u;
                 }
             }
         }
@@ -701,7 +718,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         tc_commit2(empty_bar(s));
                     }
                     __syncwarp();
-                    if (++s == STAGES2) { s = 0; ph ^= 1u; }
+                    if (++s == NST) { s = 0; ph ^= 1u; }
                 }
                 if (ok && lane == 0) tc_commit2(tfull_bar(acc));
                 __syncwarp();
@@ -724,14 +741,15 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         __syncwarp();
                         tail_ph ^= 1u << s;
                     }
-                    if (++s == STAGES2) s = 0;
+                    if (++s == NST) s = 0;
                 }
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         const int quarter = warp & 3, half = (warp - 2) >> 2;
-        uint8_t *stage_o = smem + STAGES2 * STAGE2_BYTES + 256 + (warp - 2) * 4096;
+        uint8_t *stage_o = smem + NST * STAGE2_BYTES + (warp - 2) * 4096;
+        uint32_t mask_ph = 0;
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
@@ -757,6 +775,11 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const int my_piece = lane & 7, my_sub = lane >> 3;
             const bool row_ok = lane < rows_valid;
             const int64_t out_row = tile_row0 + lane;
+            if (MASKT) {
+                ok = mbar_wait(mfull_bar, mask_ph, abort_flag, p.status);
+                if (!ok) break;
+                mask_ph ^= 1u;
+            }
             for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                 const int col0 = t.n0 + c * 32;
                 if (col0 >= p.N) break;
@@ -790,7 +813,13 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         for (int q = 0; q < 4; ++q)
                             bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
                     }
-                    if (p.mask) {
+                    if (MASKT) {  // from the tile in shared memory: row = this thread's row, 16-B pieces swizzled by row
+                        const int mrow = quarter * 32 + lane;
+                        const uint8_t *mrow_p = smem + NST * STAGE2_BYTES + (c >> 1) * 16384 + mrow * 128;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            mask_raw[q] = *reinterpret_cast<const uint4 *>(mrow_p + ((((c & 1) * 4 + q) ^ (mrow & 7)) << 4));
+                    } else if (p.mask) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
@@ -813,6 +842,10 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                     for (int q = 0; q < 4; ++q) dst[q] = packed[q];
                 }
+            }
+            if (MASKT) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(mempty_bar);
             }
             if (have_acc) {
                 tc_fence_before();
@@ -940,8 +973,9 @@ template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tm
     return MOE_OK;
 }
 
-template <int KIND> int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p,
-                                    int64_t max_tiles, cudaStream_t st) {
+template <int KIND, bool MASKT = false>
+int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p, int64_t max_tiles,
+                cudaStream_t st, const CUtensorMap *tmM = nullptr) {
     static int max_clusters = 0;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -951,15 +985,15 @@ template <int KIND> int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &t
     cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM2_BYTES; cfg.stream = st;
     cfg.attrs = &attr; cfg.numAttrs = 1;
     if (!max_clusters) {
-        MOE_CUDA(cudaFuncSetAttribute(grouped_gemm2_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+        MOE_CUDA(cudaFuncSetAttribute(grouped_gemm2_kernel<KIND, MASKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
         cfg.gridDim = dim3(2 * (sm_count() / 2));
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, grouped_gemm2_kernel<KIND>, &cfg) != cudaSuccess || n <= 0) return MOE_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&n, grouped_gemm2_kernel<KIND, MASKT>, &cfg) != cudaSuccess || n <= 0) return MOE_ERR_CUDA;
         max_clusters = n;
     }
     if (max_tiles <= 0) return MOE_OK;
     cfg.gridDim = dim3(2 * (unsigned)imin(max_tiles, max_clusters));
-    MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND>, tmA, tmB, p));
+    MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND, MASKT>, tmA, tmB, tmM ? *tmM : tmA, p));
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -995,6 +1029,11 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
         else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
         MOE_TRY(launch_tile_prefix(offsets, nseg, 256, tile_prefix, st));
         const int64_t max_tiles2 = (cdiv(R, 256) + nseg) * cdiv(N, BN);
+        if (transposed && mask) {  // the ReLU-mask rows come in as TMA tiles
+            CUtensorMap tmM;
+            MOE_TRY(map_rows_kmajor(&tmM, mask, R, N));
+            return launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM);
+        }
         return transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st) : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st);
     }
     if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
