@@ -90,8 +90,24 @@ int32_t reset_status(void *ws, cudaStream_t st) {
 // ---------------------------------------------------------------------------- stage workspaces
 struct GateWs {
     int32_t *idx_p, *idx_s, *perm_p, *inv_perm_p, *counts_p, *offsets_p, *scratch, *tile_prefix;
+    // tensor-core routing screen (flat layer, or the primary level of the hierarchical one)
+    bool screen;
+    float *cr, *wnorm, *xnorm;
+    void *wsplit;
+    int32_t *unsafe_list, *unsafe_count;
     GateWs(Carver &cv, const Dims &D) {
         idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
+        cr = wnorm = xnorm = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = nullptr;
+        const int64_t n1 = D.hier ? D.a : D.n;  // width of the (first) gate
+        screen = tc_gate_fwd_supported(D.act, D.T, (int32_t)D.d, (int32_t)n1);
+        if (screen) {
+            cr = cv.take<float>(D.T * 2 * n1);
+            wsplit = cv.take<bf16>(3 * D.d * 2 * n1);
+            wnorm = cv.take<float>(2 * n1);
+            xnorm = cv.take<float>(D.T);
+            unsafe_list = cv.take<int32_t>(D.T);
+            unsafe_count = cv.take<int32_t>(64);
+        }
         if (!D.hier) return;
         idx_p = cv.take<int32_t>(D.T * D.k1);
         idx_s = cv.take<int32_t>(D.T * D.k);
@@ -260,21 +276,32 @@ struct BwdWs {
 
 int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *Wg, const float *Wnoise,
                 const float *noise, int32_t *topk_idx, float *gates, float *clean, float *raw_noise,
-                float *kth_vals, int32_t *kth_idx, Carver &cv, cudaStream_t st) {
+                float *kth_vals, int32_t *kth_idx, void *ws_base, Carver &cv, cudaStream_t st) {
     GateWs w(cv, D);
-    if (!D.hier) {
-        MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, (int32_t)D.n, Wg, Wnoise, clean, raw_noise, nullptr,
-                                  0, nullptr, 1, nullptr, st));
-        return launch_gate_select(clean, raw_noise, noise, D.T, (int32_t)D.n, (int32_t)D.k, topk_idx, gates,
-                                  kth_vals, kth_idx, st);
-    }
+    // One gate over n1 columns with top-k1 (the flat gate, or the primary gate of the hierarchical layer).
+    // With bf16 activations the routing is screened on the tensor cores and only the tokens whose order is
+    // not provably that of the fixed fma chain are redone with the chain; otherwise the chain does all rows.
+    auto first_gate = [&](int32_t n1, int32_t k1, int32_t *idx_out, float *gates_out) -> int32_t {
+        if (w.screen) {
+            MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, w.wsplit, w.wnorm, w.xnorm,
+                                               w.unsafe_count, st));
+            MOE_TRY(launch_tc_gate_fwd(x, D.T, (int32_t)D.d, n1, w.wsplit, w.cr, status_word(ws_base), st));
+            MOE_TRY(launch_gate_screen(w.cr, noise, w.xnorm, w.wnorm, (int32_t)D.d, D.T, n1, k1, idx_out, gates_out,
+                                       clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_count, st));
+            MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, clean, raw_noise, nullptr, 0,
+                                      w.unsafe_list, 1, nullptr, st, w.unsafe_count));
+            return launch_gate_select(clean, raw_noise, noise, D.T, n1, k1, idx_out, gates_out, kth_vals, kth_idx, st,
+                                      w.unsafe_list, w.unsafe_count);
+        }
+        MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, clean, raw_noise, nullptr, 0, nullptr, 1,
+                                  nullptr, st));
+        return launch_gate_select(clean, raw_noise, noise, D.T, n1, k1, idx_out, gates_out, kth_vals, kth_idx, st);
+    };
+    if (!D.hier) return first_gate((int32_t)D.n, (int32_t)D.k, topk_idx, gates);
     // primary gate over the a groups
     const int64_t P1 = D.T * D.k1;
     float *g_p = gates + D.T * D.k, *g_s = g_p + P1;
-    MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, (int32_t)D.a, Wg, Wnoise, clean, raw_noise, nullptr, 0,
-                              nullptr, 1, nullptr, st));
-    MOE_TRY(launch_gate_select(clean, raw_noise, noise, D.T, (int32_t)D.a, (int32_t)D.k1, w.idx_p, g_p, kth_vals,
-                               kth_idx, st));
+    MOE_TRY(first_gate((int32_t)D.a, (int32_t)D.k1, w.idx_p, g_p));
     // secondary gates: rows (t, s1) grouped by their group so each tile uses one group's matrices
     MOE_TRY(launch_dispatch_index(w.idx_p, P1, (int32_t)D.a, w.perm_p, w.inv_perm_p, w.counts_p, w.offsets_p,
                                   w.scratch, st));
@@ -561,7 +588,8 @@ int32_t moe_gate(const moe_config *cfg, const void *x, const float *Wg, const fl
     const Dims D = dims_of(cfg);
     Carver cv(ws);
     cv.take_bytes(kWsHeader);
-    return do_gate(cfg, D, x, Wg, Wnoise, noise, topk_idx, gates, clean, raw_noise, kth_vals, kth_idx, cv,
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return do_gate(cfg, D, x, Wg, Wnoise, noise, topk_idx, gates, clean, raw_noise, kth_vals, kth_idx, ws, cv,
                    as_stream(stream));
 }
 
@@ -672,7 +700,7 @@ int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const
     auto fresh = [&]() { Carver cv(ws); cv.take_bytes(kWsHeader); return cv; };
     { Carver cv = fresh();
       MOE_TRY(do_gate(cfg, D, x, Wg, Wnoise, noise, C.topk_idx, C.gates, C.clean, C.raw_noise, C.kth_vals,
-                      C.kth_idx, cv, st)); }
+                      C.kth_idx, ws, cv, st)); }
     { Carver cv = fresh();
       MOE_TRY(do_dispatch(D, x, C.topk_idx, C.xs, C.perm, C.inv_perm, C.counts, C.offsets, cv, st)); }
     { Carver cv = fresh();

@@ -1168,6 +1168,26 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
     return MOE_OK;
 }
 
+// Forward gate projection for the routing screen: cr = x . (W_lo + W_mid + W_hi), smallest term first.
+bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n) {
+    const char *env = getenv("MOE_GATE_EXACT_ONLY");
+    if (env && env[0] == '1') return false;
+    return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0 && T >= 1024;
+}
+
+int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,
+                           int32_t *status, cudaStream_t st) {
+    const int32_t n2 = 2 * n;
+    CUtensorMap tmA, tmB;
+    MOE_TRY(map_rows_kmajor(&tmA, x, T, d));
+    MOE_TRY(map_weight_mnmajor_half(&tmB, wsplit, 1, 3 * (int64_t)d, n2));
+    GemmParams p = default_params();
+    p.nseg = 1; p.N = n2; p.K = d; p.R = T; p.out_f32 = cr; p.status = status;
+    p.nterms = 3;
+    for (int i = 0; i < 3; ++i) { p.a_term_col[i] = 0; p.b_term_col[i] = (2 - i) * d; }
+    return launch2<ROW_BMN>(tmA, tmB, p, cdiv(T, 256) * cdiv(n2, BN), st);
+}
+
 // Secondary gates of the hierarchical layer: the slots (t, s1) sorted by primary group are the rows.
 // xs_p [P1, d] token rows in sorted order, dsplit_s [P1, 3 * 2b] split logit gradients in sorted order.
 bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b) {

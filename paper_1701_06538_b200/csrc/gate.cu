@@ -26,6 +26,7 @@ struct ProjArgs {
     const int32_t *offsets;      // grouped only
     const int32_t *perm;         // grouped only
     const int32_t *tile_prefix;  // grouped only
+    const int32_t *row_count;    // optional (ungrouped): number of rows, read on the device
     int64_t M;
     int32_t d, n0, nseg, kdiv;
 };
@@ -49,7 +50,8 @@ __global__ void __launch_bounds__(256) proj_kernel(ProjArgs a) {
     int64_t r0, r_end;
     if (a.offsets == nullptr) {
         r0 = (int64_t)blockIdx.x * PBM;
-        r_end = a.M;
+        r_end = a.row_count ? (int64_t)*a.row_count : a.M;
+        if (r0 >= r_end) return;
     } else {
         const int32_t b = blockIdx.x;
         if (b >= a.tile_prefix[a.nseg]) return;
@@ -167,11 +169,12 @@ __global__ void __launch_bounds__(256) proj_kernel(ProjArgs a) {
 
 int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int32_t n0, const float *W0,
                           const float *W1, float *out0, float *out1, const int32_t *offsets, int32_t nseg,
-                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st) {
+                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st,
+                          const int32_t *row_count) {
     if (M == 0) return MOE_OK;
     ProjArgs a;
     a.x = x; a.W0 = W0; a.W1 = W1; a.out0 = out0; a.out1 = out1;
-    a.offsets = offsets; a.perm = perm; a.tile_prefix = tile_prefix;
+    a.offsets = offsets; a.perm = perm; a.tile_prefix = tile_prefix; a.row_count = row_count;
     a.M = M; a.d = d; a.n0 = n0; a.nseg = nseg; a.kdiv = kdiv;
     int64_t tiles_m = cdiv(M, PBM);
     if (offsets) {
@@ -206,10 +209,17 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
                                                           const float *__restrict__ noise, int64_t rows, int32_t n,
                                                           int32_t k, int32_t *__restrict__ idx,
                                                           float *__restrict__ gates, float *__restrict__ kth_vals,
-                                                          int32_t *__restrict__ kth_idx) {
+                                                          int32_t *__restrict__ kth_idx,
+                                                          const int32_t *__restrict__ row_list,
+                                                          const int32_t *__restrict__ row_count) {
     const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= rows) return;
+    int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row_list) {  // only the listed rows (their number is read on the device)
+        if (row >= *row_count) return;
+        row = row_list[row];
+    } else if (row >= rows) {
+        return;
+    }
     float lv[KL];
     int32_t li[KL];
 #pragma unroll
@@ -273,10 +283,184 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
 
 int32_t launch_gate_select(const float *clean, const float *raw, const float *noise, int64_t rows, int32_t n,
                            int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
-                           cudaStream_t st) {
+                           cudaStream_t st, const int32_t *row_list, const int32_t *row_count) {
     if (rows == 0) return MOE_OK;
     gate_select_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates,
-                                                                  kth_vals, kth_idx);
+                                                                  kth_vals, kth_idx, row_list, row_count);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// Tensor-core screening of the routing (bf16 activations). The projection x.[W_g|W_noise] is first
+// done on the tensor cores with W split into three bf16 terms (~1e-7 of the fma-chain value). From
+// those approximate logits each token's top-(k+2) is found together with a bound U on how far any
+// approximate noisy logit can be from the value the fixed fma chain would give:
+//     |H~_j - H_j| <= theta * |x|_2 * (|W_g[:,j]|_2 + |noise_j| * |W_noise[:,j]|_2) + rounding slack,
+// theta covering the worst-case rounding of the chain (d * 2^-24) and of the tensor-core accumulation
+// (modelled as one truncation of an fp32 accumulator per MMA step, doubled). If every gap between
+// consecutive ranks 1..k+2 exceeds 2U, the order of the top k+1 under the chain values is provably the
+// same, so the routing taken from the approximate logits IS the bit-exact routing. The other tokens
+// (a few per cent) are listed and redone with the fma chain by the kernels above.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) split_gate_weights_kernel(const float *__restrict__ Wg,
+                                                                 const float *__restrict__ Wn, int32_t d, int32_t n,
+                                                                 bf16 *__restrict__ wsplit) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t n2 = 2 * n;
+    if (i >= (int64_t)d * n2) return;
+    const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
+    float v = j < n ? Wg[(int64_t)q * n + j] : Wn[(int64_t)q * n + (j - n)];
+#pragma unroll
+    for (int term = 0; term < 3; ++term) {  // wsplit[term][q][j]: hi, mid, lo
+        const bf16 b = __float2bfloat16_rn(v);
+        wsplit[((int64_t)term * d + q) * n2 + j] = b;
+        v -= __bfloat162float(b);
+    }
+}
+
+__global__ void __launch_bounds__(256) gate_col_norms_kernel(const float *__restrict__ Wg, const float *__restrict__ Wn,
+                                                             int32_t d, int32_t n, float *__restrict__ wnorm) {
+    const int32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= 2 * n) return;
+    const float *W = j < n ? Wg + j : Wn + (j - n);
+    double s = 0.0;
+    for (int32_t q = 0; q < d; ++q) { const double v = W[(int64_t)q * n]; s += v * v; }
+    wnorm[j] = (float)(sqrt(s) * (1.0 + 1e-6));
+}
+
+template <typename XT>
+__global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x, int64_t T, int32_t d,
+                                                        float *__restrict__ xnorm) {
+    const int lane = threadIdx.x & 31;
+    const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= T) return;
+    float s = 0.0f;
+    for (int32_t q = lane; q < d; q += 32) { const float v = to_f32(x[t * d + q]); s = fmaf(v, v, s); }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) xnorm[t] = sqrtf(s) * (1.0f + 1e-5f);
+}
+
+constexpr int KL2 = MOE_MAX_K + 2;
+
+__global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
+                                                          const float *__restrict__ xnorm,
+                                                          const float *__restrict__ wnorm, float theta, int64_t T,
+                                                          int32_t n, int32_t k, int32_t *__restrict__ idx,
+                                                          float *__restrict__ gates, float *__restrict__ clean,
+                                                          float *__restrict__ raw, float *__restrict__ kth_vals,
+                                                          int32_t *__restrict__ kth_idx,
+                                                          int32_t *__restrict__ unsafe_list,
+                                                          int32_t *__restrict__ unsafe_count) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= T) return;
+    float lv[KL2];
+    int32_t li[KL2];
+#pragma unroll
+    for (int s = 0; s < KL2; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; }
+    const float *c = cr + row * 2 * n, *r = c + n, *e = noise + row * n;
+    const float xn = theta * xnorm[row];
+    float umax = 0.0f, hmax = 0.0f;
+    for (int32_t j = lane; j < n; j += 32) {
+        const float cj = c[j], rj = r[j], ej = e[j];
+        clean[row * n + j] = cj;
+        raw[row * n + j] = rj;
+        const double rd = (double)rj;
+        const float sigma = (float)(fmax(rd, 0.0) + log1p(exp(-fabs(rd))));
+        float v = fmaf(ej, sigma, cj);
+        umax = fmaxf(umax, xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]));
+        hmax = fmaxf(hmax, fabsf(v));
+        int32_t id = j;
+        bool shifting = false;
+#pragma unroll
+        for (int s = 0; s < KL2; ++s) {
+            if (shifting || v > lv[s]) {
+                float tv = lv[s]; int32_t ti = li[s];
+                lv[s] = v; li[s] = id; v = tv; id = ti;
+                shifting = true;
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        umax = fmaxf(umax, __shfl_xor_sync(0xffffffffu, umax, off));
+        hmax = fmaxf(hmax, __shfl_xor_sync(0xffffffffu, hmax, off));
+    }
+    const float U = umax + 8.0f * 1.1920929e-7f * hmax;  // + rounding of softplus and of the final fma on both sides
+    const int rounds = min(k + 2, n);
+    float myv = -CUDART_INF_F, prev = 0.0f, min_gap = CUDART_INF_F;
+    int32_t myi = -1;
+    float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
+    int32_t i_k = -1, i_k1 = -1;
+    for (int s = 0; s < rounds; ++s) {
+        float hv = lv[0];
+        int32_t hi = li[0];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, hv, off);
+            int32_t oi = __shfl_xor_sync(0xffffffffu, hi, off);
+            if (ov > hv || (ov == hv && oi < hi)) { hv = ov; hi = oi; }
+        }
+        if (li[0] == hi) {
+#pragma unroll
+            for (int q = 0; q < KL2 - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; }
+            lv[KL2 - 1] = -CUDART_INF_F;
+            li[KL2 - 1] = INT32_MAX;
+        }
+        if (s > 0) min_gap = fminf(min_gap, prev - hv);
+        prev = hv;
+        if (s < k && lane == s) { myv = hv; myi = hi; }
+        if (s == k - 1) { v_k = hv; i_k = hi; }
+        if (s == k && k < n) { v_k1 = hv; i_k1 = hi; }
+    }
+    if (!(min_gap > 2.0f * U)) {  // not provably the chain's routing: redo this token with the fma chain
+        if (lane == 0) unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
+        return;
+    }
+    const float m = __shfl_sync(0xffffffffu, myv, 0);
+    const float ex = lane < k ? expf(myv - m) : 0.0f;
+    float den = 0.0f;
+    for (int s = 0; s < k; ++s) den += __shfl_sync(0xffffffffu, ex, s);
+    if (lane < k) {
+        idx[row * k + lane] = myi;
+        gates[row * k + lane] = ex / den;
+    }
+    if (lane == 0) {
+        kth_vals[row * 2 + 0] = v_k;
+        kth_vals[row * 2 + 1] = v_k1;
+        kth_idx[row * 2 + 0] = i_k;
+        kth_idx[row * 2 + 1] = i_k1;
+    }
+}
+
+int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
+                                   const float *Wn, void *wsplit, float *wnorm, float *xnorm,
+                                   int32_t *unsafe_count, cudaStream_t st) {
+    split_gate_weights_kernel<<<(unsigned)cdiv((int64_t)d * 2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
+    MOE_LAUNCHED();
+    gate_col_norms_kernel<<<(unsigned)cdiv(2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
+    MOE_LAUNCHED();
+    if (act == MOE_BF16) row_norms_kernel<bf16><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const bf16 *)x, T, d, xnorm);
+    else row_norms_kernel<float><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const float *)x, T, d, xnorm);
+    MOE_LAUNCHED();
+    MOE_CUDA(cudaMemsetAsync(unsafe_count, 0, sizeof(int32_t), st));
+    return MOE_OK;
+}
+
+int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
+                           int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
+                           float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
+                           cudaStream_t st) {
+    // worst-case rounding of the fma chain, plus two truncations of an fp32 accumulator per MMA step of the
+    // three-term tensor-core product (3d/16 steps and the additions inside a step), plus the split residual
+    const double u = ldexp(1.0, -24);
+    const double chain = d * u / (1.0 - d * u);
+    const double tc = 2.0 * (3.0 * d / 16.0 + 8.0) * ldexp(1.0, -23) + ldexp(1.0, -22);
+    const float theta = (float)((chain + tc) * 1.01);
+    gate_screen_kernel<<<(unsigned)cdiv(T, 8), 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean,
+                                                              raw, kth_vals, kth_idx, unsafe_list, unsafe_count);
     MOE_LAUNCHED();
     return MOE_OK;
 }

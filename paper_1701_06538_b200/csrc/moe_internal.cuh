@@ -66,11 +66,24 @@ static const int64_t kWsHeader = 256;
 // reads token perm[r] / kdiv, uses W0 + e*d*n0, and writes output row perm[r].
 int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int32_t n0, const float *W0,
                           const float *W1, float *out0, float *out1, const int32_t *offsets, int32_t nseg,
-                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st);
+                          const int32_t *perm, int32_t kdiv, int32_t *tile_prefix, cudaStream_t st,
+                          const int32_t *row_count = nullptr);
 // Noisy logits, top-k, masked softmax for `rows` rows of n columns.
 int32_t launch_gate_select(const float *clean, const float *raw, const float *noise, int64_t rows, int32_t n,
                            int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
+                           cudaStream_t st, const int32_t *row_list = nullptr, const int32_t *row_count = nullptr);
+// Tensor-core screening of the routing (see gate.cu): weights split / norms, then the screening select.
+int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
+                                   const float *Wn, void *wsplit, float *wnorm, float *xnorm,
+                                   int32_t *unsafe_count, cudaStream_t st);
+int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
+                           int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
+                           float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
                            cudaStream_t st);
+bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n);
+// cr [T, 2n] (float) = x . [W_g | W_noise] from the three-term split wsplit [3, d, 2n]
+int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,
+                           int32_t *status, cudaStream_t st);
 int32_t launch_hier_merge(int64_t T, int32_t k1, int32_t k2, int32_t b, const int32_t *idx_p, const float *g_p,
                           const int32_t *idx_s, const float *g_s, int32_t *topk_idx, float *gates,
                           cudaStream_t st);

@@ -10,6 +10,8 @@ from paper_1701_06538_b200 import synth
 from helpers import (TOL_F32, act_empty, assert_close, cat_parts, cfg_of, dev, dev_act, device_inputs, f32, host, i32,
                      oracle_run, prec_of, small_workload, tol_act)
 
+from test_gpu_stages import screened
+
 pytestmark = pytest.mark.gpu
 
 HIER = [
@@ -48,8 +50,13 @@ def test_hier_gate(case):
     B.moe_gate(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], idx, gates, clean, raw, kv, ki, ws)
     want = gate_tensors(F.G)
     assert (host(idx) == want["topk_idx"]).all(), "hierarchical routing must be bit-exact"
-    assert (host(clean) == want["clean"]).all() and (host(raw) == want["raw"]).all()
-    assert (host(ki) == want["kth_idx"]).all() and (host(kv) == want["kth_vals"]).all()
+    assert (host(ki) == want["kth_idx"]).all()
+    if screened(w):  # primary logits of provably-routed tokens come from the tensor-core product
+        for name, got in (("clean", clean), ("raw", raw), ("kth_vals", kv)):
+            assert_close(host(got), want[name], TOL_F32, name)
+    else:
+        assert (host(clean) == want["clean"]).all() and (host(raw) == want["raw"]).all()
+        assert (host(kv) == want["kth_vals"]).all()
     assert_close(host(gates), want["gates"], TOL_F32, "gates")
 
 
