@@ -26,7 +26,7 @@ sys.path.insert(0, ROOT)
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-from paper_1701_06538_b200 import synth  # noqa: E402
+from paper_1701_06538_b200 import replicas, synth  # noqa: E402
 
 METRIC = "moe_layer_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
@@ -87,17 +87,17 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def cpu_sample_tokens(w):
-    # about 10-30 s of oracle work per forward+backward on the host cores
+def cpu_sample_tokens(w, flop_budget=2.0e12):
+    # flop_budget 2e12: about 10-30 s of oracle work per forward+backward on the host cores
     per_token_flop = 12.0 * w.k * w.d * w.h + 12.0 * w.d * (w.n if w.a == 0 else w.a + w.k1 * w.b)
-    return int(max(256, min(w.T, 2 ** int(np.log2(2.0e12 / per_token_flop)))))
+    return int(max(256, min(w.T, 2 ** int(np.log2(flop_budget / per_token_flop)))))
 
 
 def run_reference(args, w):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    Ts = cpu_sample_tokens(w)
+    Ts = cpu_sample_tokens(w, 5.0e11)  # a few seconds per step, so that K + W steps end within minutes
     ws, I = host_inputs_sample(w, Ts)
     for _ in range(min(args.warmup, 1)):
         oracle_step(ws, I)
@@ -324,13 +324,9 @@ def run_ours(args, w):
     h2d = hx.numel() * hx.element_size() * 2 + hnoise.numel() * 4
     d2h = hy.numel() * hy.element_size() * 2 + 8
 
-    total_ms, total_e2e = sum(ms), sum(ms_e2e)
-    if world > 1:
-        t = torch.tensor([total_ms, total_e2e], device="cuda", dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms, total_e2e = t.tolist()
-    value = world * w.T * args.steps / (total_ms / 1e3)
-    value_e2e = world * w.T * args.steps / (total_e2e / 1e3)
+    total_ms, total_e2e = replicas.max_over_ranks([sum(ms), sum(ms_e2e)], device="cuda")
+    value = replicas.job_throughput(w.T, args.steps, total_ms, world)
+    value_e2e = replicas.job_throughput(w.T, args.steps, total_e2e, world)
 
     stages = stage_timings(B, cfg, S, D, w, timed, max(3, min(args.steps, 10)), peaks)
     gemm_flop = 12.0 * w.R * w.d * w.h
