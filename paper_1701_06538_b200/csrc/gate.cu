@@ -344,6 +344,7 @@ __global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x
 
 constexpr int KL2 = MOE_MAX_K + 2;
 
+template <int NV>  // columns per lane (n <= 32 * NV); 0: any n, plain loop
 __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
                                                           const float *__restrict__ xnorm,
                                                           const float *__restrict__ wnorm, float theta, int64_t T,
@@ -356,66 +357,99 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= T) return;
-    float lv[KL2];
+    // per-lane sorted list of (value, index, uncertainty); rest_hi = largest possible chain value of anything
+    // that is not in a list
+    float lv[KL2], lu[KL2];
     int32_t li[KL2];
 #pragma unroll
-    for (int s = 0; s < KL2; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; }
+    for (int s = 0; s < KL2; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
     const float *c = cr + row * 2 * n, *r = c + n, *e = noise + row * n;
     const float xn = theta * xnorm[row];
-    float umax = 0.0f, hmax = 0.0f;
-    for (int32_t j = lane; j < n; j += 32) {
-        const float cj = c[j], rj = r[j], ej = e[j];
+    float rest_hi = -CUDART_INF_F;
+    auto consider = [&](int32_t j, float cj, float rj, float ej) {
         clean[row * n + j] = cj;
         raw[row * n + j] = rj;
-        const double rd = (double)rj;
-        const float sigma = (float)(fmax(rd, 0.0) + log1p(exp(-fabs(rd))));
+        // single-precision softplus is enough for screening: its few ulp go into the uncertainty
+        const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
         float v = fmaf(ej, sigma, cj);
-        umax = fmaxf(umax, xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]));
-        hmax = fmaxf(hmax, fabsf(v));
+        // |H~_j - H_j|: projection errors through c and through softplus(r) (slope <= 1) times |noise|, plus the
+        // rounding of softplus (here single, there double rounded once) and of the final fma on both sides
+        float u = xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]) +
+                  1.1920929e-7f * (8.0f * fabsf(v) + 16.0f * fabsf(ej) * sigma);
         int32_t id = j;
         bool shifting = false;
 #pragma unroll
         for (int s = 0; s < KL2; ++s) {
             if (shifting || v > lv[s]) {
-                float tv = lv[s]; int32_t ti = li[s];
-                lv[s] = v; li[s] = id; v = tv; id = ti;
+                float tv = lv[s], tu = lu[s]; int32_t ti = li[s];
+                lv[s] = v; li[s] = id; lu[s] = u; v = tv; id = ti; u = tu;
                 shifting = true;
             }
         }
-    }
+        if (id != INT32_MAX) rest_hi = fmaxf(rest_hi, v + u);  // fell off (or never entered) the list
+    };
+    if (NV > 0) {
+        float cv[NV > 0 ? NV : 1], rv[NV > 0 ? NV : 1], ev[NV > 0 ? NV : 1];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        umax = fmaxf(umax, __shfl_xor_sync(0xffffffffu, umax, off));
-        hmax = fmaxf(hmax, __shfl_xor_sync(0xffffffffu, hmax, off));
+        for (int q = 0; q < NV; ++q) {
+            const int32_t j = lane + 32 * q;
+            const bool in = j < n;
+            cv[q] = in ? c[j] : 0.0f; rv[q] = in ? r[j] : 0.0f; ev[q] = in ? e[j] : 0.0f;
+        }
+#pragma unroll
+        for (int q = 0; q < NV; ++q)
+            if (lane + 32 * q < n) consider(lane + 32 * q, cv[q], rv[q], ev[q]);
+    } else {
+        for (int32_t j = lane; j < n; j += 32) consider(j, c[j], r[j], e[j]);
     }
-    const float U = umax + 8.0f * 1.1920929e-7f * hmax;  // + rounding of softplus and of the final fma on both sides
     const int rounds = min(k + 2, n);
-    float myv = -CUDART_INF_F, prev = 0.0f, min_gap = CUDART_INF_F;
+    float hvv[KL2], huu[KL2];
+    float myv = -CUDART_INF_F;
     int32_t myi = -1;
     float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
     int32_t i_k = -1, i_k1 = -1;
-    for (int s = 0; s < rounds; ++s) {
-        float hv = lv[0];
-        int32_t hi = li[0];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, hv, off);
-            int32_t oi = __shfl_xor_sync(0xffffffffu, hi, off);
-            if (ov > hv || (ov == hv && oi < hi)) { hv = ov; hi = oi; }
-        }
-        if (li[0] == hi) {
+    for (int s = 0; s < KL2; ++s) {
+        hvv[s] = -CUDART_INF_F; huu[s] = 0.0f;
+        if (s < rounds) {
+            float hv = lv[0], hu = lu[0];
+            int32_t hi = li[0];
 #pragma unroll
-            for (int q = 0; q < KL2 - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; }
-            lv[KL2 - 1] = -CUDART_INF_F;
-            li[KL2 - 1] = INT32_MAX;
+            for (int off = 16; off > 0; off >>= 1) {
+                float ov = __shfl_xor_sync(0xffffffffu, hv, off), ou = __shfl_xor_sync(0xffffffffu, hu, off);
+                int32_t oi = __shfl_xor_sync(0xffffffffu, hi, off);
+                if (ov > hv || (ov == hv && oi < hi)) { hv = ov; hi = oi; hu = ou; }
+            }
+            if (li[0] == hi) {
+#pragma unroll
+                for (int q = 0; q < KL2 - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; lu[q] = lu[q + 1]; }
+                lv[KL2 - 1] = -CUDART_INF_F;
+                li[KL2 - 1] = INT32_MAX;
+            }
+            hvv[s] = hv; huu[s] = hu;
+            if (s < k && lane == s) { myv = hv; myi = hi; }
+            if (s == k - 1) { v_k = hv; i_k = hi; }
+            if (s == k && k < n) { v_k1 = hv; i_k1 = hi; }
         }
-        if (s > 0) min_gap = fminf(min_gap, prev - hv);
-        prev = hv;
-        if (s < k && lane == s) { myv = hv; myi = hi; }
-        if (s == k - 1) { v_k = hv; i_k = hi; }
-        if (s == k && k < n) { v_k1 = hv; i_k1 = hi; }
     }
-    if (!(min_gap > 2.0f * U)) {  // not provably the chain's routing: redo this token with the fma chain
+    // whatever is still in the lists is "rest" as well
+#pragma unroll
+    for (int s = 0; s < KL2; ++s)
+        if (li[s] != INT32_MAX) rest_hi = fmaxf(rest_hi, lv[s] + lu[s]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) rest_hi = fmaxf(rest_hi, __shfl_xor_sync(0xffffffffu, rest_hi, off));
+    // ranks 1..k+1 are certain iff each one's lowest possible value beats the highest possible value of
+    // everything ranked after it
+    bool safe = true;
+    float suffix = rest_hi;
+#pragma unroll
+    for (int s = KL2 - 1; s >= 0; --s) {
+        if (s < rounds) {
+            if (s <= k && !(hvv[s] - huu[s] > suffix)) safe = false;
+            suffix = fmaxf(suffix, hvv[s] + huu[s]);
+        }
+    }
+    if (!safe) {  // not provably the chain's routing: redo this token with the fma chain
         if (lane == 0) unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
         return;
     }
@@ -459,8 +493,16 @@ int32_t launch_gate_screen(const float *cr, const float *noise, const float *xno
     const double chain = d * u / (1.0 - d * u);
     const double tc = 2.0 * (3.0 * d / 16.0 + 8.0) * ldexp(1.0, -23) + ldexp(1.0, -22);
     const float theta = (float)((chain + tc) * 1.01);
-    gate_screen_kernel<<<(unsigned)cdiv(T, 8), 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean,
-                                                              raw, kth_vals, kth_idx, unsafe_list, unsafe_count);
+    const unsigned grid = (unsigned)cdiv(T, 8);
+#define MOE_SCREEN(NV)                                                                                              \
+    gate_screen_kernel<NV><<<grid, 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean, raw, \
+                                                 kth_vals, kth_idx, unsafe_list, unsafe_count)
+    if (n <= 32) MOE_SCREEN(1);
+    else if (n <= 64) MOE_SCREEN(2);
+    else if (n <= 128) MOE_SCREEN(4);
+    else if (n <= 256) MOE_SCREEN(8);
+    else MOE_SCREEN(0);
+#undef MOE_SCREEN
     MOE_LAUNCHED();
     return MOE_OK;
 }
