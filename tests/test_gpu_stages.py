@@ -114,6 +114,31 @@ def test_gate_screen_sends_ties_and_near_ties_to_the_exact_chain():
     assert_close(host(clean), G.clean, TOL_F32, "clean")
 
 
+def test_screened_routing_equals_pure_chain_routing_on_many_batches():
+    """The screen must never change the routing: with MOE_GATE_EXACT_ONLY=1 every token goes through the fma
+    chain; both runs must give identical indices on fresh batches of a wide, skewed gate (c5's shape)."""
+    import os
+    from dataclasses import replace
+    base = replace(synth.CONFIGS["c5"], T=16384)
+    for seed in range(6):
+        w = replace(base, seed=synth.BASE_SEED + 500 + seed, name=f"c5-seed{seed}")
+        cfg = cfg_of(w)
+        ws, S = ws_for(cfg)
+        x, (Wg, Wn, noise) = dev_act(synth.make_x(w), w), [dev(a) for a in synth.make_gate(w)]
+        out = []
+        for exact_only in ("0", "1"):
+            os.environ["MOE_GATE_EXACT_ONLY"] = exact_only
+            idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
+            kv, ki = f32(w.T, 2), i32(w.T, 2)
+            B.moe_gate(cfg, x, Wg, Wn, noise, idx, gates, clean, raw, kv, ki, ws)
+            assert B.moe_check_status(ws) == 0
+            out.append((idx, ki, gates, clean))
+        os.environ.pop("MOE_GATE_EXACT_ONLY")
+        assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
+        assert_close(host(out[0][2]), host(out[1][2]), TOL_F32, "gates")
+        assert_close(host(out[0][3]), host(out[1][3]), TOL_F32, "clean")
+
+
 def test_dispatch(case):
     w, I, F, _, D, cfg = case
     ws, S = ws_for(cfg)
