@@ -1170,9 +1170,13 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
 
 // Forward gate projection for the routing screen: cr = x . (W_lo + W_mid + W_hi), smallest term first.
 bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n) {
-    const char *env = getenv("MOE_GATE_EXACT_ONLY");
-    if (env && env[0] == '1') return false;
-    return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0 && T >= 1024;
+    // MOE_GATE_SCREEN=0: every token through the fma chain; =1: screen whenever the shapes allow;
+    // unset: screen when the projection is large enough to pay for the extra launches
+    const char *env = getenv("MOE_GATE_SCREEN");
+    if (env && env[0] == '0') return false;
+    if (!(act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0 && T >= 256)) return false;
+    if (env && env[0] == '1') return true;
+    return (double)T * d * 2.0 * n >= 1.0e9;
 }
 
 int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,

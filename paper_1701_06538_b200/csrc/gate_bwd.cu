@@ -13,6 +13,7 @@ namespace moe {
 //                                 the threshold is another entry's noisy logit:
 //                                 dH[j_(k+1)] -= sum_{kept j} q_j ; dH[j_k] -= sum_{other j} q_j
 //   H = c + eps * sigma:          dc += dH ; dsigma += eps * dH ; dr = dsigma * sigmoid(r)
+template <int NV>  // columns per lane kept in registers (n <= 32 * NV); 0: any n, recompute in a second pass
 __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
     const float *__restrict__ noise, const float *__restrict__ clean, const float *__restrict__ raw,
     const int32_t *__restrict__ idx, const float *__restrict__ gates, const float *__restrict__ kth_vals,
@@ -38,42 +39,27 @@ __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
     const float *dl = dload + (dload_row_group ? (int64_t)dload_row_group[row] * n : 0);
     const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
 
-    auto load_terms = [&](int32_t j, bool &sel, float &dh_soft, float &q, float &zq) {
+    // per column: is it kept, its softmax-path gradient, q = dLoad * phi(z) / sigma and z * q
+    auto load_terms = [&](int32_t j, float cj, float rj, float dlj, bool &sel, float &dh_soft, float &q, float &zq) {
         sel = false;
         dh_soft = 0.0f;
 #pragma unroll
         for (int s = 0; s < MOE_MAX_K; ++s)
             if (sel_idx[s] == j) { sel = true; dh_soft = sel_dh[s]; }
-        const float rj = r[j];
         const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
-        const float z = (c[j] - (sel ? thr_sel : thr_unsel)) / sigma;
+        const float z = (cj - (sel ? thr_sel : thr_unsel)) / sigma;
         if (isfinite(z)) {
-            q = dl[j] * (expf(-0.5f * z * z) * 0.39894228040143267794f) / sigma;
+            q = dlj * (expf(-0.5f * z * z) * 0.39894228040143267794f) / sigma;
             zq = z * q;
         } else {
             q = 0.0f;
             zq = 0.0f;
         }
     };
-
-    float q_sel = 0.0f, q_uns = 0.0f;
-    for (int32_t j = lane; j < n; j += 32) {
-        bool sel; float dh, q, zq;
-        load_terms(j, sel, dh, q, zq);
-        if (sel) q_sel += q; else q_uns += q;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        q_sel += __shfl_xor_sync(0xffffffffu, q_sel, off);
-        q_uns += __shfl_xor_sync(0xffffffffu, q_uns, off);
-    }
-    for (int32_t j = lane; j < n; j += 32) {
-        bool sel; float dh, q, zq;
-        load_terms(j, sel, dh, q, zq);
+    auto finish = [&](int32_t j, float rj, float ej, float dh, float q, float zq, float q_sel, float q_uns) {
         if (j == j_k1) dh -= q_sel;
         if (j == j_k && k < n) dh -= q_uns;
-        const float rj = r[j];
-        const float dsigma = fmaf(e[j], dh, -zq);
+        const float dsigma = fmaf(ej, dh, -zq);
         const float dc = q + dh, dr = dsigma / (1.0f + expf(-rj));
         if (dsplit) {
             // three-term bf16 split (hi | mid | lo), row layout [3][clean n | raw n], for the tensor-core products
@@ -97,6 +83,54 @@ __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
             dclean[row * n + j] = dc;
             draw[row * n + j] = dr;
         }
+    };
+
+    float q_sel = 0.0f, q_uns = 0.0f;
+    if (NV > 0) {
+        float cv[NV > 0 ? NV : 1], rv[NV > 0 ? NV : 1], ev[NV > 0 ? NV : 1], dv[NV > 0 ? NV : 1];
+        float dhv[NV > 0 ? NV : 1], qv[NV > 0 ? NV : 1], zqv[NV > 0 ? NV : 1];
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {  // all loads of the row first
+            const int32_t j = lane + 32 * u;
+            const bool in = j < n;
+            cv[u] = in ? c[j] : 0.0f; rv[u] = in ? r[j] : 0.0f; ev[u] = in ? e[j] : 0.0f; dv[u] = in ? dl[j] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int32_t j = lane + 32 * u;
+            bool sel = false;
+            dhv[u] = qv[u] = zqv[u] = 0.0f;
+            if (j < n) {
+                load_terms(j, cv[u], rv[u], dv[u], sel, dhv[u], qv[u], zqv[u]);
+                if (sel) q_sel += qv[u]; else q_uns += qv[u];
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            q_sel += __shfl_xor_sync(0xffffffffu, q_sel, off);
+            q_uns += __shfl_xor_sync(0xffffffffu, q_uns, off);
+        }
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int32_t j = lane + 32 * u;
+            if (j < n) finish(j, rv[u], ev[u], dhv[u], qv[u], zqv[u], q_sel, q_uns);
+        }
+    } else {
+        for (int32_t j = lane; j < n; j += 32) {
+            bool sel; float dh, q, zq;
+            load_terms(j, c[j], r[j], dl[j], sel, dh, q, zq);
+            if (sel) q_sel += q; else q_uns += q;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            q_sel += __shfl_xor_sync(0xffffffffu, q_sel, off);
+            q_uns += __shfl_xor_sync(0xffffffffu, q_uns, off);
+        }
+        for (int32_t j = lane; j < n; j += 32) {
+            bool sel; float dh, q, zq;
+            load_terms(j, c[j], r[j], dl[j], sel, dh, q, zq);
+            finish(j, r[j], e[j], dh, q, zq, q_sel, q_uns);
+        }
     }
 }
 
@@ -106,10 +140,17 @@ int32_t launch_gate_logit_grads(const float *noise, const float *clean, const fl
                                 int64_t rows, int32_t n, int32_t k, float *dclean, float *draw, void *dsplit,
                                 const int32_t *split_row_index, cudaStream_t st) {
     if (rows == 0) return MOE_OK;
-    gate_logit_grads_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals,
-                                                                       kth_idx, dgates, dload, dload_row_group,
-                                                                       rows, n, k, dclean, draw, (bf16 *)dsplit,
-                                                                       split_row_index);
+    const unsigned grid = (unsigned)cdiv(rows, 8);
+#define MOE_LOGIT_GRADS(NV)                                                                                          \
+    gate_logit_grads_kernel<NV><<<grid, 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals, kth_idx, dgates, dload, \
+                                                      dload_row_group, rows, n, k, dclean, draw, (bf16 *)dsplit,      \
+                                                      split_row_index)
+    if (n <= 32) MOE_LOGIT_GRADS(1);
+    else if (n <= 64) MOE_LOGIT_GRADS(2);
+    else if (n <= 128) MOE_LOGIT_GRADS(4);
+    else if (n <= 256) MOE_LOGIT_GRADS(8);
+    else MOE_LOGIT_GRADS(0);
+#undef MOE_LOGIT_GRADS
     MOE_LAUNCHED();
     return MOE_OK;
 }
