@@ -250,8 +250,19 @@ int32_t launch_dispatch_rows(const void *x, int32_t act, int64_t T, int32_t k, i
     return MOE_OK;
 }
 
+// The three kernels below gather or scatter the k rows of a token. KT is k rounded up to a power of two and VB
+// the number of 16-byte vectors a lane handles per batch (KT * VB = 8): all loads of a batch are issued before
+// any of them is used, so a lane keeps up to eight 16-byte loads in flight.
+#define MOE_DISPATCH_KT(K_, CALL)          \
+    do {                                   \
+        if ((K_) <= 1) { CALL(1, 8); }     \
+        else if ((K_) <= 2) { CALL(2, 4); }\
+        else if ((K_) <= 4) { CALL(4, 2); }\
+        else { CALL(8, 1); }               \
+    } while (0)
+
 // y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]]   (Eq. 1), float sum in slot order
-template <typename XT>
+template <typename XT, int KT, int VB>
 __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys, const float *__restrict__ gates,
                                                       const int32_t *__restrict__ inv_perm, int64_t T, int32_t k,
                                                       int32_t d, XT *__restrict__ y) {
@@ -261,30 +272,37 @@ __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys,
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = d / VN;
     for (int64_t t = warp; t < T; t += nwarps) {
-        int32_t rows[MOE_MAX_K];
-        float g[MOE_MAX_K];
+        const uint4 *rowp[KT];
+        float g[KT];
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) {
-            rows[s] = s < k ? inv_perm[t * k + s] : 0;
+        for (int s = 0; s < KT; ++s) {
+            rowp[s] = reinterpret_cast<const uint4 *>(ys + (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d);
             g[s] = s < k ? gates[t * k + s] : 0.0f;
         }
-        for (int v = lane; v < nvec; v += 32) {
-            float acc[VN];
+        for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
+            Vec16<XT> in[KT][VB];
 #pragma unroll
-            for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
+            for (int b = 0; b < VB; ++b)
 #pragma unroll
-            for (int s = 0; s < MOE_MAX_K; ++s) {
-                if (s < k) {
-                    Vec16<XT> in;
-                    in.raw = reinterpret_cast<const uint4 *>(ys + (int64_t)rows[s] * d)[v];
+                for (int s = 0; s < KT; ++s)
+                    if (s < k && v0 + 32 * b < nvec) in[s][b].raw = rowp[s][v0 + 32 * b];
 #pragma unroll
-                    for (int i = 0; i < VN; ++i) acc[i] = fmaf(g[s], in.get(i), acc[i]);
-                }
+            for (int b = 0; b < VB; ++b) {
+                if (v0 + 32 * b >= nvec) break;
+                float acc[VN];
+#pragma unroll
+                for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
+#pragma unroll
+                for (int s = 0; s < KT; ++s)
+                    if (s < k) {
+#pragma unroll
+                        for (int i = 0; i < VN; ++i) acc[i] = fmaf(g[s], in[s][b].get(i), acc[i]);
+                    }
+                Vec16<XT> out;
+#pragma unroll
+                for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
+                reinterpret_cast<uint4 *>(y + t * d)[v0 + 32 * b] = out.raw;
             }
-            Vec16<XT> out;
-#pragma unroll
-            for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
-            reinterpret_cast<uint4 *>(y + t * d)[v] = out.raw;
         }
     }
 }
@@ -293,16 +311,19 @@ int32_t launch_combine(const void *ys, int32_t act, const float *gates, const in
                        int32_t k, int32_t d, void *y, cudaStream_t st) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
-    if (act == MOE_BF16)
-        combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)ys, gates, inv_perm, T, k, d, (bf16 *)y);
-    else
-        combine_kernel<float><<<grid, 256, 0, st>>>((const float *)ys, gates, inv_perm, T, k, d, (float *)y);
+#define MOE_CALL(KT, VB)                                                                                          \
+    if (act == MOE_BF16)                                                                                          \
+        combine_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)ys, gates, inv_perm, T, k, d, (bf16 *)y); \
+    else                                                                                                          \
+        combine_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)ys, gates, inv_perm, T, k, d, (float *)y)
+    MOE_DISPATCH_KT(k, MOE_CALL);
+#undef MOE_CALL
     MOE_LAUNCHED();
     return MOE_OK;
 }
 
 // dgates[t,s] = <dY[t], ys[row]>,  dys[row] = gates[t,s] * dY[t]
-template <typename XT>
+template <typename XT, int KT, int VB>
 __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__ dY, const XT *__restrict__ ys,
                                                           const float *__restrict__ gates,
                                                           const int32_t *__restrict__ inv_perm, int64_t T,
@@ -314,33 +335,44 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = d / VN;
     for (int64_t t = warp; t < T; t += nwarps) {
-        int32_t rows[MOE_MAX_K];
-        float g[MOE_MAX_K], dot[MOE_MAX_K];
+        int64_t rowo[KT];
+        float g[KT], dot[KT];
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) {
-            rows[s] = s < k ? inv_perm[t * k + s] : 0;
+        for (int s = 0; s < KT; ++s) {
+            rowo[s] = (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d;
             g[s] = s < k ? gates[t * k + s] : 0.0f;
             dot[s] = 0.0f;
         }
-        for (int v = lane; v < nvec; v += 32) {
-            Vec16<XT> dy;
-            dy.raw = reinterpret_cast<const uint4 *>(dY + t * d)[v];
+        for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
+            Vec16<XT> dy[VB], in[KT][VB];
 #pragma unroll
-            for (int s = 0; s < MOE_MAX_K; ++s) {
-                if (s < k) {
-                    Vec16<XT> in, out;
-                    in.raw = reinterpret_cast<const uint4 *>(ys + (int64_t)rows[s] * d)[v];
+            for (int b = 0; b < VB; ++b) {
+                if (v0 + 32 * b < nvec) {
+                    dy[b].raw = reinterpret_cast<const uint4 *>(dY + t * d)[v0 + 32 * b];
 #pragma unroll
-                    for (int i = 0; i < VN; ++i) {
-                        dot[s] = fmaf(dy.get(i), in.get(i), dot[s]);
-                        out.set(i, g[s] * dy.get(i));
+                    for (int s = 0; s < KT; ++s)
+                        if (s < k) in[s][b].raw = reinterpret_cast<const uint4 *>(ys + rowo[s])[v0 + 32 * b];
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < VB; ++b) {
+                if (v0 + 32 * b >= nvec) break;
+#pragma unroll
+                for (int s = 0; s < KT; ++s) {
+                    if (s < k) {
+                        Vec16<XT> out;
+#pragma unroll
+                        for (int i = 0; i < VN; ++i) {
+                            dot[s] = fmaf(dy[b].get(i), in[s][b].get(i), dot[s]);
+                            out.set(i, g[s] * dy[b].get(i));
+                        }
+                        reinterpret_cast<uint4 *>(dys + rowo[s])[v0 + 32 * b] = out.raw;
                     }
-                    reinterpret_cast<uint4 *>(dys + (int64_t)rows[s] * d)[v] = out.raw;
                 }
             }
         }
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) {
+        for (int s = 0; s < KT; ++s) {
             if (s < k) {
                 float v = dot[s];
 #pragma unroll
@@ -356,18 +388,21 @@ int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const fl
                            cudaStream_t st) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
-    if (act == MOE_BF16)
-        combine_bwd_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)dY, (const bf16 *)ys, gates, inv_perm, T, k,
-                                                        d, dgates, (bf16 *)dys);
-    else
-        combine_bwd_kernel<float><<<grid, 256, 0, st>>>((const float *)dY, (const float *)ys, gates, inv_perm, T,
-                                                         k, d, dgates, (float *)dys);
+#define MOE_CALL(KT, VB)                                                                                             \
+    if (act == MOE_BF16)                                                                                             \
+        combine_bwd_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)dY, (const bf16 *)ys, gates, inv_perm, T, \
+                                                                k, d, dgates, (bf16 *)dys);                           \
+    else                                                                                                             \
+        combine_bwd_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)dY, (const float *)ys, gates, inv_perm, \
+                                                                 T, k, d, dgates, (float *)dys)
+    MOE_DISPATCH_KT(k, MOE_CALL);
+#undef MOE_CALL
     MOE_LAUNCHED();
     return MOE_OK;
 }
 
 // out[t] = sum_s dxs[inv_perm[t*k+s]] (+ add[t]); float output, or rounded to the act type
-template <typename XT>
+template <typename XT, int KT, int VB>
 __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict__ dxs,
                                                            const int32_t *__restrict__ inv_perm, int64_t T,
                                                            int32_t k, int32_t d, const float *add,
@@ -378,34 +413,57 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = d / VN;
     for (int64_t t = warp; t < T; t += nwarps) {
-        int32_t rows[MOE_MAX_K];
+        const uint4 *rowp[KT];
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) rows[s] = s < k ? inv_perm[t * k + s] : 0;
-        for (int v = lane; v < nvec; v += 32) {
-            float acc[VN];
+        for (int s = 0; s < KT; ++s)
+            rowp[s] = reinterpret_cast<const uint4 *>(dxs + (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d);
+        for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
+            Vec16<XT> in[KT][VB];
+            float4 addv[VB][VN / 4];
 #pragma unroll
-            for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
+            for (int b = 0; b < VB; ++b) {
+                if (v0 + 32 * b < nvec) {
 #pragma unroll
-            for (int s = 0; s < MOE_MAX_K; ++s) {
-                if (s < k) {
-                    Vec16<XT> in;
-                    in.raw = reinterpret_cast<const uint4 *>(dxs + (int64_t)rows[s] * d)[v];
+                    for (int s = 0; s < KT; ++s)
+                        if (s < k) in[s][b].raw = rowp[s][v0 + 32 * b];
+                    if (add) {
 #pragma unroll
-                    for (int i = 0; i < VN; ++i) acc[i] += in.get(i);
+                        for (int q = 0; q < VN / 4; ++q)
+                            addv[b][q] = reinterpret_cast<const float4 *>(add + t * d + (int64_t)(v0 + 32 * b) * VN)[q];
+                    }
                 }
             }
-            if (add) {
 #pragma unroll
-                for (int i = 0; i < VN; ++i) acc[i] += add[t * d + (int64_t)v * VN + i];
-            }
-            if (out_act) {
-                Vec16<XT> out;
+            for (int b = 0; b < VB; ++b) {
+                if (v0 + 32 * b >= nvec) break;
+                float acc[VN];
 #pragma unroll
-                for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
-                reinterpret_cast<uint4 *>(out_act + t * d)[v] = out.raw;
-            } else {
+                for (int i = 0; i < VN; ++i) acc[i] = 0.0f;
 #pragma unroll
-                for (int i = 0; i < VN; ++i) out_f32[t * d + (int64_t)v * VN + i] = acc[i];
+                for (int s = 0; s < KT; ++s)
+                    if (s < k) {
+#pragma unroll
+                        for (int i = 0; i < VN; ++i) acc[i] += in[s][b].get(i);
+                    }
+                if (add) {
+#pragma unroll
+                    for (int q = 0; q < VN / 4; ++q) {
+                        acc[4 * q] += addv[b][q].x; acc[4 * q + 1] += addv[b][q].y;
+                        acc[4 * q + 2] += addv[b][q].z; acc[4 * q + 3] += addv[b][q].w;
+                    }
+                }
+                const int64_t at = t * d + (int64_t)(v0 + 32 * b) * VN;
+                if (out_act) {
+                    Vec16<XT> out;
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
+                    *reinterpret_cast<uint4 *>(out_act + at) = out.raw;
+                } else {
+#pragma unroll
+                    for (int q = 0; q < VN / 4; ++q)
+                        reinterpret_cast<float4 *>(out_f32 + at)[q] =
+                            make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+                }
             }
         }
     }
@@ -415,12 +473,15 @@ int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_per
                             int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
-    if (act == MOE_BF16)
-        dispatch_bwd_kernel<bf16><<<grid, 256, 0, st>>>((const bf16 *)dxs, inv_perm, T, k, d, add_f32, out_f32,
-                                                         (bf16 *)out_act);
-    else
-        dispatch_bwd_kernel<float><<<grid, 256, 0, st>>>((const float *)dxs, inv_perm, T, k, d, add_f32, out_f32,
-                                                          (float *)out_act);
+#define MOE_CALL(KT, VB)                                                                                              \
+    if (act == MOE_BF16)                                                                                              \
+        dispatch_bwd_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)dxs, inv_perm, T, k, d, add_f32, out_f32, \
+                                                                 (bf16 *)out_act);                                     \
+    else                                                                                                              \
+        dispatch_bwd_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)dxs, inv_perm, T, k, d, add_f32,       \
+                                                                  out_f32, (float *)out_act)
+    MOE_DISPATCH_KT(k, MOE_CALL);
+#undef MOE_CALL
     MOE_LAUNCHED();
     return MOE_OK;
 }
