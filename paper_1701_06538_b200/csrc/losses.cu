@@ -55,6 +55,67 @@ __global__ void __launch_bounds__(256) level_sums_kernel(const int32_t *__restri
     }
 }
 
+// Same sums with one warp per row and the lanes across the columns (n <= 32 * NV): all loads of a row are
+// issued first, a lane accumulates its columns over the rows of its warp, the block's 8 warps are then added
+// in order through shared memory.
+template <int NV>
+__global__ void __launch_bounds__(256) level_sums_rows_kernel(const int32_t *__restrict__ idx,
+                                                              const float *__restrict__ gates,
+                                                              const float *__restrict__ clean,
+                                                              const float *__restrict__ raw,
+                                                              const float *__restrict__ kth_vals, int64_t rows,
+                                                              int32_t n, int32_t k, float *__restrict__ part_imp,
+                                                              float *__restrict__ part_load) {
+    __shared__ float red[2][8][32 * NV];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t per = (rows + gridDim.x - 1) / gridDim.x;
+    const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(r0 + per, rows);
+    float s_imp[NV], s_load[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) s_imp[u] = s_load[u] = 0.0f;
+    for (int64_t t = r0 + w; t < r1; t += 8) {
+        float cv[NV], rv[NV];
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int32_t j = lane + 32 * u;
+            cv[u] = j < n ? clean[t * n + j] : 0.0f;
+            rv[u] = j < n ? raw[t * n + j] : 0.0f;
+        }
+        int32_t sel_idx[MOE_MAX_K];
+        float sel_g[MOE_MAX_K];
+#pragma unroll
+        for (int s = 0; s < MOE_MAX_K; ++s) {
+            sel_idx[s] = s < k ? idx[t * k + s] : -1;
+            sel_g[s] = s < k ? gates[t * k + s] : 0.0f;
+        }
+        const float thr_unsel = kth_vals[t * 2 + 0], thr_sel = kth_vals[t * 2 + 1];
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int32_t j = lane + 32 * u;
+            if (j < n) {
+                bool sel = false;
+                float g = 0.0f;
+#pragma unroll
+                for (int s = 0; s < MOE_MAX_K; ++s)
+                    if (sel_idx[s] == j) { sel = true; g = sel_g[s]; }
+                const float z = (cv[u] - (sel ? thr_sel : thr_unsel)) / softplus_f(rv[u]);
+                s_load[u] += 0.5f * erfcf(-z * 0.70710678118654752440f);  // Phi(z)
+                s_imp[u] += g;
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < NV; ++u) { red[0][w][lane + 32 * u] = s_imp[u]; red[1][w][lane + 32 * u] = s_load[u]; }
+    __syncthreads();
+    for (int32_t j = threadIdx.x; j < n; j += 256) {
+        float a = 0.0f, b = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { a += red[0][q][j]; b += red[1][q][j]; }
+        part_imp[(int64_t)blockIdx.x * n + j] = a;
+        part_load[(int64_t)blockIdx.x * n + j] = b;
+    }
+}
+
 __global__ void __launch_bounds__(256) level_reduce_kernel(const float *__restrict__ part_imp,
                                                            const float *__restrict__ part_load, int32_t chunks,
                                                            int32_t n, float *__restrict__ importance,
@@ -62,7 +123,18 @@ __global__ void __launch_bounds__(256) level_reduce_kernel(const float *__restri
     const int32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
     double a = 0.0, b = 0.0;
-    for (int32_t c = 0; c < chunks; ++c) {
+    int32_t c = 0;
+    for (; c + 8 <= chunks; c += 8) {  // eight independent loads in flight, added in order
+        float pa[8], pb[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            pa[q] = part_imp[(int64_t)(c + q) * n + j];
+            pb[q] = part_load[(int64_t)(c + q) * n + j];
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { a += (double)pa[q]; b += (double)pb[q]; }
+    }
+    for (; c < chunks; ++c) {
         a += (double)part_imp[(int64_t)c * n + j];
         b += (double)part_load[(int64_t)c * n + j];
     }
@@ -82,7 +154,11 @@ int32_t launch_level_sums(const int32_t *idx, const float *gates, const float *c
     int32_t CW = 1;
     while (CW < n && CW < 256) CW <<= 1;
     float *part_imp = scratch, *part_load = scratch + (int64_t)chunks * n;
-    level_sums_kernel<<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, CW, part_imp, part_load);
+    if (n <= 32) level_sums_rows_kernel<1><<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, part_imp, part_load);
+    else if (n <= 64) level_sums_rows_kernel<2><<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, part_imp, part_load);
+    else if (n <= 128) level_sums_rows_kernel<4><<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, part_imp, part_load);
+    else if (n <= 256) level_sums_rows_kernel<8><<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, part_imp, part_load);
+    else level_sums_kernel<<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, CW, part_imp, part_load);
     MOE_LAUNCHED();
     level_reduce_kernel<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(part_imp, part_load, chunks, n, importance_out,
                                                                  load_out);
