@@ -145,6 +145,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
         : "memory");
 }
 
+// 256-bit store (sm_100): a whole 32-byte sector per instruction
+__device__ __forceinline__ void st_global_32B(uint4 *dst, const uint4 &a, const uint4 &b) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(a.x), "r"(a.y), "r"(a.z),
+                 "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -474,8 +480,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
                     uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) dst[q] = packed[q];
+                    st_global_32B(dst, packed[0], packed[1]);      // two full 32-byte sectors per row piece
+                    st_global_32B(dst + 2, packed[2], packed[3]);
                 }
             }
             if (have_acc) {
@@ -839,8 +845,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
                     uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) dst[q] = packed[q];
+                    st_global_32B(dst, packed[0], packed[1]);      // two full 32-byte sectors per row piece
+                    st_global_32B(dst + 2, packed[2], packed[3]);
                 }
             }
             if (MASKT) {

@@ -319,14 +319,18 @@ __global__ void __launch_bounds__(256) split_gate_weights_kernel(const float *__
     }
 }
 
+// one warp per column of [W_g | W_noise]
 __global__ void __launch_bounds__(256) gate_col_norms_kernel(const float *__restrict__ Wg, const float *__restrict__ Wn,
                                                              int32_t d, int32_t n, float *__restrict__ wnorm) {
-    const int32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int32_t j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (j >= 2 * n) return;
     const float *W = j < n ? Wg + j : Wn + (j - n);
     double s = 0.0;
-    for (int32_t q = 0; q < d; ++q) { const double v = W[(int64_t)q * n]; s += v * v; }
-    wnorm[j] = (float)(sqrt(s) * (1.0 + 1e-6));
+    for (int32_t q = lane; q < d; q += 32) { const double v = W[(int64_t)q * n]; s += v * v; }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) wnorm[j] = (float)(sqrt(s) * (1.0 + 1e-6));
 }
 
 template <typename XT>
@@ -474,7 +478,7 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
                                    int32_t *unsafe_count, cudaStream_t st) {
     split_gate_weights_kernel<<<(unsigned)cdiv((int64_t)d * 2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
     MOE_LAUNCHED();
-    gate_col_norms_kernel<<<(unsigned)cdiv(2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
+    gate_col_norms_kernel<<<(unsigned)cdiv(2 * n, 8), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
     MOE_LAUNCHED();
     if (act == MOE_BF16) row_norms_kernel<bf16><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const bf16 *)x, T, d, xnorm);
     else row_norms_kernel<float><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const float *)x, T, d, xnorm);
