@@ -11,7 +11,7 @@
  *    allocates or frees device memory, keeps no state between calls and never synchronises
  *    the host with the device (except moe_check_status, which says so). All work is enqueued
  *    on `stream` (a cudaStream_t passed as void*; NULL is the default stream).
- *  - Tensors are row-major, contiguous, and start on a 16-byte boundary (256-byte for the
+ *  - Tensors are row-major, contiguous, and start on a 32-byte boundary (256-byte for the
  *    workspace and the context). Outputs are overwritten, not accumulated into.
  *  - "act" tensors (x, xs, hid, ys, y, W1, b1, W2, b2 and their gradients) have the element
  *    type moe_config.act (float or bfloat16). Gating tensors (W_g, W_noise, noise, clean,
@@ -120,6 +120,10 @@ int32_t moe_check_status(const void *ws, void *stream);
  * The logits that decide the routing are evaluated in single precision in one fixed order
  * (one fused-multiply-add chain per output over ascending input feature; softplus in double
  * rounded once; H by one fused multiply-add), so the routing is reproducible bit for bit.
+ * For large bf16 batches the routing is first screened with a tensor-core product and an error
+ * bound; tokens whose order the bound proves keep that result (indices identical to the chain's,
+ * clean / raw_noise / kth_vals within 1e-7 of it), all other tokens are redone with the chain.
+ * Environment: MOE_GATE_SCREEN=0 disables the screen, =1 uses it whenever the shapes allow.
  * `noise` is an input: standard normal draws, or zeros for noiseless gating.
  * in : x [T,d] act, Wg/Wnoise [d,n], noise [T,n]
  * out: topk_idx [T,k], gates [T,k], clean [T,n], raw_noise [T,n], kth_vals [T,2], kth_idx [T,2] */

@@ -39,7 +39,7 @@ template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __f
 static inline size_t act_bytes(int32_t act) { return act == MOE_BF16 ? 2 : 4; }
 static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline int64_t imin(int64_t a, int64_t b) { return a < b ? a : b; }
-static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31) == 0; }  // 32 bytes: the epilogues use 256-bit stores
 
 // Carves 256-byte aligned pieces out of a workspace. With base == nullptr it only measures,
 // so the size queries and the calls that use the workspace run the same code.
