@@ -147,7 +147,7 @@ struct HierIdxWs {
         counts_p = cv.take<int32_t>(D.a);
         offsets_p = cv.take<int32_t>(D.a + 1);
         scratch = cv.take<int32_t>(dispatch_ws_elems(D.T * D.k1, (int32_t)D.a));
-        tile_prefix = cv.take<int32_t>(D.a + 1);
+        tile_prefix = cv.take<int32_t>(tc_tile_ws_ints(D.T * D.k1, D.a));  // prefix + tile table of the secondary-gate GEMMs
     }
     int32_t build(const Dims &D, const int32_t *topk_idx, cudaStream_t st) {
         MOE_TRY(launch_hier_split_idx(topk_idx, D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.b, idx_p, idx_s, st));
@@ -180,8 +180,13 @@ struct FfnBwdWs {
     float *colsum;
     FfnBwdWs(Carver &cv, const Dims &D) {
         dz = cv.take_bytes(D.R * D.h * (int64_t)D.esz);
-        tile_prefix = cv.take<int32_t>(D.n + 1);
-        colsum = cv.take<float>(colsum_ws_floats(D.R, (int32_t)D.n, (int32_t)(D.h > D.d ? D.h : D.d)));
+        tile_prefix = cv.take<int32_t>(tc_tile_ws_ints(D.R, D.n));  // prefix + tile table of the row GEMMs
+        int64_t cs = colsum_ws_floats(D.R, (int32_t)D.n, (int32_t)(D.h > D.d ? D.h : D.d));
+        if (D.act == MOE_BF16) {  // the tensor-core path sums dz's columns per 32-row block in the GEMM epilogue
+            const int64_t cs_tc = tc_colsum_part_floats(D.R, (int32_t)D.n, (int32_t)D.h);
+            if (cs_tc > cs) cs = cs_tc;
+        }
+        colsum = cv.take<float>(cs);
     }
 };
 

@@ -49,7 +49,10 @@ constexpr int MAX_TERMS = 8;
 
 struct GemmParams {
     const int32_t *offsets;      // [nseg + 1] segment bounds (rows); nullptr = uniform segments
-    const int32_t *tile_prefix;  // ROW_* with offsets: [nseg + 1] prefix of 128-row tiles
+    const int32_t *tile_prefix;  // ROW_* with offsets: [nseg + 1] prefix of the M tiles
+    const int4 *tile_info;       // ROW_* with offsets: per M tile {segment or -1, first row, segment end, 0}
+    // set by the launchers: N tiles per row of tiles, WGRAD tiles per segment, number of tile ids, K blocks of a ROW tile
+    int32_t tiles_n, per_e, total_tiles, kblocks_row;
     int32_t nseg;
     int32_t M;  // WGRAD: rows of the per-segment output; ROW_*: unused
     int32_t N;  // output columns
@@ -58,6 +61,9 @@ struct GemmParams {
     float *out_f32;    // if set, results are written here as float instead of `out`
     const bf16 *bias;  // [nseg, N] or nullptr
     const bf16 *mask;  // [R, N] or nullptr: result kept where mask > 0
+    // ROW_* with bf16 output: if set, column sums of the stored values over each epilogue warp's 32 rows,
+    // [32-row block][N] floats; block = (global M tile * CTAs per tile + CTA rank) * 4 + row quarter
+    float *colsum_part;
     int32_t relu;
     int32_t *status;
     // uniform segments (offsets == nullptr): ROW_*: one segment of R rows. WGRAD: segment s covers
@@ -66,7 +72,7 @@ struct GemmParams {
     int64_t R;
     int32_t rows_per_seg, segs_per_term, b_term_chunks;
     int32_t segs_term0, rows_per_seg0;  // if segs_term0 > 0: term 0 is cut into that many ranges of rows_per_seg0
-    int32_t off_mod;                    // WGRAD with offsets: see decode_tile
+    int32_t off_mod;                    // WGRAD with offsets: see tile_fetch
     // ROW_*: the contraction is the concatenation of nterms pieces of length K; piece i reads A
     // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
     int32_t nterms;
@@ -197,6 +203,22 @@ __host__ __device__ constexpr uint32_t make_idesc(int a_mn, int b_mn) {
            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// Column sums over the 32 rows a warp holds (one row per lane, 32 columns per lane): returns in lane l
+// the sum of column l. Butterfly: each step a lane keeps one half of its columns and sends the other.
+__device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool up = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            const float keep = up ? a[i + s] : a[i];
+            const float send = up ? a[i] : a[i + s];
+            a[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    return a[0];
+}
+
 struct Tile {
     int32_t e;        // expert / segment
     int32_t row0;     // ROW_*: first sorted row; WGRAD: first row of the segment
@@ -205,32 +227,46 @@ struct Tile {
     int32_t n0;       // first output column
     int32_t kblocks;  // number of K blocks
     int32_t b_chunk;  // WGRAD: first 64-column chunk of B
+    int32_t mt;       // ROW_*: index of the M tile over all segments
 };
 
-template <int KIND, int TM = BM>
-__device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Tile &t) {
-    const int32_t tiles_n = (p.N + BN - 1) / BN;
+// Tile ids are handed out round-robin. What a tile needs from global memory (its segment's bounds) is
+// fetched one tile ahead (tile_fetch) and only turned into a Tile (tile_decode) when the tile starts, so
+// the load latency never sits between two tiles. ROW_* with ragged segments read one 16-byte record per
+// M tile from a table built by tile_table_kernel; WGRAD reads the two segment bounds.
+template <int KIND>
+__device__ __forceinline__ int4 tile_fetch(const GemmParams &p, int32_t id) {
+    if (!p.offsets || id >= p.total_tiles) return make_int4(-1, 0, 0, 0);
     if (KIND == WGRAD) {
-        const int32_t tiles_m = (p.M + TM - 1) / TM;
-        const int64_t per_e = (int64_t)tiles_m * tiles_n;
-        if (id >= per_e * p.nseg) return false;
-        t.e = (int32_t)(id / per_e);
-        const int32_t rem = (int32_t)(id % per_e);
-        t.m0 = (rem / tiles_n) * TM;
-        t.n0 = (rem % tiles_n) * BN;
+        const int32_t e = id / p.per_e;
+        const int32_t seg = p.off_mod > 0 ? e % p.off_mod : e;  // with off_mod: segment s reads the rows of group s % off_mod
+        return make_int4(e, p.offsets[seg], p.offsets[seg + 1], 0);
+    }
+    return p.tile_info[id / p.tiles_n];
+}
+
+template <int KIND, int TM>
+__device__ __forceinline__ bool tile_decode(const GemmParams &p, int32_t id, const int4 &raw, Tile &t) {
+    if (id >= p.total_tiles) return false;
+    if (KIND == WGRAD) {
+        const int32_t e = id / p.per_e, rem = id - e * p.per_e;
+        const int32_t tm = rem / p.tiles_n;
+        t.e = e;
+        t.mt = 0;
+        t.m0 = tm * TM;
+        t.n0 = (rem - tm * p.tiles_n) * BN;
         t.b_chunk = t.n0 / 64;
-        if (p.offsets) {  // with off_mod: segment s reads the rows of group s % off_mod, B term s / off_mod
-            const int32_t seg = p.off_mod > 0 ? t.e % p.off_mod : t.e;
-            t.row0 = p.offsets[seg];
-            t.row_end = p.offsets[seg + 1];
-            if (p.off_mod > 0) t.b_chunk += (t.e / p.off_mod) * p.b_term_chunks;
+        if (p.offsets) {
+            t.row0 = raw.y;
+            t.row_end = raw.z;
+            if (p.off_mod > 0) t.b_chunk += (e / p.off_mod) * p.b_term_chunks;  // B term s / off_mod
         } else {
             int64_t c, rps;
             int32_t term;
-            if (t.e < p.segs_term0) {  // term 0 may use its own (shorter) row ranges
-                c = t.e; rps = p.rows_per_seg0; term = 0;
+            if (e < p.segs_term0) {  // term 0 may use its own (shorter) row ranges
+                c = e; rps = p.rows_per_seg0; term = 0;
             } else {
-                const int32_t e2 = t.e - p.segs_term0;
+                const int32_t e2 = e - p.segs_term0;
                 c = e2 % p.segs_per_term; rps = p.rows_per_seg;
                 term = e2 / p.segs_per_term + (p.segs_term0 > 0 ? 1 : 0);
             }
@@ -242,31 +278,40 @@ __device__ __forceinline__ bool decode_tile(const GemmParams &p, int64_t id, Til
         t.kblocks = (t.row_end - t.row0 + BK - 1) / BK;
         return true;
     } else {
+        const int32_t mt = id / p.tiles_n;
+        t.mt = mt;
         t.m0 = 0;
         t.b_chunk = 0;
-        t.kblocks = p.nterms * (p.K / BK);
-        t.n0 = (int32_t)(id % tiles_n) * BN;
-        const int32_t mt = (int32_t)(id / tiles_n);
-        if (!p.offsets) {
-            if ((int64_t)mt * TM >= p.R) return false;
+        t.kblocks = p.kblocks_row;
+        t.n0 = (id - mt * p.tiles_n) * BN;
+        if (!p.offsets) {  // one segment of R rows; total_tiles is exact
             t.e = 0;
             t.row0 = mt * TM;
             t.row_end = (int32_t)p.R;
             return true;
         }
-        const int32_t total_m = p.tile_prefix[p.nseg];
-        if (id >= (int64_t)total_m * tiles_n) return false;
-        int lo = 0, hi = p.nseg;
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (p.tile_prefix[mid] <= mt) lo = mid; else hi = mid;
-        }
-        t.e = lo;
-        t.row0 = p.offsets[lo] + (mt - p.tile_prefix[lo]) * TM;
-        t.row_end = p.offsets[lo + 1];
+        if (raw.x < 0) return false;  // past the last M tile
+        t.e = raw.x;
+        t.row0 = raw.y;
+        t.row_end = raw.z;
         return true;
     }
 }
+
+template <int KIND, int TM> struct TileIter {
+    const GemmParams &p;
+    int32_t id, stride;
+    int4 raw;
+    __device__ __forceinline__ TileIter(const GemmParams &p_, int32_t first, int32_t stride_)
+        : p(p_), id(first), stride(stride_) { raw = tile_fetch<KIND>(p, id); }
+    // the current tile; starts the fetch for the following one
+    __device__ __forceinline__ bool next(Tile &t) {
+        if (!tile_decode<KIND, TM>(p, id, raw, t)) return false;
+        id += stride;
+        raw = tile_fetch<KIND>(p, id);
+        return true;
+    }
+};
 
 template <int KIND>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -310,9 +355,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
-                Tile t;
-                if (!decode_tile<KIND>(p, id, t)) break;
+            TileIter<KIND, BM> it(p, (int32_t)blockIdx.x, (int32_t)gridDim.x);
+            Tile t;
+            while (ok && it.next(t)) {
+                int term = 0, kk = 0;  // ROW_*: piece of the contraction and column inside it
                 for (int kb = 0; kb < t.kblocks && ok; ++kb) {
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
@@ -323,10 +369,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         tma_load_3d(a_dst, &tmA, full_bar(s), 0, r, t.m0 / 64);
                         tma_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk);
                     } else {
-                        const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
                         tma_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0);
                         if (KIND == ROW_BMN) tma_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64, t.e);
                         else tma_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0, t.e);
+                        kk += BK;
+                        if (kk == p.K) { kk = 0; ++term; }
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -345,9 +392,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int s = 0, acc = 0;
         uint32_t ph = 0, acc_ph = 0;
         bool ok = true;
-        for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
-            Tile t;
-            if (!decode_tile<KIND>(p, id, t)) break;
+        TileIter<KIND, BM> it(p, (int32_t)blockIdx.x, (int32_t)gridDim.x);
+        Tile t;
+        while (ok && it.next(t)) {
             if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
             ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
             if (!ok) break;
@@ -398,9 +445,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
-        for (int64_t id = blockIdx.x; ok; id += gridDim.x) {
-            Tile t;
-            if (!decode_tile<KIND>(p, id, t)) break;
+        TileIter<KIND, BM> it(p, (int32_t)blockIdx.x, (int32_t)gridDim.x);
+        Tile t;
+        while (ok && it.next(t)) {
             const bool have_acc = t.kblocks > 0;
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
@@ -452,7 +499,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                 *reinterpret_cast<const uint4 *>(stage_o + row * 128 + ((my_piece ^ (row & 7)) << 4));
                     }
                     __syncwarp();
-                } else if (row_ok) {
+                } else if (row_ok || p.colsum_part) {  // with column sums the whole warp takes part (shuffles)
                     uint4 packed[4];
                     uint4 bias_raw[4], mask_raw[4];
                     if (p.bias) {
@@ -460,7 +507,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int q = 0; q < 4; ++q)
                             bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
                     }
-                    if (p.mask) {
+                    if (p.mask && row_ok) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
@@ -479,9 +526,22 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
-                    st_global_32B(dst, packed[0], packed[1]);      // two full 32-byte sectors per row piece
-                    st_global_32B(dst + 2, packed[2], packed[3]);
+                    if (row_ok) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
+                        st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
+                        st_global_32B(dst + 2, packed[2], packed[3]);
+                    }
+                    if (p.colsum_part) {  // sums of the rounded values, rows past the segment end count as 0
+                        float a[32];
+                        const uint32_t *pw = reinterpret_cast<const uint32_t *>(packed);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            a[2 * j] = row_ok ? __uint_as_float(pw[j] << 16) : 0.0f;
+                            a[2 * j + 1] = row_ok ? __uint_as_float(pw[j] & 0xffff0000u) : 0.0f;
+                        }
+                        const float sum = warp_column_sums(a, lane);
+                        p.colsum_part[(int64_t)(t.mt * 4 + quarter) * p.N + col0 + lane] = sum;
+                    }
                 }
             }
             if (have_acc) {
@@ -629,9 +689,10 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int s = 0;
             uint32_t ph = 0, mask_ph = 0;
             bool ok = true;
-            for (int64_t id = cluster_id; ok; id += n_clusters) {
-                Tile t;
-                if (!decode_tile<KIND, 256>(p, id, t)) break;
+            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            Tile t;
+            while (ok && it.next(t)) {
+                int term = 0, kk = 0;  // ROW_*: piece of the contraction and column inside it
                 for (int kb = 0; kb < t.kblocks && ok; ++kb) {
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
@@ -649,12 +710,13 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         tma2_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk + 2 * (int)rank);
                     } else {
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
-                        const int per_term = p.K / BK, term = kb / per_term, kk = (kb % per_term) * BK;
                         tma2_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0 + 128 * (int)rank);
                         if (KIND == ROW_BMN)
                             tma2_load_4d(b_dst, &tmB, full_bar(s), 0, p.b_term_col[term] + kk, t.n0 / 64 + 2 * (int)rank, t.e);
                         else
                             tma2_load_3d(b_dst, &tmB, full_bar(s), p.b_term_col[term] + kk, t.n0 + 128 * (int)rank, t.e);
+                        kk += BK;
+                        if (kk == p.K) { kk = 0; ++term; }
                     }
                     if (++s == NST) { s = 0; ph ^= 1u; }
                 }
@@ -689,9 +751,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0, tail_ph = 0;  // tail_ph: one phase bit per stage for afull / ready
             bool ok = true;
-            for (int64_t id = cluster_id; ok; id += n_clusters) {
-                Tile t;
-                if (!decode_tile<KIND, 256>(p, id, t)) break;
+            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            Tile t;
+            while (ok && it.next(t)) {
                 if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
                 ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
@@ -734,9 +796,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int s = 0;
             uint32_t tail_ph = 0;
             bool ok = true;
-            for (int64_t id = cluster_id; ok; id += n_clusters) {
-                Tile t;
-                if (!decode_tile<KIND, 256>(p, id, t)) break;
+            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            Tile t;
+            while (ok && it.next(t)) {
                 for (int kb = 0; kb < t.kblocks; ++kb) {
                     const int valid = t.row_end - (t.row0 + kb * BK);
                     if (valid < BK) {
@@ -759,9 +821,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
-        for (int64_t id = cluster_id; ok; id += n_clusters) {
-            Tile t;
-            if (!decode_tile<KIND, 256>(p, id, t)) break;
+        TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+        Tile t;
+        while (ok && it.next(t)) {
             const bool have_acc = t.kblocks > 0;
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
@@ -811,7 +873,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                 *reinterpret_cast<const uint4 *>(stage_o + row * 128 + ((my_piece ^ (row & 7)) << 4));
                     }
                     __syncwarp();
-                } else if (row_ok) {
+                } else if (row_ok || p.colsum_part) {  // with column sums the whole warp takes part (shuffles)
                     uint4 packed[4];
                     uint4 bias_raw[4], mask_raw[4];
                     if (p.bias) {
@@ -825,7 +887,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = *reinterpret_cast<const uint4 *>(mrow_p + ((((c & 1) * 4 + q) ^ (mrow & 7)) << 4));
-                    } else if (p.mask) {
+                    } else if (p.mask && row_ok) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
@@ -844,9 +906,22 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         }
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
-                    st_global_32B(dst, packed[0], packed[1]);      // two full 32-byte sectors per row piece
-                    st_global_32B(dst + 2, packed[2], packed[3]);
+                    if (row_ok) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
+                        st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
+                        st_global_32B(dst + 2, packed[2], packed[3]);
+                    }
+                    if (p.colsum_part) {  // sums of the rounded values, rows past the segment end count as 0
+                        float a[32];
+                        const uint32_t *pw = reinterpret_cast<const uint32_t *>(packed);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            a[2 * j] = row_ok ? __uint_as_float(pw[j] << 16) : 0.0f;
+                            a[2 * j + 1] = row_ok ? __uint_as_float(pw[j] & 0xffff0000u) : 0.0f;
+                        }
+                        const float sum = warp_column_sums(a, lane);
+                        p.colsum_part[(int64_t)((t.mt * 2 + (int)rank) * 4 + quarter) * p.N + col0 + lane] = sum;
+                    }
                 }
             }
             if (MASKT) {
@@ -965,8 +1040,20 @@ int sm_count() {
     return n;
 }
 
-template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p,
+// Derived tile counts the device code divides by; ids are 32-bit.
+template <int KIND, int TM> int32_t complete_params(GemmParams &q, int64_t max_tiles) {
+    if (max_tiles >= ((int64_t)1 << 31) - ((int64_t)1 << 22)) return MOE_ERR_UNSUPPORTED;
+    q.tiles_n = (int32_t)cdiv(q.N, BN);
+    q.per_e = KIND == WGRAD ? (int32_t)cdiv(q.M, TM) * q.tiles_n : 1;
+    q.total_tiles = (int32_t)max_tiles;
+    q.kblocks_row = KIND == WGRAD ? 0 : q.nterms * (q.K / BK);
+    return MOE_OK;
+}
+
+template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p_in,
                                    int64_t max_tiles, cudaStream_t st) {
+    GemmParams p = p_in;
+    MOE_TRY((complete_params<KIND, BM>(p, max_tiles)));
     static bool configured = false;
     if (!configured) {
         MOE_CUDA(cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
@@ -980,8 +1067,10 @@ template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tm
 }
 
 template <int KIND, bool MASKT = false>
-int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p, int64_t max_tiles,
+int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p_in, int64_t max_tiles,
                 cudaStream_t st, const CUtensorMap *tmM = nullptr) {
+    GemmParams p = p_in;
+    MOE_TRY((complete_params<KIND, 256>(p, max_tiles)));
     static int max_clusters = 0;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -1010,7 +1099,8 @@ bool tc_ffn_supported(const moe_config &c) {
     return c.act == MOE_BF16 && c.d % 64 == 0 && c.h % 64 == 0 && c.d >= 64 && c.h >= 64;
 }
 
-int64_t tc_ffn_ws_bytes(const moe_config &c) { return ((int64_t)(c.n + 1) * 4 + 255) & ~255ll; }
+int64_t tc_tile_ws_ints(int64_t R, int64_t nseg);
+int64_t tc_ffn_ws_bytes(const moe_config &c) { return (tc_tile_ws_ints((int64_t)c.T * c.k, c.n) * 4 + 255) & ~255ll; }
 
 // The 256-row tiles of the two-CTA kernel pay off when the average segment fills them.
 static bool use_two_cta(int64_t R, int32_t nseg) {
@@ -1021,32 +1111,145 @@ static bool use_two_cta(int64_t R, int32_t nseg) {
 
 // C[rows, N] = epilogue(A[rows, K] . B_e) over the segments; B_e = W[e] as [K, N] (transposed = false)
 // or as [N, K] read transposed (transposed = true).
+// Tile table of a ragged row GEMM: tile_prefix[e] = number of tm-row tiles of the segments before e
+// (tile_prefix[nseg] = total), and one record per M tile {segment, first row, segment end, 0}; records past
+// the last tile carry segment -1. One block.
+__global__ void __launch_bounds__(1024) tile_table_kernel(const int32_t *__restrict__ offsets, int32_t n, int32_t tm,
+                                                          int32_t max_m, int32_t *__restrict__ tile_prefix,
+                                                          int4 *__restrict__ info) {
+    __shared__ int32_t warp_sum[32];
+    __shared__ int32_t carry;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int32_t base = 0; base < n; base += 1024) {
+        const int32_t e = base + threadIdx.x;
+        const int32_t v = e < n ? (offsets[e + 1] - offsets[e] + tm - 1) / tm : 0;
+        int32_t inc = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t o = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += o;
+        }
+        if (lane == 31) warp_sum[w] = inc;
+        __syncthreads();
+        if (w == 0) {
+            const int32_t sw = warp_sum[lane];
+            int32_t si = sw;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t o = __shfl_up_sync(0xffffffffu, si, off);
+                if (lane >= off) si += o;
+            }
+            warp_sum[lane] = si - sw;
+        }
+        __syncthreads();
+        const int32_t excl = carry + warp_sum[w] + inc - v;
+        if (e < n) tile_prefix[e] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) tile_prefix[n] = carry;
+    __syncthreads();  // the prefix (global memory, this block's own writes) is complete
+    const int32_t total = carry;
+    for (int32_t mt = threadIdx.x; mt < max_m; mt += 1024) {
+        if (mt >= total) { info[mt] = make_int4(-1, 0, 0, 0); continue; }
+        int lo = 0, hi = n;  // last e with tile_prefix[e] <= mt (empty segments share a prefix: take the last)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (tile_prefix[mid] <= mt) lo = mid; else hi = mid;
+        }
+        info[mt] = make_int4(lo, offsets[lo] + (mt - tile_prefix[lo]) * tm, offsets[lo + 1], 0);
+    }
+}
+
+// ints a tile table needs behind its [nseg + 1] prefix (records are 16 bytes, 16-byte aligned)
+int64_t tc_tile_ws_ints(int64_t R, int64_t nseg) { return ((nseg + 1 + 3) & ~(int64_t)3) + 4 * (cdiv(R, 128) + nseg + 1); }
+static int4 *tile_info_of(int32_t *tile_prefix, int32_t nseg) {
+    return reinterpret_cast<int4 *>(tile_prefix + ((nseg + 1 + 3) & ~3));
+}
+static int32_t launch_tile_table(const int32_t *offsets, int32_t nseg, int32_t tm, int64_t R, int32_t *tile_prefix,
+                                 cudaStream_t st) {
+    tile_table_kernel<<<1, 1024, 0, st>>>(offsets, nseg, tm, (int32_t)(cdiv(R, tm) + nseg), tile_prefix,
+                                          tile_info_of(tile_prefix, nseg));
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+// Sum of the epilogue's 32-row column sums over each segment (bias gradient), G blocks per M tile.
+// A thread block takes 32 columns of one segment; its 8 warps take the blocks b = b0 + w, b0 + w + 8, ...
+// and the 8 sums are added in warp order: the result does not depend on timing.
+__global__ void __launch_bounds__(256) colsum_blocks_final_kernel(const float *__restrict__ part, int32_t N,
+                                                                  const int32_t *__restrict__ tile_prefix, int32_t G,
+                                                                  bf16 *__restrict__ out) {
+    __shared__ float sh[8][32];
+    const int32_t e = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int32_t j = blockIdx.y * 32 + lane;  // N is a multiple of 64
+    const int32_t b0 = tile_prefix[e] * G, b1 = tile_prefix[e + 1] * G;
+    float s = 0.0f;
+    int32_t b = b0 + w;
+    for (; b + 24 < b1; b += 32) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = part[(int64_t)(b + 8 * u) * N + j];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) s += v[u];
+    }
+    for (; b < b1; b += 8) s += part[(int64_t)b * N + j];
+    sh[w][lane] = s;
+    __syncthreads();
+    if (w == 0) {
+        float t = sh[0][lane];
+#pragma unroll
+        for (int u = 1; u < 8; ++u) t += sh[u][lane];
+        out[(int64_t)e * N + j] = __float2bfloat16_rn(t);
+    }
+}
+
+int64_t tc_colsum_part_floats(int64_t R, int32_t nseg, int32_t N) { return (cdiv(R, 128) * 4 + 8 * (int64_t)nseg + 8) * N; }
+
+// colsum_part / colsum_out: if set, out's column sums per segment (a bias gradient) are formed in the epilogue
+// and reduced into colsum_out [nseg, N]; colsum_part needs tc_colsum_part_floats(R, nseg, N) floats
 int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t *offsets, int32_t nseg, int64_t R,
                     int32_t N, int32_t K, void *out, const void *bias, const void *mask, int relu,
-                    int32_t *tile_prefix, int32_t *status, cudaStream_t st) {
-    if (R == 0) return MOE_OK;
+                    int32_t *tile_prefix, int32_t *status, cudaStream_t st, float *colsum_part = nullptr,
+                    void *colsum_out = nullptr) {
+    if (R == 0) {
+        if (colsum_out) MOE_CUDA(cudaMemsetAsync(colsum_out, 0, sizeof(bf16) * (size_t)nseg * N, st));
+        return MOE_OK;
+    }
+    auto finish = [&](int32_t rc, int32_t G) -> int32_t {
+        if (rc != MOE_OK || !colsum_out) return rc;
+        colsum_blocks_final_kernel<<<dim3((unsigned)nseg, (unsigned)(N / 32)), 256, 0, st>>>(colsum_part, N, tile_prefix, G,
+                                                                                                   (bf16 *)colsum_out);
+        MOE_LAUNCHED();
+        return MOE_OK;
+    };
     CUtensorMap tmA, tmB;
     MOE_TRY(map_rows_kmajor(&tmA, A, R, K));
     GemmParams p = default_params();
-    p.offsets = offsets; p.tile_prefix = tile_prefix; p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
+    p.offsets = offsets; p.tile_prefix = tile_prefix; p.tile_info = tile_info_of(tile_prefix, nseg);
+    p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
     p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
+    p.colsum_part = colsum_out ? colsum_part : nullptr;
     if (use_two_cta(R, nseg)) {  // segments long enough to fill 256-row tiles: SM pairs
         if (transposed) MOE_TRY(map_weight_kmajor_half(&tmB, W, nseg, N, K));
         else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
-        MOE_TRY(launch_tile_prefix(offsets, nseg, 256, tile_prefix, st));
+        MOE_TRY(launch_tile_table(offsets, nseg, 256, R, tile_prefix, st));
         const int64_t max_tiles2 = (cdiv(R, 256) + nseg) * cdiv(N, BN);
         if (transposed && mask) {  // the ReLU-mask rows come in as TMA tiles
             CUtensorMap tmM;
             MOE_TRY(map_rows_kmajor(&tmM, mask, R, N));
-            return launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM);
+            return finish(launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM), 8);
         }
-        return transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st) : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st);
+        return finish(transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st) : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st), 8);
     }
     if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
     else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
-    MOE_TRY(launch_tile_prefix(offsets, nseg, BM, tile_prefix, st));
+    MOE_TRY(launch_tile_table(offsets, nseg, BM, R, tile_prefix, st));
     const int64_t max_tiles = (cdiv(R, BM) + nseg) * cdiv(N, BN);
-    return transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st);
+    return finish(transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st), 4);
 }
 
 // dW[e] [M, N] = A_e^T . B_e, contraction over the rows of segment e; A [R, M], B [R, N]
@@ -1227,9 +1430,10 @@ int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, voi
         CUtensorMap tmA, tmB;
         MOE_TRY(map_rows_kmajor(&tmA, dsplit_s, P1, 3 * n2));
         MOE_TRY(map_weight_kmajor(&tmB, wsplit_s, a, d, 3 * n2));
-        MOE_TRY(launch_tile_prefix(offsets_p, a, BM, tile_prefix, st));
+        MOE_TRY(launch_tile_table(offsets_p, a, BM, P1, tile_prefix, st));
         GemmParams p = default_params();
-        p.offsets = offsets_p; p.tile_prefix = tile_prefix; p.nseg = a; p.N = d; p.K = n2; p.R = P1;
+        p.offsets = offsets_p; p.tile_prefix = tile_prefix; p.tile_info = tile_info_of(tile_prefix, a);
+        p.nseg = a; p.N = d; p.K = n2; p.R = P1;
         p.out_f32 = dX_sec; p.status = status;
         p.nterms = 6;
         const int32_t at[6] = {2, 0, 1, 0, 1, 0}, bt[6] = {0, 2, 1, 1, 0, 0};
@@ -1246,8 +1450,8 @@ int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, 
     const int64_t R = (int64_t)c.T * c.k;
     MOE_TRY(launch_segment_colsum(dys, c.act, offsets, c.n, R, c.d, db2, colsum, tile_prefix, st));
     MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st));
-    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st));
-    MOE_TRY(launch_segment_colsum(dz, c.act, offsets, c.n, R, c.h, db1, colsum, tile_prefix, st));
+    // db1 = column sums of dz, formed in the epilogue of the GEMM that produces dz
+    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, colsum, db1));
     MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st));
     return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st);
 }

@@ -197,6 +197,8 @@ int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, voi
                                      const float *Wn_s, const int32_t *offsets_p, int32_t *tile_prefix, int32_t a,
                                      int64_t P1, int32_t d, int32_t b, float *partials, float *dWg_s, float *dWn_s,
                                      float *dX_sec, int32_t *status, cudaStream_t st);
+int64_t tc_tile_ws_ints(int64_t R, int64_t nseg);  // int32s of a [nseg + 1] tile prefix followed by its tile table
+int64_t tc_colsum_part_floats(int64_t R, int32_t nseg, int32_t N);  // scratch of the fused bias-gradient sums
 int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
                           void *dW2, void *db2, void *dz, float *colsum, int32_t *tile_prefix, int32_t *status_word,
