@@ -64,6 +64,7 @@ struct GemmParams {
     // ROW_* with bf16 output: if set, column sums of the stored values over each epilogue warp's 32 rows,
     // [32-row block][N] floats; block = (global M tile * CTAs per tile + CTA rank) * 4 + row quarter
     float *colsum_part;
+    int32_t tma_out;  // two-CTA ROW_*: full 32-row pieces leave through shared memory and bulk tensor stores
     int32_t relu;
     int32_t *status;
     // uniform segments (offsets == nullptr): ROW_*: one segment of R rows. WGRAD: segment s covers
@@ -150,6 +151,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
         "[%2];" ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+
+// bulk tensor store of a [32 rows][64 columns] box from 128-byte-swizzled shared memory
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *tm, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(c0),
+                 "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // 256-bit store (sm_100): a whole 32-byte sector per instruction
 __device__ __forceinline__ void st_global_32B(uint4 *dst, const uint4 &a, const uint4 &b) {
@@ -590,6 +601,13 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_BIT_MASK) : "memory");
 }
+// The same without release semantics, for handing an accumulator buffer back: the tensor-memory reads are
+// complete (tcgen05.wait::ld) and fenced (tcgen05.fence::before_thread_sync) before the arrive, and nothing
+// the other side reads was written through memory. A release at cluster scope would wait here for all of this
+// thread's earlier global stores (the output rows) to reach L2, several thousand cycles per tile.
+__device__ __forceinline__ void mbar_arrive_leader_relaxed(uint32_t bar) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_BIT_MASK) : "memory");
+}
 __device__ __forceinline__ void tc_commit2(uint32_t bar) {  // arrives at this offset in both CTAs of the pair
     asm volatile(
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -635,8 +653,11 @@ __host__ __device__ constexpr uint32_t make_idesc2(int a_mn, int b_mn) {  // M 2
 template <int KIND, bool MASKT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                     const __grid_constant__ CUtensorMap tmM, const GemmParams p) {
-    constexpr int NST = MASKT ? 5 : 6;
+                     const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmO,
+                     const GemmParams p) {
+    // ROW_*: 5 stages and a 64 KiB region of four [128 rows][64 columns] blocks (128-byte swizzle) that holds the
+    // ReLU-mask tile (MASKT) and stages the bf16 output for bulk tensor stores; WGRAD: 6 stages + 32 KiB of staging
+    constexpr int NST = KIND == WGRAD ? 6 : 5;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
@@ -670,6 +691,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
         if (MASKT) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmM) : "memory");
+        if (KIND != WGRAD) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmO) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)),
@@ -691,9 +713,29 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool ok = true;
             TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
             Tile t;
+            // MASKT: the mask tile of a row tile can only land after the epilogue has read the previous one, which
+            // happens while the next tile's K blocks are already being loaded: the load stays "due" and is issued
+            // from the K loop as soon as the region is free, so the producer never stops to wait for the epilogue.
+            bool mask_due = false;
+            int mask_n0 = 0, mask_row0 = 0;
+            auto load_mask = [&](bool blocking) -> bool {
+                if (blocking) {
+                    if (!mbar_wait(mempty_bar, mask_ph ^ 1u, abort_flag, p.status)) return false;
+                } else if (!mbar_try_wait(mempty_bar, mask_ph ^ 1u)) {
+                    return true;
+                }
+                const int nblk = min(4, (p.N - mask_n0) / 64);
+                mbar_expect_tx(mfull_bar, nblk * 16384);
+                for (int b = 0; b < nblk; ++b)
+                    tma_load_2d(mask_smem + b * 16384, &tmM, mfull_bar, mask_n0 + b * 64, mask_row0 + 128 * (int)rank);
+                mask_ph ^= 1u;
+                mask_due = false;
+                return true;
+            };
             while (ok && it.next(t)) {
                 int term = 0, kk = 0;  // ROW_*: piece of the contraction and column inside it
                 for (int kb = 0; kb < t.kblocks && ok; ++kb) {
+                    if (MASKT && mask_due) load_mask(false);
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
                     const uint32_t a_dst = base + s * STAGE2_BYTES, b_dst = a_dst + A2_BYTES;
@@ -720,16 +762,14 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                     if (++s == NST) { s = 0; ph ^= 1u; }
                 }
-                if (MASKT && ok) {  // this tile's mask rows, once the previous tile's have been read
-                    ok = mbar_wait(mempty_bar, mask_ph ^ 1u, abort_flag, p.status);
-                    if (!ok) break;
-                    const int nblk = min(4, (p.N - t.n0) / 64);
-                    mbar_expect_tx(mfull_bar, nblk * 16384);
-                    for (int b = 0; b < nblk; ++b)
-                        tma_load_2d(mask_smem + b * 16384, &tmM, mfull_bar, t.n0 + b * 64, t.row0 + 128 * (int)rank);
-                    mask_ph ^= 1u;
+                if (MASKT && ok) {  // this tile's mask rows are due once the previous tile's have been read
+                    if (mask_due) ok = load_mask(true);  // the previous tile's mask is still due: now it has to go
+                    mask_due = ok;
+                    mask_n0 = t.n0; mask_row0 = t.row0;
+                    if (ok) load_mask(false);
                 }
             }
+            if (MASKT && ok && mask_due) load_mask(true);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
@@ -848,6 +888,15 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (!ok) break;
                 mask_ph ^= 1u;
             }
+            // Whole 32-row pieces go out as bulk tensor stores: each lane writes its row's 64-byte pieces into the
+            // warp's own rows of a [128][64] block (the place the mask values were just read from, for MASKT), and one
+            // lane stores each finished [32][64] box. Ragged pieces (segment end) use the guarded row stores.
+            const bool staged = KIND != WGRAD && p.tma_out && !p.out_f32 && rows_valid >= 32;
+            const int mrow = quarter * 32 + lane;
+            if (staged && !MASKT) {  // the previous tile's boxes must have been read out of shared memory
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+            }
             for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                 const int col0 = t.n0 + c * 32;
                 if (col0 >= p.N) break;
@@ -882,7 +931,6 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
                     }
                     if (MASKT) {  // from the tile in shared memory: row = this thread's row, 16-B pieces swizzled by row
-                        const int mrow = quarter * 32 + lane;
                         const uint8_t *mrow_p = smem + NST * STAGE2_BYTES + (c >> 1) * 16384 + mrow * 128;
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
@@ -906,7 +954,20 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         }
                         ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
                     }
-                    if (row_ok) {
+                    if (staged) {
+                        uint8_t *blk = smem + NST * STAGE2_BYTES + (c >> 1) * 16384;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4 *>(blk + mrow * 128 + ((((c & 1) * 4 + q) ^ (mrow & 7)) << 4)) = packed[q];
+                        if (c & 1) {  // the box of 64 columns is complete
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&tmO, smem_u32(blk + quarter * 4096), t.n0 + (c >> 1) * 64, (int)tile_row0);
+                                tma_store_commit();
+                            }
+                        }
+                    } else if (row_ok) {
                         uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
                         st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
                         st_global_32B(dst + 2, packed[2], packed[3]);
@@ -924,17 +985,21 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                 }
             }
-            if (MASKT) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(mempty_bar);
-            }
             if (have_acc) {
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_leader(tempty_bar(acc));
+                if (lane == 0) mbar_arrive_leader_relaxed(tempty_bar(acc));
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
+            if (MASKT) {  // the next mask tile may land once this warp's boxes have been read out
+                __syncwarp();
+                if (lane == 0) {
+                    if (staged) tma_store_wait_read();
+                    mbar_arrive(mempty_bar);
+                }
+            }
         }
+        if (KIND != WGRAD && lane == 0) tma_store_wait_all();  // no bulk store may outlive the CTA's shared memory
     }
 
     tc_fence_before();
@@ -1068,8 +1133,9 @@ template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tm
 
 template <int KIND, bool MASKT = false>
 int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p_in, int64_t max_tiles,
-                cudaStream_t st, const CUtensorMap *tmM = nullptr) {
+                cudaStream_t st, const CUtensorMap *tmM = nullptr, const CUtensorMap *tmO = nullptr) {
     GemmParams p = p_in;
+    p.tma_out = tmO != nullptr;
     MOE_TRY((complete_params<KIND, 256>(p, max_tiles)));
     static int max_clusters = 0;
     cudaLaunchConfig_t cfg;
@@ -1088,7 +1154,7 @@ int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams
     }
     if (max_tiles <= 0) return MOE_OK;
     cfg.gridDim = dim3(2 * (unsigned)imin(max_tiles, max_clusters));
-    MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND, MASKT>, tmA, tmB, tmM ? *tmM : tmA, p));
+    MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND, MASKT>, tmA, tmB, tmM ? *tmM : tmA, tmO ? *tmO : tmA, p));
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -1238,12 +1304,20 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
         else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
         MOE_TRY(launch_tile_table(offsets, nseg, 256, R, tile_prefix, st));
         const int64_t max_tiles2 = (cdiv(R, 256) + nseg) * cdiv(N, BN);
+        CUtensorMap tmO;  // output rows as [32][64] boxes
+        {
+            const uint64_t dims[2] = {(uint64_t)N, (uint64_t)R};
+            const uint64_t str[1] = {(uint64_t)N * 2};
+            const uint32_t box[2] = {64, 32};
+            MOE_TRY(make_map(&tmO, out, 2, dims, str, box));
+        }
         if (transposed && mask) {  // the ReLU-mask rows come in as TMA tiles
             CUtensorMap tmM;
             MOE_TRY(map_rows_kmajor(&tmM, mask, R, N));
-            return finish(launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM), 8);
+            return finish(launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM, &tmO), 8);
         }
-        return finish(transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st) : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st), 8);
+        return finish(transposed ? launch2<ROW_BK>(tmA, tmB, p, max_tiles2, st, nullptr, &tmO)
+                                 : launch2<ROW_BMN>(tmA, tmB, p, max_tiles2, st, nullptr, &tmO), 8);
     }
     if (transposed) MOE_TRY(map_weight_kmajor(&tmB, W, nseg, N, K));
     else MOE_TRY(map_weight_mnmajor(&tmB, W, nseg, K, N));
