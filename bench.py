@@ -34,6 +34,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 L2_BYTES = 126 * 2 ** 20
 # FP32 FMA peak of a B200 at its maximum SM clock: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+# dram__bytes_read.sum + dram__bytes_write.sum of the six expert GEMMs of one step, from one ncu capture of the bench
+# command (the summary under profiles/ names it); workloads without a capture report null
+NCU_TRAFFIC_BYTES_PER_STEP = {"c5-wide-zipf-128": 31.32e9}  # profiles/grouped_gemm_c5_full_dram_traffic.txt
 
 
 def load_peaks():
@@ -329,19 +332,30 @@ def run_ours(args, w):
     value_e2e = replicas.job_throughput(w.T, args.steps, total_e2e, world)
 
     stages = stage_timings(B, cfg, S, D, w, timed, max(3, min(args.steps, 10)), peaks)
+    # Roofline of the dominant kernel family, the expert grouped GEMMs (six launches per step). They are bound by the
+    # tensor cores when the segments are long and by HBM when there are so many experts that every weight is read
+    # for a handful of rows (c4): both fractions are computed from the algorithmic flop / bytes, the larger one binds.
+    esz = 2 if w.act == "bf16" else 4
     gemm_flop = 12.0 * w.R * w.d * w.h
+    gemm_bytes = (6 * w.R * w.d + 5 * w.R * w.h) * esz + 6 * w.n * w.d * w.h * esz
     gemm_ms = stages["expert_ffn"]["ms"] + stages["expert_ffn_bwd"]["ms"]
     achieved = gemm_flop / (gemm_ms / 1e3) / 1e12
-    if w.act == "bf16":
-        roof = {"bound": "tensor", "kernel": "expert grouped GEMMs (moe_expert_ffn + moe_expert_ffn_bwd)",
-                "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
-                "peak_kind": f"{peak_kind} sustained bf16 (kernels timed back to back inside a long loop)",
-                "frac_of_nominal_2250": achieved / 2250.0}
-    else:
+    achieved_gbs = gemm_bytes / (gemm_ms / 1e3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES_PER_STEP.get(workload_config(w)["workload"])
+    kernel = "expert grouped GEMMs (moe_expert_ffn + moe_expert_ffn_bwd, 6 launches; achieved = per-step flop or bytes / per-step time)"
+    if w.act != "bf16":
         roof = {"bound": "alu", "kernel": "expert grouped GEMMs, fp32 SIMT", "achieved": achieved,
                 "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
                 "peak_kind": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"}
+    elif achieved_gbs / peaks["hbm_gbs"] > achieved / peaks["bf16_tflops_sustained"]:
+        roof = {"bound": "hbm", "kernel": kernel, "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": traffic,
+                "peak_kind": f"{peak_kind} copy bandwidth", "tensor_tflops": achieved}
+    else:
+        roof = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": traffic,
+                "peak_kind": f"{peak_kind} sustained bf16 (kernels timed back to back inside a long loop)",
+                "frac_of_nominal_2250": achieved / 2250.0, "algorithmic_bytes": gemm_bytes}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
