@@ -92,21 +92,25 @@ struct GateWs {
     int32_t *idx_p, *idx_s, *perm_p, *inv_perm_p, *counts_p, *offsets_p, *scratch, *tile_prefix;
     // tensor-core routing screen (flat layer, or the primary level of the hierarchical one)
     bool screen;
-    float *cr, *wnorm, *xnorm;
+    float *cr, *wnorm, *xnorm, *wt;
     void *wsplit;
-    int32_t *unsafe_list, *unsafe_count;
+    int32_t *unsafe_list, *unsafe_count, *full_list;
+    void *chain_list;
     GateWs(Carver &cv, const Dims &D) {
         idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
-        cr = wnorm = xnorm = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = nullptr;
+        cr = wnorm = xnorm = wt = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = full_list = nullptr; chain_list = nullptr;
         const int64_t n1 = D.hier ? D.a : D.n;  // width of the (first) gate
         screen = tc_gate_fwd_supported(D.act, D.T, (int32_t)D.d, (int32_t)n1);
         if (screen) {
             cr = cv.take<float>(D.T * 2 * n1);
             wsplit = cv.take<bf16>(3 * D.d * 2 * n1);
             wnorm = cv.take<float>(2 * n1);
+            wt = cv.take<float>(2 * n1 * D.d);
             xnorm = cv.take<float>(D.T);
             unsafe_list = cv.take<int32_t>(D.T);
             unsafe_count = cv.take<int32_t>(64);
+            full_list = cv.take<int32_t>(D.T);
+            chain_list = cv.take_bytes(D.T * 2 * SCREEN_MAX_CAND * 8);
         }
         if (!D.hier) return;
         idx_p = cv.take<int32_t>(D.T * D.k1);
@@ -289,12 +293,16 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
     auto first_gate = [&](int32_t n1, int32_t k1, int32_t *idx_out, float *gates_out) -> int32_t {
         if (w.screen) {
             MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, w.wsplit, w.wnorm, w.xnorm,
-                                               w.unsafe_count, st));
+                                               w.unsafe_count, w.wt, st));
             MOE_TRY(launch_tc_gate_fwd(x, D.T, (int32_t)D.d, n1, w.wsplit, w.cr, status_word(ws_base), st));
             MOE_TRY(launch_gate_screen(w.cr, noise, w.xnorm, w.wnorm, (int32_t)D.d, D.T, n1, k1, idx_out, gates_out,
-                                       clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_count, st));
+                                       clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_count, w.chain_list,
+                                       w.full_list, st));
+            // exact chains for the few columns that decide an uncertain row; whole rows only where there are many
+            MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, n1, w.wt, w.chain_list, w.unsafe_count + 1, clean, raw_noise,
+                                       st));
             MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, clean, raw_noise, nullptr, 0,
-                                      w.unsafe_list, 1, nullptr, st, w.unsafe_count));
+                                      w.full_list, 1, nullptr, st, w.unsafe_count + 2));
             return launch_gate_select(clean, raw_noise, noise, D.T, n1, k1, idx_out, gates_out, kth_vals, kth_idx, st,
                                       w.unsafe_list, w.unsafe_count);
         }

@@ -202,8 +202,7 @@ int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int3
 // over the list heads then produce the global order. Lowest index wins ties everywhere.
 // softplus is evaluated in double and rounded once, H by one fused multiply-add.
 // ------------------------------------------------------------------------------------------
-constexpr int KL = MOE_MAX_K + 1;
-
+template <int KL>  // length of the per-lane sorted lists, >= k + 1
 __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restrict__ clean,
                                                           const float *__restrict__ raw,
                                                           const float *__restrict__ noise, int64_t rows, int32_t n,
@@ -285,8 +284,13 @@ int32_t launch_gate_select(const float *clean, const float *raw, const float *no
                            int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
                            cudaStream_t st, const int32_t *row_list, const int32_t *row_count) {
     if (rows == 0) return MOE_OK;
-    gate_select_kernel<<<(unsigned)cdiv(rows, 8), 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates,
-                                                                  kth_vals, kth_idx, row_list, row_count);
+    const unsigned grid = (unsigned)cdiv(rows, 8);
+#define MOE_SELECT(KL) \
+    gate_select_kernel<KL><<<grid, 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates, kth_vals, kth_idx, row_list, row_count)
+    if (k <= 2) MOE_SELECT(3);
+    else if (k <= 4) MOE_SELECT(5);
+    else MOE_SELECT(MOE_MAX_K + 1);
+#undef MOE_SELECT
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -346,9 +350,9 @@ __global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x
     if (lane == 0) xnorm[t] = sqrtf(s) * (1.0f + 1e-5f);
 }
 
-constexpr int KL2 = MOE_MAX_K + 2;
-
-template <int NV>  // columns per lane (n <= 32 * NV); 0: any n, plain loop
+// NV: columns per lane (n <= 32 * NV), 0: any n, plain loop. KL: length of the per-lane sorted lists, >= k + 2
+// (short lists for small k: the insertion into them is most of this kernel's instructions)
+template <int NV, int KL>
 __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
                                                           const float *__restrict__ xnorm,
                                                           const float *__restrict__ wnorm, float theta, int64_t T,
@@ -357,33 +361,39 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
                                                           float *__restrict__ raw, float *__restrict__ kth_vals,
                                                           int32_t *__restrict__ kth_idx,
                                                           int32_t *__restrict__ unsafe_list,
-                                                          int32_t *__restrict__ unsafe_count) {
+                                                          int32_t *__restrict__ unsafe_count,
+                                                          int2 *__restrict__ chain_list,
+                                                          int32_t *__restrict__ full_list) {
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= T) return;
     // per-lane sorted list of (value, index, uncertainty); rest_hi = largest possible chain value of anything
     // that is not in a list
-    float lv[KL2], lu[KL2];
-    int32_t li[KL2];
+    float lv[KL], lu[KL];
+    int32_t li[KL];
 #pragma unroll
-    for (int s = 0; s < KL2; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
+    for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
     const float *c = cr + row * 2 * n, *r = c + n, *e = noise + row * n;
     const float xn = theta * xnorm[row];
     float rest_hi = -CUDART_INF_F;
+    // approximate noisy logit v of column j and a bound u on its distance from the fma chain's value
+    auto eval = [&](int32_t j, float cj, float rj, float ej, float &v, float &u) {
+        // single-precision softplus is enough for screening: its few ulp go into the uncertainty
+        const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
+        v = fmaf(ej, sigma, cj);
+        // |H~_j - H_j|: projection errors through c and through softplus(r) (slope <= 1) times |noise|, plus the
+        // rounding of softplus (here single, there double rounded once) and of the final fma on both sides
+        u = xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]) + 1.1920929e-7f * (8.0f * fabsf(v) + 16.0f * fabsf(ej) * sigma);
+    };
     auto consider = [&](int32_t j, float cj, float rj, float ej) {
         clean[row * n + j] = cj;
         raw[row * n + j] = rj;
-        // single-precision softplus is enough for screening: its few ulp go into the uncertainty
-        const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
-        float v = fmaf(ej, sigma, cj);
-        // |H~_j - H_j|: projection errors through c and through softplus(r) (slope <= 1) times |noise|, plus the
-        // rounding of softplus (here single, there double rounded once) and of the final fma on both sides
-        float u = xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]) +
-                  1.1920929e-7f * (8.0f * fabsf(v) + 16.0f * fabsf(ej) * sigma);
+        float v, u;
+        eval(j, cj, rj, ej, v, u);
         int32_t id = j;
         bool shifting = false;
 #pragma unroll
-        for (int s = 0; s < KL2; ++s) {
+        for (int s = 0; s < KL; ++s) {
             if (shifting || v > lv[s]) {
                 float tv = lv[s], tu = lu[s]; int32_t ti = li[s];
                 lv[s] = v; li[s] = id; lu[s] = u; v = tv; id = ti; u = tu;
@@ -407,13 +417,13 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
         for (int32_t j = lane; j < n; j += 32) consider(j, c[j], r[j], e[j]);
     }
     const int rounds = min(k + 2, n);
-    float hvv[KL2], huu[KL2];
+    float hvv[KL], huu[KL];
     float myv = -CUDART_INF_F;
     int32_t myi = -1;
     float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
     int32_t i_k = -1, i_k1 = -1;
 #pragma unroll
-    for (int s = 0; s < KL2; ++s) {
+    for (int s = 0; s < KL; ++s) {
         hvv[s] = -CUDART_INF_F; huu[s] = 0.0f;
         if (s < rounds) {
             float hv = lv[0], hu = lu[0];
@@ -426,9 +436,9 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
             }
             if (li[0] == hi) {
 #pragma unroll
-                for (int q = 0; q < KL2 - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; lu[q] = lu[q + 1]; }
-                lv[KL2 - 1] = -CUDART_INF_F;
-                li[KL2 - 1] = INT32_MAX;
+                for (int q = 0; q < KL - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; lu[q] = lu[q + 1]; }
+                lv[KL - 1] = -CUDART_INF_F;
+                li[KL - 1] = INT32_MAX;
             }
             hvv[s] = hv; huu[s] = hu;
             if (s < k && lane == s) { myv = hv; myi = hi; }
@@ -438,7 +448,7 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
     }
     // whatever is still in the lists is "rest" as well
 #pragma unroll
-    for (int s = 0; s < KL2; ++s)
+    for (int s = 0; s < KL; ++s)
         if (li[s] != INT32_MAX) rest_hi = fmaxf(rest_hi, lv[s] + lu[s]);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) rest_hi = fmaxf(rest_hi, __shfl_xor_sync(0xffffffffu, rest_hi, off));
@@ -447,14 +457,86 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
     bool safe = true;
     float suffix = rest_hi;
 #pragma unroll
-    for (int s = KL2 - 1; s >= 0; --s) {
+    for (int s = KL - 1; s >= 0; --s) {
         if (s < rounds) {
             if (s <= k && !(hvv[s] - huu[s] > suffix)) safe = false;
             suffix = fmaxf(suffix, hvv[s] + huu[s]);
         }
     }
-    if (!safe) {  // not provably the chain's routing: redo this token with the fma chain
-        if (lane == 0) unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
+    if (!safe) {
+        // Not provably the chain's routing. Only the columns that can still reach rank k+1 matter: those whose
+        // highest possible value is at least `low`, a lower bound of the (k+1)-th largest chain value (the (k+1)-th
+        // largest lower end among the extracted columns). They get their two fma chains redone (chain_list), the
+        // selection is then repeated on the patched row. Rows with too many candidates (ties) take the full chain.
+        float low = -CUDART_INF_F;
+        if (k < rounds) {
+#pragma unroll
+            for (int s = 0; s < KL; ++s) {
+                if (s < rounds) {
+                    const float ls = hvv[s] - huu[s];
+                    int above = 0;
+#pragma unroll
+                    for (int s2 = 0; s2 < KL; ++s2)
+                        if (s2 < rounds && s2 != s) {
+                            const float l2 = hvv[s2] - huu[s2];
+                            above += (l2 > ls || (l2 == ls && s2 < s)) ? 1 : 0;
+                        }
+                    if (above == k) low = ls;
+                }
+            }
+        }
+        // (the row is re-read and re-evaluated here: keeping every column's value in registers through the
+        // selection above would cost the certified rows, the common case, their occupancy)
+        int total = 0;
+        uint32_t mine = 0;  // NV > 0: bit q = this lane's column lane + 32 q is a candidate
+        if (NV > 0) {
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                const int32_t j = lane + 32 * q;
+                float v = -CUDART_INF_F, u = 0.0f;
+                if (j < n) eval(j, c[j], r[j], e[j], v, u);
+                const bool cand = j < n && v + u >= low;
+                if (cand) mine |= 1u << q;
+                total += __popc(__ballot_sync(0xffffffffu, cand));
+            }
+        } else {
+            for (int32_t j0 = 0; j0 < n; j0 += 32) {
+                const int32_t j = j0 + lane;
+                float v = -CUDART_INF_F, u = 0.0f;
+                if (j < n) eval(j, c[j], r[j], e[j], v, u);
+                total += __popc(__ballot_sync(0xffffffffu, j < n && v + u >= low));
+            }
+        }
+        int32_t base = 0;
+        const bool few = total <= SCREEN_MAX_CAND;
+        if (lane == 0) {
+            unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
+            if (few) base = atomicAdd(unsafe_count + 1, 2 * total);
+            else full_list[atomicAdd(unsafe_count + 2, 1)] = (int32_t)row;
+        }
+        if (!few) return;
+        base = __shfl_sync(0xffffffffu, base, 0);
+        int pos = 0;
+        auto emit = [&](int32_t j, bool cand) {
+            const uint32_t b = __ballot_sync(0xffffffffu, cand);
+            if (cand) {
+                const int at = base + 2 * (pos + __popc(b & ((1u << lane) - 1u)));
+                chain_list[at] = make_int2((int32_t)row, j);
+                chain_list[at + 1] = make_int2((int32_t)row, n + j);
+            }
+            pos += __popc(b);
+        };
+        if (NV > 0) {
+#pragma unroll
+            for (int q = 0; q < NV; ++q) emit(lane + 32 * q, (mine >> q) & 1u);
+        } else {
+            for (int32_t j0 = 0; j0 < n; j0 += 32) {
+                const int32_t j = j0 + lane;
+                float v = -CUDART_INF_F, u = 0.0f;
+                if (j < n) eval(j, c[j], r[j], e[j], v, u);
+                emit(j, j < n && v + u >= low);
+            }
+        }
         return;
     }
     const float m = __shfl_sync(0xffffffffu, myv, 0);
@@ -473,9 +555,123 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
     }
 }
 
+// One fma chain per thread: entry (row, c) of chain_list recomputes clean[row, c] (c < n) or raw[row, c - n] exactly
+// as the projection kernel does: fp32, from +0, ascending input feature. Wt [2n, d] holds the columns of
+// [W_g | W_noise] as rows. The 32 chains of a warp read 32 different weight rows; a load instruction that touches 32
+// lines costs the load/store unit 32 tag look-ups, which is what bounds this kernel, so the warp fetches the next 32
+// features of its 32 rows cooperatively (eight lanes per 128-byte line, four lines per instruction), parks them in
+// shared memory and every lane then reads its own row back. Loads for step s + 1 are in flight during the 32
+// dependent fused multiply-adds of step s.
+constexpr int CHAIN_PITCH = 144;  // bytes per staged row: 128 + 16, conflict-free both ways
+template <typename XT>
+__global__ void __launch_bounds__(128) gate_chain_kernel(const XT *__restrict__ x, int32_t d, int32_t n,
+                                                         const float *__restrict__ Wt,
+                                                         const int2 *__restrict__ chain_list,
+                                                         const int32_t *__restrict__ chain_count,
+                                                         float *__restrict__ clean, float *__restrict__ raw) {
+    __shared__ __align__(16) uint8_t stage[4][2][32 * CHAIN_PITCH];
+    const int32_t total = *chain_count;
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int32_t steps = d / 32;  // d is a multiple of 64 on this path
+    for (int32_t i0 = (blockIdx.x * 4 + wp) * 32; i0 < total; i0 += gridDim.x * 128) {  // warp-uniform
+        const int32_t i = i0 + lane;
+        const int2 en = chain_list[i < total ? i : total - 1];  // idle lanes shadow the last chain
+        const XT *xr = x + (int64_t)en.x * d;
+        const float *wrow = Wt + (int64_t)en.y * d;
+        // instruction u of a step loads 16 bytes of the row of lane 4 u + lane / 8, at byte (lane % 8) * 16
+        const float *src[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const unsigned long long ptr = __shfl_sync(0xffffffffu, (unsigned long long)wrow, 4 * u + (lane >> 3));
+            src[u] = reinterpret_cast<const float *>(ptr) + (lane & 7) * 4;
+        }
+        float4 wreg[8];
+        uint4 xreg[4];
+        auto fetch = [&](int32_t st) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) wreg[u] = *reinterpret_cast<const float4 *>(src[u] + st * 32);
+            if constexpr (sizeof(XT) == 2) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) xreg[g] = *reinterpret_cast<const uint4 *>(xr + st * 32 + 8 * g);
+            }
+        };
+        auto park = [&](int b) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                *reinterpret_cast<float4 *>(&stage[wp][b][(4 * u + (lane >> 3)) * CHAIN_PITCH + (lane & 7) * 16]) = wreg[u];
+        };
+        float acc = 0.0f;
+        fetch(0);
+        __syncwarp();  // the previous chains' last reads of the staging rows are done
+        park(0);
+        uint4 xcur[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) xcur[g] = xreg[g];
+        __syncwarp();
+        for (int32_t st = 0; st < steps; ++st) {
+            if (st + 1 < steps) fetch(st + 1);
+            const uint8_t *mine = &stage[wp][st & 1][lane * CHAIN_PITCH];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const float4 wv = *reinterpret_cast<const float4 *>(mine + 16 * u);
+                float x0, x1, x2, x3;
+                if constexpr (sizeof(XT) == 2) {
+                    const bf16 *hx = reinterpret_cast<const bf16 *>(&xcur[u >> 1]) + 4 * (u & 1);
+                    x0 = __bfloat162float(hx[0]); x1 = __bfloat162float(hx[1]);
+                    x2 = __bfloat162float(hx[2]); x3 = __bfloat162float(hx[3]);
+                } else {
+                    const int32_t q = st * 32 + 4 * u;
+                    x0 = to_f32(xr[q]); x1 = to_f32(xr[q + 1]); x2 = to_f32(xr[q + 2]); x3 = to_f32(xr[q + 3]);
+                }
+                acc = fmaf(x0, wv.x, acc); acc = fmaf(x1, wv.y, acc);
+                acc = fmaf(x2, wv.z, acc); acc = fmaf(x3, wv.w, acc);
+            }
+            if (st + 1 < steps) {
+                park((st + 1) & 1);  // the other buffer: its readers finished a step ago (syncwarp below)
+#pragma unroll
+                for (int g = 0; g < 4; ++g) xcur[g] = xreg[g];
+            }
+            __syncwarp();
+        }
+        if (i < total) {
+            if (en.y >= n) raw[(int64_t)en.x * n + (en.y - n)] = acc;
+            else clean[(int64_t)en.x * n + en.y] = acc;
+        }
+    }
+}
+
+// Wt[c, q] = [W_g | W_noise][q, c]
+__global__ void __launch_bounds__(256) gate_transpose_weights_kernel(const float *__restrict__ Wg, const float *__restrict__ Wn,
+                                                                     int32_t d, int32_t n, float *__restrict__ Wt) {
+    __shared__ float tile[32][33];
+    const int q0 = blockIdx.x * 32, c0 = blockIdx.y * 32;  // 2n and d are multiples of 32 on this path
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + tx, q = q0 + i;
+        tile[i][tx] = c < n ? Wg[(int64_t)q * n + c] : Wn[(int64_t)q * n + (c - n)];
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) Wt[(int64_t)(c0 + i) * d + q0 + tx] = tile[tx][i];
+}
+
+int32_t launch_gate_chains(const void *x, int32_t act, int32_t d, int32_t n, const float *Wt, const void *chain_list,
+                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st) {
+    const unsigned grid = 148 * 16;
+    if (act == MOE_BF16)
+        gate_chain_kernel<bf16><<<grid, 128, 0, st>>>((const bf16 *)x, d, n, Wt, (const int2 *)chain_list, chain_count, clean,
+                                                      raw);
+    else
+        gate_chain_kernel<float><<<grid, 128, 0, st>>>((const float *)x, d, n, Wt, (const int2 *)chain_list, chain_count, clean,
+                                                       raw);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
 int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
                                    const float *Wn, void *wsplit, float *wnorm, float *xnorm,
-                                   int32_t *unsafe_count, cudaStream_t st) {
+                                   int32_t *unsafe_count, float *wt, cudaStream_t st) {
+    gate_transpose_weights_kernel<<<dim3((unsigned)(d / 32), (unsigned)(2 * n / 32)), 256, 0, st>>>(Wg, Wn, d, n, wt);
+    MOE_LAUNCHED();
     split_gate_weights_kernel<<<(unsigned)cdiv((int64_t)d * 2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
     MOE_LAUNCHED();
     gate_col_norms_kernel<<<(unsigned)cdiv(2 * n, 8), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
@@ -483,14 +679,14 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
     if (act == MOE_BF16) row_norms_kernel<bf16><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const bf16 *)x, T, d, xnorm);
     else row_norms_kernel<float><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const float *)x, T, d, xnorm);
     MOE_LAUNCHED();
-    MOE_CUDA(cudaMemsetAsync(unsafe_count, 0, sizeof(int32_t), st));
+    MOE_CUDA(cudaMemsetAsync(unsafe_count, 0, 4 * sizeof(int32_t), st));  // rows to re-select, chains, full-chain rows
     return MOE_OK;
 }
 
 int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
-                           cudaStream_t st) {
+                           void *chain_list, int32_t *full_list, cudaStream_t st) {
     // worst-case rounding of the fma chain, plus two truncations of an fp32 accumulator per MMA step of the
     // three-term tensor-core product (3d/16 steps and the additions inside a step), plus the split residual
     const double u = ldexp(1.0, -24);
@@ -498,15 +694,23 @@ int32_t launch_gate_screen(const float *cr, const float *noise, const float *xno
     const double tc = 2.0 * (3.0 * d / 16.0 + 8.0) * ldexp(1.0, -23) + ldexp(1.0, -22);
     const float theta = (float)((chain + tc) * 1.01);
     const unsigned grid = (unsigned)cdiv(T, 8);
-#define MOE_SCREEN(NV)                                                                                              \
-    gate_screen_kernel<NV><<<grid, 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean, raw, \
-                                                 kth_vals, kth_idx, unsafe_list, unsafe_count)
+#define MOE_SCREEN_KL(NV, KL)                                                                                            \
+    gate_screen_kernel<NV, KL><<<grid, 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean, raw,  \
+                                                     kth_vals, kth_idx, unsafe_list, unsafe_count, (int2 *)chain_list, \
+                                                     full_list)
+#define MOE_SCREEN(NV)                                \
+    do {                                              \
+        if (k <= 2) MOE_SCREEN_KL(NV, 4);             \
+        else if (k <= 4) MOE_SCREEN_KL(NV, 6);        \
+        else MOE_SCREEN_KL(NV, MOE_MAX_K + 2);        \
+    } while (0)
     if (n <= 32) MOE_SCREEN(1);
     else if (n <= 64) MOE_SCREEN(2);
     else if (n <= 128) MOE_SCREEN(4);
     else if (n <= 256) MOE_SCREEN(8);
     else MOE_SCREEN(0);
 #undef MOE_SCREEN
+#undef MOE_SCREEN_KL
     MOE_LAUNCHED();
     return MOE_OK;
 }

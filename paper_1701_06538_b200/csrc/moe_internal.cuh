@@ -75,11 +75,17 @@ int32_t launch_gate_select(const float *clean, const float *raw, const float *no
 // Tensor-core screening of the routing (see gate.cu): weights split / norms, then the screening select.
 int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
                                    const float *Wn, void *wsplit, float *wnorm, float *xnorm,
-                                   int32_t *unsafe_count, cudaStream_t st);
+                                   int32_t *unsafe_count, float *wt /* [2n, d]: columns as rows */, cudaStream_t st);
 int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
-                           cudaStream_t st);
+                           void *chain_list, int32_t *full_list, cudaStream_t st);
+// Rows the screen cannot certify: unsafe_list / unsafe_count[0] = rows whose selection is repeated; chain_list
+// (int2 {row, column code}, unsafe_count[1] entries, at most 2 * SCREEN_MAX_CAND per row) = single fma chains to
+// recompute; full_list / unsafe_count[2] = rows with more candidates than that, which take the whole projection.
+constexpr int SCREEN_MAX_CAND = 16;
+int32_t launch_gate_chains(const void *x, int32_t act, int32_t d, int32_t n, const float *Wt, const void *chain_list,
+                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st);  // Wt [2n, d]
 bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n);
 // cr [T, 2n] (float) = x . [W_g | W_noise] from the three-term split wsplit [3, d, 2n]
 int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,
