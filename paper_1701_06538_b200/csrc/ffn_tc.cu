@@ -73,6 +73,8 @@ struct GemmParams {
     int64_t R;
     int32_t rows_per_seg, segs_per_term, b_term_chunks;
     int32_t segs_term0, rows_per_seg0;  // if segs_term0 > 0: term 0 is cut into that many ranges of rows_per_seg0
+    int32_t interleave;                 // uniform WGRAD: number of terms whose tiles alternate in the id order (0: none)
+    int32_t sub_kb0, sub_kb;            // ACC kernel: K blocks per separately accumulated sub-block, term 0 / other terms
     int32_t off_mod;                    // WGRAD with offsets: see tile_fetch
     // ROW_*: the contraction is the concatenation of nterms pieces of length K; piece i reads A
     // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
@@ -260,7 +262,11 @@ template <int KIND, int TM>
 __device__ __forceinline__ bool tile_decode(const GemmParams &p, int32_t id, const int4 &raw, Tile &t) {
     if (id >= p.total_tiles) return false;
     if (KIND == WGRAD) {
-        const int32_t e = id / p.per_e, rem = id - e * p.per_e;
+        int32_t e = id / p.per_e;
+        const int32_t rem = id - e * p.per_e;
+        // uniform ranges, interleaved terms: consecutive ids walk the terms of one row range (its rows stay in L2 for all
+        // of them) while the segment index stays term-major
+        if (p.interleave > 1) e = (e % p.interleave) * p.segs_per_term + e / p.interleave;
         const int32_t tm = rem / p.tiles_n;
         t.e = e;
         t.mt = 0;
@@ -324,25 +330,32 @@ template <int KIND, int TM> struct TileIter {
     }
 };
 
-template <int KIND>
+// ACC (WGRAD with float output over long uniform row ranges, the gate backward): the contraction of a tile is cut
+// into sub-blocks of p.sub_kb0 / p.sub_kb K blocks (first term / other terms). Each sub-block is accumulated in TMEM on
+// its own (an fp32 tensor-core accumulator truncates, and a long run of same-sign terms loses low bits: 128 rows keep
+// that below 1e-5), handed to the epilogue like a tile, and added there, with rounding to nearest, to running sums in
+// shared memory (32 rows x 128 columns of floats per warp, 16-byte units swizzled by row); the sums go to global memory
+// once per tile. Two stages of operands make room for the 128 KiB of sums.
+template <int KIND, bool ACC = false>
 __global__ void __launch_bounds__(NTHREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-B aligned for the 128-B swizzle
     uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bars = base + STAGES * STAGE_BYTES;
+    constexpr int NST = ACC ? 2 : STAGES;
+    const uint32_t bars = base + NST * STAGE_BYTES;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-    auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4) + 8);
+    auto empty_bar = [&](int s) { return bars + 8u * (NST + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * NST + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * NST + 2 + a); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + NST * STAGE_BYTES + 8 * (2 * NST + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + NST * STAGE_BYTES + 8 * (2 * NST + 4) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < NST; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -386,12 +399,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         kk += BK;
                         if (kk == p.K) { kk = 0; ++term; }
                     }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (++s == NST) { s = 0; ph ^= 1u; }
                 }
             }
             // drain: every copy this thread started must have landed before the CTA may exit
             if (!ok)
-                for (int q = 0; q < STAGES; ++q) {
+                for (int q = 0; q < NST; ++q) {
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(full_bar(q), 0) && !mbar_try_wait(full_bar(q), 1) &&
                            global_ns() - t0 < WAIT_LIMIT_NS) {}
@@ -407,11 +420,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         Tile t;
         while (ok && it.next(t)) {
             if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
-            ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * BN;
+            const int sub = ACC ? (t.e < p.segs_term0 ? p.sub_kb0 : p.sub_kb) : t.kblocks;  // K blocks per accumulator
+            uint32_t d_tmem = tmem_base + acc * BN;
             for (int kb = 0; kb < t.kblocks; ++kb) {
+                const int kin = ACC ? kb % sub : kb;  // K block inside the accumulator's sub-block
+                if (kin == 0) {
+                    ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    d_tmem = tmem_base + acc * BN;
+                }
                 ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
@@ -439,16 +457,23 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         else ad = desc_kmajor(a_src + k * 32);
                         if (KIND == ROW_BK) bd = desc_kmajor(b_src + k * 32);
                         else bd = desc_mnmajor(b_src + k * 16 * 128);
-                        tc_mma_bf16(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_bf16(d_tmem, ad, bd, idesc, (kin > 0 || k > 0) ? 1u : 0u);
                     }
                     tc_commit(empty_bar(s));  // the stage may be refilled once these MMAs have read it
                 }
                 __syncwarp();
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (++s == NST) { s = 0; ph ^= 1u; }
+                if (ACC && (kin == sub - 1 || kb == t.kblocks - 1)) {  // sub-block complete
+                    if (lane == 0) tc_commit(tfull_bar(acc));
+                    __syncwarp();
+                    if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+                }
             }
-            if (ok && lane == 0) tc_commit(tfull_bar(acc));  // accumulator complete
-            __syncwarp();
-            if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            if (!ACC) {
+                if (ok && lane == 0) tc_commit(tfull_bar(acc));  // accumulator complete
+                __syncwarp();
+                if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
@@ -460,6 +485,52 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         Tile t;
         while (ok && it.next(t)) {
             const bool have_acc = t.kblocks > 0;
+            if (ACC) {
+                const int half_a = (warp - 2) >> 2;
+                uint8_t *sums = smem + NST * STAGE_BYTES + 256 + (warp - 2) * 16384;  // [32 rows][32 x 16 B], unit ^ row
+                const int sub = t.e < p.segs_term0 ? p.sub_kb0 : p.sub_kb;
+                const int nsub = (t.kblocks + sub - 1) / sub;
+                for (int sb = 0; sb < nsub && ok; ++sb) {
+                    ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int cl = 0; cl < 4; ++cl) {
+                        uint32_t v[32];
+                        tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + (half_a * 4 + cl) * 32, v);
+                        tc_ld_wait();
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            float4 *cell = reinterpret_cast<float4 *>(sums + lane * 512 + ((((cl * 8 + q) ^ lane) & 31) << 4));
+                            float4 a = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                   __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                            if (sb > 0) {
+                                const float4 o = *cell;
+                                a.x += o.x; a.y += o.y; a.z += o.z; a.w += o.w;
+                            }
+                            *cell = a;
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));
+                    if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+                }
+                if (!ok) break;
+                // the warp's 32 x 128 sums to global memory, one 512-byte row segment per instruction
+                const int64_t row0 = (int64_t)t.m0 + quarter * 32;
+                float *dst = p.out_f32 + (int64_t)t.e * p.M * p.N + row0 * p.N + t.n0 + half_a * 128 + lane * 4;
+                if (t.n0 + half_a * 128 + lane * 4 < p.N) {
+                    for (int i = 0; i < 32; ++i) {
+                        if (row0 + i >= p.M) break;
+                        float4 val = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        if (nsub > 0) val = *reinterpret_cast<const float4 *>(sums + i * 512 + (((lane ^ i) & 31) << 4));
+                        *reinterpret_cast<float4 *>(dst + (int64_t)i * p.N) = val;
+                    }
+                }
+                __syncwarp();  // the sums are read before the next tile overwrites them
+                continue;
+            }
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
                 if (!ok) break;
@@ -1131,6 +1202,24 @@ template <int KIND> int32_t launch(const CUtensorMap &tmA, const CUtensorMap &tm
     return MOE_OK;
 }
 
+// The sub-block accumulating wgrad (float output): two operand stages + 128 KiB of running sums
+constexpr int SMEM_ACC_BYTES = 2 * STAGE_BYTES + 1024 + 256 + 8 * 16384;
+int32_t launch_acc_wgrad(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p_in, int64_t max_tiles,
+                         cudaStream_t st) {
+    GemmParams p = p_in;
+    MOE_TRY((complete_params<WGRAD, BM>(p, max_tiles)));
+    static bool configured = false;
+    if (!configured) {
+        MOE_CUDA(cudaFuncSetAttribute(grouped_gemm_kernel<WGRAD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_ACC_BYTES));
+        configured = true;
+    }
+    if (max_tiles <= 0) return MOE_OK;
+    const unsigned grid = (unsigned)imin(max_tiles, sm_count());
+    grouped_gemm_kernel<WGRAD, true><<<grid, NTHREADS, SMEM_ACC_BYTES, st>>>(tmA, tmB, p);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
 template <int KIND, bool MASKT = false>
 int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p_in, int64_t max_tiles,
                 cudaStream_t st, const CUtensorMap *tmM = nullptr, const CUtensorMap *tmO = nullptr) {
@@ -1395,20 +1484,28 @@ bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
     return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0;
 }
 
-// Row ranges of the partial sums of dW. Short on purpose for the leading (hi) term: an fp32 accumulator
-// loses low bits when a long run of same-sign terms is added (e.g. the gradient of a constant input
-// feature); 128 rows per partial keeps that below 1e-5 of the result, and the partials are added in double.
-// The mid and lo terms are 2^-8 and 2^-16 of the hi term and can use long ranges.
+// dW of the gate: the contraction over the tokens is cut into row ranges (one float partial per range and precision
+// term, added in double afterwards), and inside a range the tensor-core accumulator is restarted every GB_ROWS_HI rows
+// for the leading (hi) term: an fp32 accumulator loses low bits when a long run of same-sign terms is added (e.g. the
+// gradient of a constant input feature); 128 rows keep that below 1e-5 of the result. The mid and lo terms are 2^-8
+// and 2^-16 of the hi term and restart every GB_ROWS_LO rows. The restarts' sums are added in shared memory (see the
+// ACC kernel), so only one partial per range goes to global memory.
 constexpr int GB_ROWS_HI = 128, GB_ROWS_LO = 2048;
-static void gate_bwd_split(int64_t T, int32_t *S_hi, int32_t *S_lo) {
-    *S_hi = (int32_t)(T > 0 ? cdiv(T, GB_ROWS_HI) : 1);
-    *S_lo = (int32_t)(T > 0 ? cdiv(T, GB_ROWS_LO) : 1);
+static void gate_bwd_split(int64_t T, int32_t d, int32_t n, int32_t *nranges, int32_t *rows) {
+    const int64_t tiles_per_range = cdiv(d, BM) * cdiv(2 * n, BN);
+    int64_t want = cdiv(3 * (int64_t)sm_count(), tiles_per_range);  // about three waves of hi-term tiles
+    const int64_t most = T > 0 ? cdiv(T, GB_ROWS_LO) : 1;
+    if (want > most) want = most;
+    if (want < 1) want = 1;
+    const int64_t r = cdiv(cdiv(T > 0 ? T : 1, want), GB_ROWS_LO) * GB_ROWS_LO;  // whole lo sub-blocks per range
+    *rows = (int32_t)r;
+    *nranges = (int32_t)(T > 0 ? cdiv(T, r) : 1);
 }
 
 int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n) {
-    int32_t S_hi, S_lo;
-    gate_bwd_split(T, &S_hi, &S_lo);
-    return (int64_t)(S_hi + 2 * S_lo) * d * 2 * n;
+    int32_t nr, rows;
+    gate_bwd_split(T, d, n, &nr, &rows);
+    return (int64_t)3 * nr * d * 2 * n;
 }
 
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
@@ -1422,19 +1519,19 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
     }
     split_weights_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
     MOE_LAUNCHED();
-    int32_t S_hi, S_lo;
-    gate_bwd_split(T, &S_hi, &S_lo);
+    int32_t nr, rows;
+    gate_bwd_split(T, d, n, &nr, &rows);
     {   // dW partials: contraction over the tokens, cut into row ranges, one set per precision term
         CUtensorMap tmA, tmB;
         MOE_TRY(map_rows_mnmajor(&tmA, x, T, d, BM / 64));
         MOE_TRY(map_rows_mnmajor(&tmB, dsplit, T, 3 * n2, BN / 64));
         GemmParams p = default_params();
-        p.nseg = S_hi + 2 * S_lo; p.M = d; p.N = n2; p.R = T; p.out_f32 = partials; p.status = status;
-        p.segs_term0 = S_hi; p.rows_per_seg0 = GB_ROWS_HI;
-        p.rows_per_seg = GB_ROWS_LO; p.segs_per_term = S_lo; p.b_term_chunks = n2 / 64;
-        MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
-        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, S_hi + 2 * S_lo, (int64_t)d * n2, d, n, dWg,
-                                                                                            dWn);
+        p.nseg = 3 * nr; p.M = d; p.N = n2; p.R = T; p.out_f32 = partials; p.status = status;
+        p.segs_term0 = nr; p.rows_per_seg0 = rows;
+        p.rows_per_seg = rows; p.segs_per_term = nr; p.b_term_chunks = n2 / 64;
+        p.sub_kb0 = GB_ROWS_HI / BK; p.sub_kb = GB_ROWS_LO / BK; p.interleave = 3;
+        MOE_TRY(launch_acc_wgrad(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
+        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, 3 * nr, (int64_t)d * n2, d, n, dWg, dWn);
         MOE_LAUNCHED();
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
