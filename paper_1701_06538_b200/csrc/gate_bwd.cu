@@ -134,6 +134,101 @@ __global__ void __launch_bounds__(256) gate_logit_grads_kernel(
     }
 }
 
+// The same for the tensor-core path (split output, n a multiple of 32): a lane owns PAIRS of adjacent columns, so the
+// row is read with 8-byte loads and the six bf16 terms of a pair leave as 4-byte stores (half the memory instructions),
+// and only the first KS slots are compared (KS >= k).
+template <int NVP, int KS>  // column pairs per lane (n <= 64 * NVP)
+__global__ void __launch_bounds__(256) gate_logit_grads_pairs_kernel(
+    const float *__restrict__ noise, const float *__restrict__ clean, const float *__restrict__ raw,
+    const int32_t *__restrict__ idx, const float *__restrict__ gates, const float *__restrict__ kth_vals,
+    const int32_t *__restrict__ kth_idx, const float *__restrict__ dgates, const float *__restrict__ dload,
+    const int32_t *__restrict__ dload_row_group, int64_t rows, int32_t n, int32_t k, bf16 *__restrict__ dsplit,
+    const int32_t *__restrict__ split_row_index) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    int32_t sel_idx[KS];
+    float sel_dh[KS];
+    float inner = 0.0f;
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+        sel_idx[s] = s < k ? idx[row * k + s] : -1;
+        if (s < k) inner = fmaf(gates[row * k + s], dgates[row * k + s], inner);
+    }
+#pragma unroll
+    for (int s = 0; s < KS; ++s) sel_dh[s] = s < k ? gates[row * k + s] * (dgates[row * k + s] - inner) : 0.0f;
+    const float thr_unsel = kth_vals[row * 2 + 0], thr_sel = kth_vals[row * 2 + 1];
+    const int32_t j_k = kth_idx[row * 2 + 0], j_k1 = kth_idx[row * 2 + 1];
+    const float *dl = dload + (dload_row_group ? (int64_t)dload_row_group[row] * n : 0);
+    const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
+
+    float2 cv[NVP], rv[NVP], ev[NVP], dv[NVP];
+    float dhv[2 * NVP], qv[2 * NVP], zqv[2 * NVP];
+#pragma unroll
+    for (int u = 0; u < NVP; ++u) {  // all loads of the row first
+        const int32_t j = 2 * lane + 64 * u;
+        const bool in = j < n;
+        const float2 z2 = make_float2(0.0f, 0.0f);
+        cv[u] = in ? *reinterpret_cast<const float2 *>(c + j) : z2;
+        rv[u] = in ? *reinterpret_cast<const float2 *>(r + j) : z2;
+        ev[u] = in ? *reinterpret_cast<const float2 *>(e + j) : z2;
+        dv[u] = in ? *reinterpret_cast<const float2 *>(dl + j) : z2;
+    }
+    float q_sel = 0.0f, q_uns = 0.0f;
+#pragma unroll
+    for (int u = 0; u < 2 * NVP; ++u) {
+        const int32_t j = 2 * lane + 64 * (u >> 1) + (u & 1);
+        const float cj = (u & 1) ? cv[u >> 1].y : cv[u >> 1].x, rj = (u & 1) ? rv[u >> 1].y : rv[u >> 1].x;
+        const float dlj = (u & 1) ? dv[u >> 1].y : dv[u >> 1].x;
+        dhv[u] = qv[u] = zqv[u] = 0.0f;
+        if (j < n) {
+            bool sel = false;
+#pragma unroll
+            for (int s = 0; s < KS; ++s)
+                if (sel_idx[s] == j) { sel = true; dhv[u] = sel_dh[s]; }
+            const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
+            const float z = (cj - (sel ? thr_sel : thr_unsel)) / sigma;
+            if (isfinite(z)) {
+                qv[u] = dlj * (expf(-0.5f * z * z) * 0.39894228040143267794f) / sigma;
+                zqv[u] = z * qv[u];
+            }
+            if (sel) q_sel += qv[u]; else q_uns += qv[u];
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        q_sel += __shfl_xor_sync(0xffffffffu, q_sel, off);
+        q_uns += __shfl_xor_sync(0xffffffffu, q_uns, off);
+    }
+    const int64_t orow = split_row_index ? split_row_index[row] : row;  // e.g. sorted by primary group
+    bf16 *o = dsplit + orow * (6 * (int64_t)n);
+#pragma unroll
+    for (int u = 0; u < NVP; ++u) {
+        const int32_t j = 2 * lane + 64 * u;
+        if (j >= n) continue;
+        float dc[2], dr[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float rj = h ? rv[u].y : rv[u].x, ej = h ? ev[u].y : ev[u].x;
+            float dh = dhv[2 * u + h];
+            if (j + h == j_k1) dh -= q_sel;
+            if (j + h == j_k && k < n) dh -= q_uns;
+            const float dsigma = fmaf(ej, dh, -zqv[2 * u + h]);
+            dc[h] = qv[2 * u + h] + dh;
+            dr[h] = dsigma / (1.0f + expf(-rj));
+        }
+        // three-term bf16 split (hi | mid | lo), row layout [3][clean n | raw n], for the tensor-core products
+#pragma unroll
+        for (int term = 0; term < 3; ++term) {
+            const __nv_bfloat162 bc = __floats2bfloat162_rn(dc[0], dc[1]), br = __floats2bfloat162_rn(dr[0], dr[1]);
+            *reinterpret_cast<__nv_bfloat162 *>(o + term * 2 * n + j) = bc;
+            *reinterpret_cast<__nv_bfloat162 *>(o + term * 2 * n + n + j) = br;
+            dc[0] -= __bfloat162float(bc.x); dc[1] -= __bfloat162float(bc.y);
+            dr[0] -= __bfloat162float(br.x); dr[1] -= __bfloat162float(br.y);
+        }
+    }
+}
+
 int32_t launch_gate_logit_grads(const float *noise, const float *clean, const float *raw, const int32_t *idx,
                                 const float *gates, const float *kth_vals, const int32_t *kth_idx,
                                 const float *dgates, const float *dload, const int32_t *dload_row_group,
@@ -141,6 +236,25 @@ int32_t launch_gate_logit_grads(const float *noise, const float *clean, const fl
                                 const int32_t *split_row_index, cudaStream_t st) {
     if (rows == 0) return MOE_OK;
     const unsigned grid = (unsigned)cdiv(rows, 8);
+    if (dsplit && n % 32 == 0 && n <= 256) {  // the tensor-core path: paired columns
+#define MOE_LOGIT_PAIRS_KS(NVP, KS)                                                                                      \
+    gate_logit_grads_pairs_kernel<NVP, KS><<<grid, 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals, kth_idx, dgates, \
+                                                                 dload, dload_row_group, rows, n, k, (bf16 *)dsplit,      \
+                                                                 split_row_index)
+#define MOE_LOGIT_PAIRS(NVP)                                \
+    do {                                                    \
+        if (k <= 2) MOE_LOGIT_PAIRS_KS(NVP, 2);             \
+        else if (k <= 4) MOE_LOGIT_PAIRS_KS(NVP, 4);        \
+        else MOE_LOGIT_PAIRS_KS(NVP, MOE_MAX_K);            \
+    } while (0)
+        if (n <= 64) MOE_LOGIT_PAIRS(1);
+        else if (n <= 128) MOE_LOGIT_PAIRS(2);
+        else MOE_LOGIT_PAIRS(4);
+#undef MOE_LOGIT_PAIRS
+#undef MOE_LOGIT_PAIRS_KS
+        MOE_LAUNCHED();
+        return MOE_OK;
+    }
 #define MOE_LOGIT_GRADS(NV)                                                                                          \
     gate_logit_grads_kernel<NV><<<grid, 256, 0, st>>>(noise, clean, raw, idx, gates, kth_vals, kth_idx, dgates, dload, \
                                                       dload_row_group, rows, n, k, dclean, draw, (bf16 *)dsplit,      \

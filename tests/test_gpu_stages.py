@@ -30,6 +30,8 @@ FLAT = [
     small_workload("one-expert-f32", T=100, d=12, h=20, n=1, k=1, seed=7),
     small_workload("long-segments-bf16", T=3000, d=128, h=320, n=5, k=2, act="bf16", seed=8),  # 256-row tile pairs
     small_workload("screened-gate-bf16", T=4096, d=128, h=64, n=32, k=4, act="bf16", seed=9),  # tensor-core routing screen
+    # routing screen + tensor-core gate backward with a token count that is no multiple of any tile or row range
+    small_workload("screened-ragged-bf16", T=4100, d=128, h=64, n=32, k=2, act="bf16", seed=12),
     # SM-pair kernels with a heavily skewed load: one very long segment, short ones, (nearly) empty ones
     small_workload("skewed-long-bf16", T=4096, d=192, h=256, n=6, k=1, act="bf16", seed=11, skew="zipf", gamma=3.0),
     synth.CONFIGS["c1"],
