@@ -40,7 +40,8 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_STAGE_BYTES = 8 * 4096;  // per epilogue warp: a 32 x 128 B slab for float output
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
-constexpr int NTHREADS = 320;  // TMA warp, MMA warp, 8 epilogue warps
+constexpr int NTHREADS = 320;   // TMA warp, MMA warp, 8 epilogue warps
+constexpr int NTHREADS2 = 352;  // two-CTA kernel: + one warp that fixes the ragged K tail of the wgrad ahead of the MMAs
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Kind { ROW_BMN = 0, ROW_BK = 1, WGRAD = 2 };
@@ -722,7 +723,7 @@ __host__ __device__ constexpr uint32_t make_idesc2(int a_mn, int b_mn) {  // M 2
 // MASKT: the ReLU mask of the dgrad GEMM is not read row by row from global memory by the epilogue but
 // fetched as a 128 x 256 tile by TMA (one stage fewer in exchange for the 64 KiB it occupies).
 template <int KIND, bool MASKT>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(NTHREADS2, 1)
 grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmO,
                      const GemmParams p) {
@@ -737,8 +738,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     auto empty_bar = [&](int s) { return bars + 8u * (NST + s); };
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * NST + a); };
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * NST + 2 + a); };
-    // WGRAD only: afull = this CTA's own A tile has landed (it may need its ragged K tail zeroed before use);
-    // ready (even CTA) = the odd CTA's A tile is landed and fixed
+    // WGRAD only: afull = this CTA's own A tile has landed (its ragged K tail is zeroed before use);
+    // ready (even CTA) = both CTAs' A tiles are landed and fixed
     auto afull_bar = [&](int s) { return bars + 8u * (2 * NST + 4 + s); };
     auto ready_bar = [&](int s) { return bars + 8u * (3 * NST + 4 + s); };
     const uint32_t mfull_bar = bars + 8u * 28, mempty_bar = bars + 8u * 29;  // mask tile landed / read by all 8 epilogue warps
@@ -753,7 +754,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     if (threadIdx.x == 0) {
         for (int s = 0; s < NST; ++s) {
             mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1);
-            mbar_init(afull_bar(s), 1); mbar_init(ready_bar(s), 1);
+            mbar_init(afull_bar(s), 1); mbar_init(ready_bar(s), 2);  // ready: both CTAs' tail-fixing warps
         }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
         mbar_init(mfull_bar, 1); mbar_init(mempty_bar, 8);
@@ -776,6 +777,18 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // rows [valid, 64) of stage s's A tile (K rows past the segment end, both 64-column chunks) := 0
+    auto zero_tail = [&](int s, int valid) {
+        const int lines = (BK - valid) * 2;
+        for (int u = lane; u < lines * 8; u += 32) {
+            const int line = u >> 3, part = u & 7;
+            const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
+            *reinterpret_cast<uint4 *>(smem + s * STAGE2_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
+                make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+    };
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
@@ -844,19 +857,6 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
-        // WGRAD: both CTAs' warp 1 first fix the ragged K tail of their own A tile (rows of the last block
-        // that lie past the segment end are zeroed); the odd CTA then reports its tile ready.
-        auto zero_tail = [&](int s, int valid) {
-            const int lines = (BK - valid) * 2;
-            for (int u = lane; u < lines * 8; u += 32) {
-                const int line = u >> 3, part = u & 7;
-                const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
-                *reinterpret_cast<uint4 *>(smem + s * STAGE2_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
-                    make_uint4(0, 0, 0, 0);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-        };
         if (rank == 0) {
             constexpr uint32_t idesc = make_idesc2(KIND == WGRAD ? 1 : 0, KIND == ROW_BK ? 0 : 1);
             int s = 0, acc = 0;
@@ -874,10 +874,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (KIND == WGRAD) {
                         const int valid = t.row_end - (t.row0 + kb * BK);
                         if (valid < BK) {
-                            const uint32_t tp = (tail_ph >> s) & 1u;
-                            ok = mbar_wait(afull_bar(s), tp, abort_flag, p.status);
-                            if (!ok) break;
-                            zero_tail(s, valid);
+                            const uint32_t tp = (tail_ph >> s) & 1u;  // fixed by warp 10 of both CTAs, ahead of time
                             ok = mbar_wait(ready_bar(s), tp, abort_flag, p.status) && mbar_try_wait_cluster(ready_bar(s), tp);
                             if (!ok) break;
                             tail_ph ^= 1u << s;
@@ -903,7 +900,12 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 __syncwarp();
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
-        } else if (KIND == WGRAD) {
+        }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------------ WGRAD: ragged K tail (both CTAs)
+        // The last K block of a segment holds rows of the next segment: they are zeroed in this CTA's A tile as soon as
+        // it has landed, several stages before the MMAs get there, and reported on the even CTA's "ready" barrier.
+        if (KIND == WGRAD) {
             int s = 0;
             uint32_t tail_ph = 0;
             bool ok = true;
@@ -1232,7 +1234,7 @@ int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = SMEM2_BYTES; cfg.stream = st;
+    cfg.blockDim = dim3(NTHREADS2); cfg.dynamicSmemBytes = SMEM2_BYTES; cfg.stream = st;
     cfg.attrs = &attr; cfg.numAttrs = 1;
     if (!max_clusters) {
         MOE_CUDA(cudaFuncSetAttribute(grouped_gemm2_kernel<KIND, MASKT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
