@@ -96,7 +96,14 @@ struct GateWs {
     void *wsplit;
     int32_t *unsafe_list, *unsafe_count, *full_list;
     void *chain_list;
+    // the same for the secondary gates of the hierarchical layer (rows = slots sorted by primary group)
+    bool screen2;
+    void *xs_p, *wsplit_s, *chain_list_s;
+    float *cr_s, *wnorm_s, *wt_s;
+    int32_t *unsafe_list_s, *unsafe_count_s;
     GateWs(Carver &cv, const Dims &D) {
+        screen2 = false;
+        xs_p = wsplit_s = chain_list_s = nullptr; cr_s = wnorm_s = wt_s = nullptr; unsafe_list_s = unsafe_count_s = nullptr;
         idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
         cr = wnorm = xnorm = wt = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = full_list = nullptr; chain_list = nullptr;
         const int64_t n1 = D.hier ? D.a : D.n;  // width of the (first) gate
@@ -120,7 +127,20 @@ struct GateWs {
         counts_p = cv.take<int32_t>(D.a);
         offsets_p = cv.take<int32_t>(D.a + 1);
         scratch = cv.take<int32_t>(dispatch_ws_elems(D.T * D.k1, (int32_t)D.a));
-        tile_prefix = cv.take<int32_t>(D.a + 1);
+        tile_prefix = cv.take<int32_t>(tc_tile_ws_ints(D.T * D.k1, D.a));  // prefix + tile table of the grouped product
+        const int64_t P1 = D.T * D.k1;
+        screen2 = tc_gate_fwd_supported(D.act, P1, (int32_t)D.d, (int32_t)D.b);
+        if (screen2) {
+            if (!xnorm) xnorm = cv.take<float>(D.T);
+            xs_p = cv.take_bytes(P1 * D.d * (int64_t)D.esz);
+            cr_s = cv.take<float>(P1 * 2 * D.b);
+            wsplit_s = cv.take<bf16>(3 * D.a * D.d * 2 * D.b);
+            wnorm_s = cv.take<float>(D.a * 2 * D.b);
+            wt_s = cv.take<float>(D.a * 2 * D.b * D.d);
+            unsafe_list_s = cv.take<int32_t>(P1);
+            unsafe_count_s = cv.take<int32_t>(64);
+            chain_list_s = cv.take_bytes(P1 * 2 * D.b * 8);  // worst case: every column of every slot
+        }
     }
 };
 
@@ -319,11 +339,28 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
     MOE_TRY(launch_dispatch_index(w.idx_p, P1, (int32_t)D.a, w.perm_p, w.inv_perm_p, w.counts_p, w.offsets_p,
                                   w.scratch, st));
     const int64_t lp = D.T * D.a;  // elements of the primary part of the logits tensors
-    MOE_TRY(launch_projection(x, D.act, P1, (int32_t)D.d, (int32_t)D.b, Wg + D.d * D.a, Wnoise + D.d * D.a,
-                              clean + lp, raw_noise + lp, w.offsets_p, (int32_t)D.a, w.perm_p, (int32_t)D.k1,
-                              w.tile_prefix, st));
-    MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s,
-                               g_s, kth_vals + 2 * D.T, kth_idx + 2 * D.T, st));
+    const float *Wg_s = Wg + D.d * D.a, *Wn_s = Wnoise + D.d * D.a;
+    if (w.screen2) {
+        // the routing screen on the grouped product: token rows gathered by group, one weight pair per group
+        MOE_TRY(launch_dispatch_rows(x, D.act, D.T, (int32_t)D.k1, (int32_t)D.d, w.inv_perm_p, w.xs_p, st));
+        MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, (int32_t)D.b, Wg_s, Wn_s, w.wsplit_s, w.wnorm_s,
+                                           w.xnorm, w.unsafe_count_s, w.wt_s, st, (int32_t)D.a, !w.screen));
+        MOE_TRY(launch_tc_gate_fwd_grouped(w.xs_p, P1, (int32_t)D.d, (int32_t)D.a, (int32_t)D.b, w.wsplit_s, w.offsets_p,
+                                           w.tile_prefix, w.cr_s, status_word(ws_base), st));
+        MOE_TRY(launch_gate_screen(w.cr_s, noise + lp, w.xnorm, w.wnorm_s, (int32_t)D.d, P1, (int32_t)D.b, (int32_t)D.k2,
+                                   w.idx_s, g_s, clean + lp, raw_noise + lp, kth_vals + 2 * D.T, kth_idx + 2 * D.T,
+                                   w.unsafe_list_s, w.unsafe_count_s, w.chain_list_s, nullptr, st, w.perm_p,
+                                   (int32_t)D.k1, w.idx_p));
+        MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, (int32_t)D.b, w.wt_s, w.chain_list_s, w.unsafe_count_s + 1,
+                                   clean + lp, raw_noise + lp, st, (int32_t)D.k1));
+        MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s, g_s,
+                                   kth_vals + 2 * D.T, kth_idx + 2 * D.T, st, w.unsafe_list_s, w.unsafe_count_s));
+    } else {
+        MOE_TRY(launch_projection(x, D.act, P1, (int32_t)D.d, (int32_t)D.b, Wg_s, Wn_s, clean + lp, raw_noise + lp,
+                                  w.offsets_p, (int32_t)D.a, w.perm_p, (int32_t)D.k1, w.tile_prefix, st));
+        MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s,
+                                   g_s, kth_vals + 2 * D.T, kth_idx + 2 * D.T, st));
+    }
     return launch_hier_merge(D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.b, w.idx_p, g_p, w.idx_s, g_s, topk_idx,
                              gates, st);
 }

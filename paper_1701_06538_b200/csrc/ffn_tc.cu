@@ -1574,6 +1574,34 @@ int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const
     return launch2<ROW_BMN>(tmA, tmB, p, cdiv(T, 256) * cdiv(n2, BN), st);
 }
 
+// The same for the secondary gates of the hierarchical layer: rows = the slots (t, s1) sorted by primary group
+// (xs_p [P1, d], offsets_p [a + 1]), one [d, 2b] weight pair per group. wsplit_s [3][a * d][2b] (term, group, feature);
+// cr_s [P1, 2b] comes out in sorted order.
+int32_t launch_tc_gate_fwd_grouped(const void *xs_p, int64_t P1, int32_t d, int32_t a, int32_t b, const void *wsplit_s,
+                                   const int32_t *offsets_p, int32_t *tile_prefix, float *cr_s, int32_t *status,
+                                   cudaStream_t st) {
+    if (P1 == 0) return MOE_OK;
+    const int32_t n2 = 2 * b;
+    const bool pairs = use_two_cta(P1, a);
+    CUtensorMap tmA, tmB;
+    MOE_TRY(map_rows_kmajor(&tmA, xs_p, P1, d));
+    {   // the group is the map's last coordinate (stride d rows), the precision term an offset of a * d rows along K
+        const uint64_t dims[4] = {64, (uint64_t)3 * a * d, (uint64_t)(n2 / 64), (uint64_t)a};
+        const uint64_t str[3] = {(uint64_t)n2 * 2, 128, (uint64_t)d * n2 * 2};
+        const uint32_t box[4] = {64, BK, pairs ? 2u : (uint32_t)(BN / 64), 1};
+        MOE_TRY(make_map(&tmB, wsplit_s, 4, dims, str, box));
+    }
+    GemmParams p = default_params();
+    p.offsets = offsets_p; p.tile_prefix = tile_prefix; p.tile_info = tile_info_of(tile_prefix, a);
+    p.nseg = a; p.N = n2; p.K = d; p.R = P1; p.out_f32 = cr_s; p.status = status;
+    p.nterms = 3;
+    for (int i = 0; i < 3; ++i) { p.a_term_col[i] = 0; p.b_term_col[i] = (2 - i) * a * d; }  // lo, mid, hi
+    const int32_t tm = pairs ? 256 : BM;
+    MOE_TRY(launch_tile_table(offsets_p, a, tm, P1, tile_prefix, st));
+    const int64_t max_tiles = (cdiv(P1, tm) + a) * cdiv(n2, BN);
+    return pairs ? launch2<ROW_BMN>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st);
+}
+
 // Secondary gates of the hierarchical layer: the slots (t, s1) sorted by primary group are the rows.
 // xs_p [P1, d] token rows in sorted order, dsplit_s [P1, 3 * 2b] split logit gradients in sorted order.
 bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b) {

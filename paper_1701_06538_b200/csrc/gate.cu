@@ -323,12 +323,13 @@ __global__ void __launch_bounds__(256) split_gate_weights_kernel(const float *__
     }
 }
 
-// one warp per column of [W_g | W_noise]
+// one warp per column of [W_g | W_noise]; blockIdx.y = group (stacked [groups, d, n] matrices)
 __global__ void __launch_bounds__(256) gate_col_norms_kernel(const float *__restrict__ Wg, const float *__restrict__ Wn,
                                                              int32_t d, int32_t n, float *__restrict__ wnorm) {
     const int lane = threadIdx.x & 31;
     const int32_t j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (j >= 2 * n) return;
+    Wg += (int64_t)blockIdx.y * d * n; Wn += (int64_t)blockIdx.y * d * n; wnorm += (int64_t)blockIdx.y * 2 * n;
     const float *W = j < n ? Wg + j : Wn + (j - n);
     double s = 0.0;
     for (int32_t q = lane; q < d; q += 32) { const double v = W[(int64_t)q * n]; s += v * v; }
@@ -363,18 +364,26 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
                                                           int32_t *__restrict__ unsafe_list,
                                                           int32_t *__restrict__ unsafe_count,
                                                           int2 *__restrict__ chain_list,
-                                                          int32_t *__restrict__ full_list) {
+                                                          int32_t *__restrict__ full_list,
+                                                          const int32_t *__restrict__ perm, int32_t kdiv,
+                                                          const int32_t *__restrict__ group_of) {
+    // Grouped use (secondary gates of the hierarchical layer): cr rows are sorted by group; perm maps a sorted row to
+    // its output row (the slot t * k1 + s1), the token is output row / kdiv, group_of gives the slot's group, whose
+    // column norms and weight rows are used. Flat use: perm = group_of = nullptr, kdiv = 1.
     const int lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= T) return;
+    const int64_t srow = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (srow >= T) return;
+    const int64_t row = perm ? perm[srow] : srow;
+    const int32_t group = group_of ? group_of[row] : 0;
+    wnorm += (int64_t)group * 2 * n;
     // per-lane sorted list of (value, index, uncertainty); rest_hi = largest possible chain value of anything
     // that is not in a list
     float lv[KL], lu[KL];
     int32_t li[KL];
 #pragma unroll
     for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
-    const float *c = cr + row * 2 * n, *r = c + n, *e = noise + row * n;
-    const float xn = theta * xnorm[row];
+    const float *c = cr + srow * 2 * n, *r = c + n, *e = noise + row * n;
+    const float xn = theta * xnorm[row / kdiv];
     float rest_hi = -CUDART_INF_F;
     // approximate noisy logit v of column j and a bound u on its distance from the fma chain's value
     auto eval = [&](int32_t j, float cj, float rj, float ej, float &v, float &u) {
@@ -509,20 +518,29 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
         }
         int32_t base = 0;
         const bool few = total <= SCREEN_MAX_CAND;
+        const int32_t wbase = group * 2 * n;  // this group's rows of the transposed weights
         if (lane == 0) {
             unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
             if (few) base = atomicAdd(unsafe_count + 1, 2 * total);
-            else full_list[atomicAdd(unsafe_count + 2, 1)] = (int32_t)row;
+            else if (full_list) full_list[atomicAdd(unsafe_count + 2, 1)] = (int32_t)row;
+            else base = atomicAdd(unsafe_count + 1, 2 * n);  // no whole-row fallback: every column gets its chains
         }
-        if (!few) return;
         base = __shfl_sync(0xffffffffu, base, 0);
+        if (!few) {
+            if (!full_list)
+                for (int32_t j = lane; j < n; j += 32) {
+                    chain_list[base + 2 * j] = make_int2((int32_t)row, wbase + j);
+                    chain_list[base + 2 * j + 1] = make_int2((int32_t)row, wbase + n + j);
+                }
+            return;
+        }
         int pos = 0;
         auto emit = [&](int32_t j, bool cand) {
             const uint32_t b = __ballot_sync(0xffffffffu, cand);
             if (cand) {
                 const int at = base + 2 * (pos + __popc(b & ((1u << lane) - 1u)));
-                chain_list[at] = make_int2((int32_t)row, j);
-                chain_list[at + 1] = make_int2((int32_t)row, n + j);
+                chain_list[at] = make_int2((int32_t)row, wbase + j);
+                chain_list[at + 1] = make_int2((int32_t)row, wbase + n + j);
             }
             pos += __popc(b);
         };
@@ -568,7 +586,10 @@ __global__ void __launch_bounds__(128) gate_chain_kernel(const XT *__restrict__ 
                                                          const float *__restrict__ Wt,
                                                          const int2 *__restrict__ chain_list,
                                                          const int32_t *__restrict__ chain_count,
-                                                         float *__restrict__ clean, float *__restrict__ raw) {
+                                                         float *__restrict__ clean, float *__restrict__ raw,
+                                                         int32_t kdiv) {
+    // entry {output row, row of Wt}: the token is output row / kdiv, the column code is Wt row mod 2n (grouped gates
+    // keep one [2n, d] block of Wt per group)
     __shared__ __align__(16) uint8_t stage[4][2][32 * CHAIN_PITCH];
     const int32_t total = *chain_count;
     const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
@@ -576,7 +597,7 @@ __global__ void __launch_bounds__(128) gate_chain_kernel(const XT *__restrict__ 
     for (int32_t i0 = (blockIdx.x * 4 + wp) * 32; i0 < total; i0 += gridDim.x * 128) {  // warp-uniform
         const int32_t i = i0 + lane;
         const int2 en = chain_list[i < total ? i : total - 1];  // idle lanes shadow the last chain
-        const XT *xr = x + (int64_t)en.x * d;
+        const XT *xr = x + (int64_t)(en.x / kdiv) * d;
         const float *wrow = Wt + (int64_t)en.y * d;
         // instruction u of a step loads 16 bytes of the row of lane 4 u + lane / 8, at byte (lane % 8) * 16
         const float *src[8];
@@ -634,8 +655,9 @@ __global__ void __launch_bounds__(128) gate_chain_kernel(const XT *__restrict__ 
             __syncwarp();
         }
         if (i < total) {
-            if (en.y >= n) raw[(int64_t)en.x * n + (en.y - n)] = acc;
-            else clean[(int64_t)en.x * n + en.y] = acc;
+            const int32_t code = en.y % (2 * n);
+            if (code >= n) raw[(int64_t)en.x * n + (code - n)] = acc;
+            else clean[(int64_t)en.x * n + code] = acc;
         }
     }
 }
@@ -644,6 +666,7 @@ __global__ void __launch_bounds__(128) gate_chain_kernel(const XT *__restrict__ 
 __global__ void __launch_bounds__(256) gate_transpose_weights_kernel(const float *__restrict__ Wg, const float *__restrict__ Wn,
                                                                      int32_t d, int32_t n, float *__restrict__ Wt) {
     __shared__ float tile[32][33];
+    Wg += (int64_t)blockIdx.z * d * n; Wn += (int64_t)blockIdx.z * d * n; Wt += (int64_t)blockIdx.z * 2 * n * d;  // group
     const int q0 = blockIdx.x * 32, c0 = blockIdx.y * 32;  // 2n and d are multiples of 32 on this path
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     for (int i = ty; i < 32; i += 8) {
@@ -655,30 +678,35 @@ __global__ void __launch_bounds__(256) gate_transpose_weights_kernel(const float
 }
 
 int32_t launch_gate_chains(const void *x, int32_t act, int32_t d, int32_t n, const float *Wt, const void *chain_list,
-                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st) {
+                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st, int32_t kdiv) {
     const unsigned grid = 148 * 16;
     if (act == MOE_BF16)
         gate_chain_kernel<bf16><<<grid, 128, 0, st>>>((const bf16 *)x, d, n, Wt, (const int2 *)chain_list, chain_count, clean,
-                                                      raw);
+                                                      raw, kdiv);
     else
         gate_chain_kernel<float><<<grid, 128, 0, st>>>((const float *)x, d, n, Wt, (const int2 *)chain_list, chain_count, clean,
-                                                       raw);
+                                                       raw, kdiv);
     MOE_LAUNCHED();
     return MOE_OK;
 }
 
 int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
                                    const float *Wn, void *wsplit, float *wnorm, float *xnorm,
-                                   int32_t *unsafe_count, float *wt, cudaStream_t st) {
-    gate_transpose_weights_kernel<<<dim3((unsigned)(d / 32), (unsigned)(2 * n / 32)), 256, 0, st>>>(Wg, Wn, d, n, wt);
+                                   int32_t *unsafe_count, float *wt, cudaStream_t st, int32_t groups, bool with_xnorm) {
+    // groups > 1: Wg, Wn are stacks [groups, d, n]; wsplit [3][groups * d][2n], wnorm [groups][2n], wt [groups][2n][d]
+    gate_transpose_weights_kernel<<<dim3((unsigned)(d / 32), (unsigned)(2 * n / 32), (unsigned)groups), 256, 0, st>>>(Wg, Wn, d, n,
+                                                                                                                      wt);
     MOE_LAUNCHED();
-    split_gate_weights_kernel<<<(unsigned)cdiv((int64_t)d * 2 * n, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
+    split_gate_weights_kernel<<<(unsigned)cdiv((int64_t)groups * d * 2 * n, 256), 256, 0, st>>>(Wg, Wn, groups * d, n,
+                                                                                                  (bf16 *)wsplit);
     MOE_LAUNCHED();
-    gate_col_norms_kernel<<<(unsigned)cdiv(2 * n, 8), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
+    gate_col_norms_kernel<<<dim3((unsigned)cdiv(2 * n, 8), (unsigned)groups), 256, 0, st>>>(Wg, Wn, d, n, wnorm);
     MOE_LAUNCHED();
-    if (act == MOE_BF16) row_norms_kernel<bf16><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const bf16 *)x, T, d, xnorm);
-    else row_norms_kernel<float><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const float *)x, T, d, xnorm);
-    MOE_LAUNCHED();
+    if (with_xnorm) {
+        if (act == MOE_BF16) row_norms_kernel<bf16><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const bf16 *)x, T, d, xnorm);
+        else row_norms_kernel<float><<<(unsigned)cdiv(T, 8), 256, 0, st>>>((const float *)x, T, d, xnorm);
+        MOE_LAUNCHED();
+    }
     MOE_CUDA(cudaMemsetAsync(unsafe_count, 0, 4 * sizeof(int32_t), st));  // rows to re-select, chains, full-chain rows
     return MOE_OK;
 }
@@ -686,7 +714,8 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
 int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
-                           void *chain_list, int32_t *full_list, cudaStream_t st) {
+                           void *chain_list, int32_t *full_list, cudaStream_t st, const int32_t *perm, int32_t kdiv,
+                           const int32_t *group_of) {
     // worst-case rounding of the fma chain, plus two truncations of an fp32 accumulator per MMA step of the
     // three-term tensor-core product (3d/16 steps and the additions inside a step), plus the split residual
     const double u = ldexp(1.0, -24);
@@ -697,7 +726,7 @@ int32_t launch_gate_screen(const float *cr, const float *noise, const float *xno
 #define MOE_SCREEN_KL(NV, KL)                                                                                            \
     gate_screen_kernel<NV, KL><<<grid, 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean, raw,  \
                                                      kth_vals, kth_idx, unsafe_list, unsafe_count, (int2 *)chain_list, \
-                                                     full_list)
+                                                     full_list, perm, kdiv, group_of)
 #define MOE_SCREEN(NV)                                \
     do {                                              \
         if (k <= 2) MOE_SCREEN_KL(NV, 4);             \

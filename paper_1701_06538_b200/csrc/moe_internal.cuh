@@ -75,17 +75,20 @@ int32_t launch_gate_select(const float *clean, const float *raw, const float *no
 // Tensor-core screening of the routing (see gate.cu): weights split / norms, then the screening select.
 int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, const float *Wg,
                                    const float *Wn, void *wsplit, float *wnorm, float *xnorm,
-                                   int32_t *unsafe_count, float *wt /* [2n, d]: columns as rows */, cudaStream_t st);
+                                   int32_t *unsafe_count, float *wt /* [2n, d]: columns as rows */, cudaStream_t st,
+                                   int32_t groups = 1, bool with_xnorm = true);
 int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
-                           void *chain_list, int32_t *full_list, cudaStream_t st);
+                           void *chain_list, int32_t *full_list, cudaStream_t st, const int32_t *perm = nullptr,
+                           int32_t kdiv = 1, const int32_t *group_of = nullptr);
 // Rows the screen cannot certify: unsafe_list / unsafe_count[0] = rows whose selection is repeated; chain_list
 // (int2 {row, column code}, unsafe_count[1] entries, at most 2 * SCREEN_MAX_CAND per row) = single fma chains to
 // recompute; full_list / unsafe_count[2] = rows with more candidates than that, which take the whole projection.
 constexpr int SCREEN_MAX_CAND = 16;
 int32_t launch_gate_chains(const void *x, int32_t act, int32_t d, int32_t n, const float *Wt, const void *chain_list,
-                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st);  // Wt [2n, d]
+                           const int32_t *chain_count, float *clean, float *raw, cudaStream_t st,
+                           int32_t kdiv = 1);  // Wt [2n, d] (per group); token = output row / kdiv
 bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n);
 // cr [T, 2n] (float) = x . [W_g | W_noise] from the three-term split wsplit [3, d, 2n]
 int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,
@@ -198,6 +201,9 @@ int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n);  // floats of par
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
                            float *dX_gate, int32_t *status, cudaStream_t st);
+int32_t launch_tc_gate_fwd_grouped(const void *xs_p, int64_t P1, int32_t d, int32_t a, int32_t b, const void *wsplit_s,
+                                   const int32_t *offsets_p, int32_t *tile_prefix, float *cr_s, int32_t *status,
+                                   cudaStream_t st);
 bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b);
 int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, void *wsplit_s, const float *Wg_s,
                                      const float *Wn_s, const int32_t *offsets_p, int32_t *tile_prefix, int32_t a,

@@ -120,3 +120,33 @@ def test_hier_fused(case):
             assert_close(host(G[name]), getattr(Bk, name), tol, name)
     assert_close(host(G["dWg"]), cat_parts(Bk.dWg), tol, "dWg")
     assert_close(host(G["dWnoise"]), cat_parts(Bk.dWnoise), tol, "dWnoise")
+
+
+def test_hier_secondary_ties_take_every_column_through_the_chain():
+    """Identical secondary gate columns and zero secondary noise: every expert of a group ties, far more candidates
+    than the screen resolves column by column, so each such slot gets the chains of all its columns; the oracle's
+    lowest-index rule must come out."""
+    w = small_workload("hier-sec-ties", T=600, d=64, h=64, n=3 * 32, k=4, a=3, k1=2, b=32, k2=2, act="bf16", seed=36)
+    I = synth.make_all(w)
+    Wg_p, Wg_s = I["Wg"]
+    Wn_p, Wn_s = I["Wnoise"]
+    n_p, n_s = I["noise"]
+    Wg_s[:] = Wg_s[:, :, :1]          # all columns of a group equal
+    Wn_s[:] = Wn_s[:, :, :1]
+    n_s[:] = 0.0
+    assert screened(w)
+    F, _ = oracle_run(w, I, backward=False)
+    D, cfg = device_inputs(w, I), cfg_of(w)
+    S = B.moe_query_sizes(cfg)
+    ws = B.empty_bytes(S.ws_bytes)
+    idx, gates = i32(w.T, w.k), f32(S.gates_elems)
+    clean, raw = f32(S.logits_elems), f32(S.logits_elems)
+    kv, ki = f32(S.kth_elems), i32(S.kth_elems)
+    B.moe_gate(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], idx, gates, clean, raw, kv, ki, ws)
+    assert B.moe_check_status(ws) == 0
+    want = gate_tensors(F.G)
+    sec = host(idx).reshape(w.T, w.k1, w.k2) % w.b
+    assert (sec[..., 0] == 0).all() and (sec[..., 1] == 1).all()   # lowest indices win the ties
+    assert (host(idx) == want["topk_idx"]).all()
+    assert (host(ki) == want["kth_idx"]).all()
+    assert_close(host(gates), want["gates"], TOL_F32, "gates")

@@ -50,7 +50,10 @@ def screened(w):
     """True where moe_gate screens the routing on the tensor cores: bf16, widths that are multiples of 64, and
     either forced (MOE_GATE_SCREEN=1, set by this test session) or a projection of at least 1e9 multiply-adds."""
     n1 = w.a if w.a else w.n
-    return w.act == "bf16" and w.T >= 256 and w.d % 64 == 0 and (2 * n1) % 64 == 0
+    first = w.act == "bf16" and w.T >= 256 and w.d % 64 == 0 and (2 * n1) % 64 == 0
+    # the secondary gates of the hierarchical layer are screened on their own (rows = T * k1 slots, width b)
+    second = bool(w.a) and w.act == "bf16" and w.T * w.k1 >= 256 and w.d % 64 == 0 and (2 * w.b) % 64 == 0
+    return first or second
 
 
 os.environ["MOE_GATE_SCREEN"] = "1"  # small test shapes would otherwise stay below the automatic threshold
