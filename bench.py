@@ -36,7 +36,7 @@ L2_BYTES = 126 * 2 ** 20
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of the six expert GEMMs of one step, from one ncu capture of the bench
 # command (the summary under profiles/ names it); workloads without a capture report null
-NCU_TRAFFIC_BYTES_PER_STEP = {"c5-wide-zipf-128": 31.32e9}  # profiles/grouped_gemm_c5_full_dram_traffic.txt
+NCU_TRAFFIC_BYTES_PER_STEP = {"c5-wide-zipf-128": 31.80e9}  # profiles/grouped_gemm_c5_full_dram_traffic.txt
 
 
 def load_peaks():
