@@ -21,6 +21,8 @@ HIER = [
     small_workload("hier-wide-bf16", T=777, d=128, h=64, n=96, k=6, a=3, k1=2, b=32, k2=3, act="bf16", seed=34),
     # both gating levels wide enough for the tensor-core gate backward (2a and 2b multiples of 64)
     small_workload("hier-tc-bf16", T=2100, d=64, h=64, n=1024, k=4, a=32, k1=2, b=32, k2=2, act="bf16", seed=35),
+    # primary gate wide enough for the routing screen, secondary gates too narrow for it
+    small_workload("hier-primary-screen-bf16", T=1024, d=64, h=64, n=256, k=4, a=32, k1=2, b=8, k2=2, act="bf16", seed=37),
 ]
 
 
