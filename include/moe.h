@@ -120,9 +120,12 @@ int32_t moe_check_status(const void *ws, void *stream);
  * The logits that decide the routing are evaluated in single precision in one fixed order
  * (one fused-multiply-add chain per output over ascending input feature; softplus in double
  * rounded once; H by one fused multiply-add), so the routing is reproducible bit for bit.
- * For large bf16 batches the routing is first screened with a tensor-core product and an error
- * bound; tokens whose order the bound proves keep that result (indices identical to the chain's,
- * clean / raw_noise / kth_vals within 1e-7 of it), all other tokens are redone with the chain.
+ * For large bf16 batches the routing (of the flat gate and of both levels of the hierarchical one)
+ * is first screened with a tensor-core product and an error bound; tokens whose order the bound
+ * proves keep that result (indices identical to the chain's, clean / raw_noise / kth_vals within
+ * 1e-7 of it). For every other token the columns that can still reach rank k+1 are re-evaluated
+ * with the chain and the selection is repeated, so its indices are the chain's too; its other
+ * columns keep the tensor-core values.
  * Environment: MOE_GATE_SCREEN=0 disables the screen, =1 uses it whenever the shapes allow.
  * `noise` is an input: standard normal draws, or zeros for noiseless gating.
  * in : x [T,d] act, Wg/Wnoise [d,n], noise [T,n]
