@@ -95,6 +95,9 @@ typedef struct moe_ctx_layout {
  * rows of x / hid a multiple of 16 bytes, hierarchical fields consistent (n = a*b, k = k1*k2). */
 int32_t moe_validate(const moe_config *cfg);
 int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *host_out);
+/* The two workspace sizes alone (bytes a forward / a backward call needs in `ws`), for callers that do not want
+ * the whole moe_sizes record. Host pointers; either may be NULL. */
+int32_t moe_workspace_bytes(const moe_config *cfg, size_t *host_fwd, size_t *host_bwd);
 int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *host_out);
 const char *moe_status_string(int32_t status);
 

@@ -19,7 +19,7 @@ MOE_F32, MOE_BF16 = 0, 1
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED", 3: "MOE_ERR_WORKSPACE",
                 4: "MOE_ERR_CUDA", 5: "MOE_ERR_TIMEOUT"}
 
-EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
+EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_workspace_bytes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
            "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward"]
@@ -102,6 +102,15 @@ def moe_debug_launch_count() -> int:
 
 def moe_validate(cfg) -> int:
     return lib().moe_validate(ctypes.byref(cfg))
+
+
+def moe_workspace_bytes(cfg):
+    """(forward, backward) workspace bytes."""
+    f, b = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    status = lib().moe_workspace_bytes(ctypes.byref(cfg), ctypes.byref(f), ctypes.byref(b))
+    if status:
+        raise MoeError("moe_workspace_bytes", status)
+    return f.value, b.value
 
 
 def moe_query_sizes(cfg) -> moe_sizes:

@@ -586,6 +586,14 @@ int64_t moe_debug_launch_count(void) { return (int64_t)g_launches.load(std::memo
 
 int32_t moe_validate(const moe_config *cfg) { return check_config(cfg); }
 
+int32_t moe_workspace_bytes(const moe_config *cfg, size_t *host_fwd, size_t *host_bwd) {
+    moe_sizes s;
+    MOE_TRY(moe_query_sizes(cfg, &s));
+    if (host_fwd) *host_fwd = (size_t)s.ws_fwd_bytes;
+    if (host_bwd) *host_bwd = (size_t)s.ws_bwd_bytes;
+    return MOE_OK;
+}
+
 int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *out) {
     MOE_TRY(check_config(cfg));
     if (!out) return MOE_ERR_INVALID_ARG;

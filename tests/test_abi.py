@@ -44,6 +44,7 @@ def test_validate_accepts_the_five_workloads_and_rejects_bad_ones(lib):
         assert B.moe_validate(cfg) == 0, w.name
         S = B.moe_query_sizes(cfg)
         assert S.R == w.T * w.k and S.ctx_bytes > 0 and S.ws_bwd_bytes >= S.ws_bytes > 0
+        assert B.moe_workspace_bytes(cfg) == (S.ws_fwd_bytes, S.ws_bwd_bytes)
     ok = dict(T=16, d=64, h=64, n=8, k=2, act="f32")
     bad = [dict(ok, k=0), dict(ok, k=9), dict(ok, k=3, n=2), dict(ok, d=3), dict(ok, h=0), dict(ok, T=-1),
            dict(ok, act=7), dict(ok, n=1 << 20), dict(ok, a=2, b=3, k1=1, k2=1), dict(ok, a=2, b=4, k1=2, k2=2),
