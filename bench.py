@@ -286,7 +286,9 @@ def run_ours(args, w):
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
     def run_e2e(K):
-        ev_in = [torch.cuda.Event() for _ in range(K)]
+        ev_in_f = [torch.cuda.Event() for _ in range(K)]   # x and noise of step i are on the device
+        ev_in_b = [torch.cuda.Event() for _ in range(K)]   # dY too
+        ev_fwd = [torch.cuda.Event() for _ in range(K)]
         ev_comp = [torch.cuda.Event() for _ in range(K)]
         ev_out = [torch.cuda.Event() for _ in range(K)]
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -299,22 +301,26 @@ def run_ours(args, w):
                 if i >= 2:
                     s_in.wait_event(ev_comp[i - 2])  # the kernels that read this input set are done
                 Bf["x"].copy_(hx, non_blocking=True); Bf["noise"].copy_(hnoise, non_blocking=True)
-                Bf["dY"].copy_(hdY, non_blocking=True)
-                ev_in[i].record()
+                ev_in_f[i].record()
+                Bf["dY"].copy_(hdY, non_blocking=True)  # only the backward needs it: it arrives during the forward
+                ev_in_b[i].record()
             with torch.cuda.stream(s_comp):
-                s_comp.wait_event(ev_in[i])
+                s_comp.wait_event(ev_in_f[i])
                 if i >= 2:
                     s_comp.wait_event(ev_out[i - 2])  # this output set has been copied out
                 B.moe_forward(cfg, Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
                               Bf["y"], Bf["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+                ev_fwd[i].record()
+                s_comp.wait_event(ev_in_b[i])
                 B.moe_backward(cfg, Bf["dY"], Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"],
                                D["b2"], D["ctx"], Bf["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"],
                                D["db2"], D["ws"])
                 ev_comp[i].record()
             with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_fwd[i])  # y and the losses leave while the backward runs
+                hy.copy_(Bf["y"], non_blocking=True); hl.copy_(Bf["losses"], non_blocking=True)
                 s_out.wait_event(ev_comp[i])
-                hy.copy_(Bf["y"], non_blocking=True); hdX.copy_(Bf["dX"], non_blocking=True)
-                hl.copy_(Bf["losses"], non_blocking=True)
+                hdX.copy_(Bf["dX"], non_blocking=True)
                 ev_out[i].record()
         with torch.cuda.stream(s_out):
             t1.record()
