@@ -19,7 +19,7 @@ def _worker(rank, world, port, out):
 
 def test_timing_is_the_max_over_ranks_and_throughput_is_whole_job():
     world = 2
-    with mp.Manager() as m:
+    with mp.get_context("spawn").Manager() as m:
         out = m.dict()
         mp.spawn(_worker, args=(world, 29517 + os.getpid() % 200, out), nprocs=world, join=True)
         res = dict(out)
