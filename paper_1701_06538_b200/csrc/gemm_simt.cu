@@ -155,11 +155,16 @@ int32_t launch_simt_gemm(const SimtGemm &g, int32_t *tile_prefix, cudaStream_t s
 constexpr int CS_ROWS = 128;
 int64_t colsum_ws_floats(int64_t R, int32_t n, int32_t N) { return (cdiv(R, CS_ROWS) + n) * (int64_t)N + 64; }
 
+// One block per 128-row tile and per slab of 32 * V columns (V = elements of a 16-byte vector): lane l owns V adjacent
+// columns, warp w the tile's rows w, w + 8, ..., read with 16-byte loads, four rows in flight; the eight warps' sums are
+// added in warp order.
 template <typename XT>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const XT *__restrict__ in,
                                                              const int32_t *__restrict__ offsets, int32_t nseg,
                                                              int32_t N, const int32_t *__restrict__ tile_prefix,
                                                              float *__restrict__ part) {
+    constexpr int V = 16 / sizeof(XT);
+    __shared__ float sh[8][32 * V];
     const int32_t b = blockIdx.x;
     if (b >= tile_prefix[nseg]) return;
     int lo = 0, hi = nseg;
@@ -169,11 +174,43 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const XT *__restric
     }
     const int64_t r0 = offsets[lo] + (int64_t)(b - tile_prefix[lo]) * CS_ROWS;
     const int64_t r1 = min(r0 + (int64_t)CS_ROWS, (int64_t)offsets[lo + 1]);
-    const int32_t j = blockIdx.y * 256 + threadIdx.x;
-    if (j >= N) return;
-    float s = 0.0f;
-    for (int64_t r = r0; r < r1; ++r) s += to_f32(in[r * N + j]);
-    part[(int64_t)b * N + j] = s;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int32_t j = (blockIdx.y * 32 + lane) * V;
+    float s[V];
+#pragma unroll
+    for (int u = 0; u < V; ++u) s[u] = 0.0f;
+    if (j + V <= N) {  // N is a multiple of V wherever rows are 16-byte aligned
+        int64_t r = r0 + w;
+        for (; r + 24 < r1; r += 32) {
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const uint4 *>(in + (r + 8 * q) * N + j);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const XT *e = reinterpret_cast<const XT *>(&v[q]);
+#pragma unroll
+                for (int u = 0; u < V; ++u) s[u] += to_f32(e[u]);
+            }
+        }
+        for (; r < r1; r += 8) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(in + r * N + j);
+            const XT *e = reinterpret_cast<const XT *>(&v);
+#pragma unroll
+            for (int u = 0; u < V; ++u) s[u] += to_f32(e[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < V; ++u) sh[w][lane * V + u] = s[u];
+    __syncthreads();
+    for (int c = threadIdx.x; c < 32 * V; c += 256) {
+        const int32_t col = blockIdx.y * 32 * V + c;
+        if (col < N) {
+            float t = sh[0][c];
+#pragma unroll
+            for (int q = 1; q < 8; ++q) t += sh[q][c];
+            part[(int64_t)b * N + col] = t;
+        }
+    }
 }
 
 template <typename XT>
@@ -191,7 +228,8 @@ __global__ void __launch_bounds__(256) colsum_final_kernel(const float *__restri
 int32_t launch_segment_colsum(const void *in, int32_t act, const int32_t *offsets, int32_t nseg, int64_t R,
                               int32_t N, void *out, float *scratch, int32_t *tile_prefix, cudaStream_t st) {
     MOE_TRY(launch_tile_prefix(offsets, nseg, CS_ROWS, tile_prefix, st));
-    dim3 g1((unsigned)(cdiv(R, CS_ROWS) + nseg), (unsigned)cdiv(N, 256));
+    const int vcols = act == MOE_BF16 ? 256 : 128;  // columns per block of the partial sums: 32 lanes x one 16-byte vector
+    dim3 g1((unsigned)(cdiv(R, CS_ROWS) + nseg), (unsigned)cdiv(N, vcols));
     dim3 g2((unsigned)nseg, (unsigned)cdiv(N, 256));
     if (act == MOE_BF16) {
         colsum_partial_kernel<bf16><<<g1, 256, 0, st>>>((const bf16 *)in, offsets, nseg, N, tile_prefix, scratch);
