@@ -1491,7 +1491,10 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float *__res
 }
 
 bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
-    return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0;
+    // dX_gate contracts over the 2n logit columns (six split terms each) in one fp32 tensor-core accumulator, which
+    // truncates: beyond 2n = 4096 the result drifts past 1e-5 (measured 2e-5 at n = 8192), so very wide flat gates take
+    // the fp32 SIMT contractions instead
+    return act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0 && 2 * n <= 4096;
 }
 
 // dW of the gate: the contraction over the tokens is cut into row ranges (one float partial per range and precision

@@ -34,6 +34,8 @@ FLAT = [
     small_workload("screened-ragged-bf16", T=4100, d=128, h=64, n=32, k=2, act="bf16", seed=12),
     # SM-pair kernels with a heavily skewed load: one very long segment, short ones, (nearly) empty ones
     small_workload("skewed-long-bf16", T=4096, d=192, h=256, n=6, k=1, act="bf16", seed=11, skew="zipf", gamma=3.0),
+    # the largest expert count the ABI admits, the largest k: generic (any-n) paths of the gating, loss and routing kernels
+    small_workload("max-experts-bf16", T=600, d=64, h=64, n=8192, k=8, act="bf16", seed=13),
     synth.CONFIGS["c1"],
 ]
 
