@@ -5,6 +5,7 @@ indices and permutations bit-exact, fp32 gating tensors within 1e-5, expert-side
 1e-5 (fp32 layer) or 2e-2 max / 1e-2 mean (bf16 layer), in the rms-floored relative metric of
 helpers.rel_err.
 """
+import dataclasses
 import os
 
 import numpy as np
@@ -34,6 +35,8 @@ FLAT = [
     small_workload("screened-ragged-bf16", T=4100, d=128, h=64, n=32, k=2, act="bf16", seed=12),
     # SM-pair kernels with a heavily skewed load: one very long segment, short ones, (nearly) empty ones
     small_workload("skewed-long-bf16", T=4096, d=192, h=256, n=6, k=1, act="bf16", seed=11, skew="zipf", gamma=3.0),
+    # SM-pair kernels with a deep model width and a hidden width that is no multiple of the 256-column tile
+    small_workload("deep-d-bf16", T=2048, d=2048, h=192, n=4, k=2, act="bf16", seed=14),
     # the largest expert count the ABI admits, the largest k: generic (any-n) paths of the gating, loss and routing kernels
     small_workload("max-experts-bf16", T=600, d=64, h=64, n=8192, k=8, act="bf16", seed=13),
     synth.CONFIGS["c1"],
@@ -243,6 +246,26 @@ def test_losses_bwd_and_gate_bwd(case):
     assert_close(host(dWg), GB.dWg, TOL_F32, "dWg")
     assert_close(host(dWn), GB.dWnoise, TOL_F32, "dWnoise")
     assert_close(host(dXg), GB.dX_gate, TOL_F32, "dX_gate")
+
+
+@pytest.mark.parametrize("act", ["f32", "bf16"])
+def test_expert_stages_with_no_rows_give_zero_gradients(act):
+    """T = 0: every segment is empty; the weight and bias gradients must come out as exact zeros (both GEMM paths)."""
+    w = small_workload("no-rows", T=0, d=64, h=128, n=8, k=2, act=act)
+    cfg = cfg_of(w)
+    ws, S = ws_for(cfg)
+    I = synth.make_all(dataclasses.replace(w, T=4))
+    offsets = torch.zeros(w.n + 1, dtype=torch.int32, device="cuda")
+    one = lambda *shape: torch.full(shape, 7.0, dtype=torch.bfloat16 if act == "bf16" else torch.float32, device="cuda")
+    dW1, db1, dW2, db2 = one(w.n, w.d, w.h), one(w.n, w.h), one(w.n, w.h, w.d), one(w.n, w.d)
+    rows_d, rows_h = act_empty(w, 1, w.d), act_empty(w, 1, w.h)
+    B.moe_expert_ffn(cfg, rows_d, offsets, dev_act(I["W1"], w), dev_act(I["b1"], w), dev_act(I["W2"], w),
+                     dev_act(I["b2"], w), rows_h, act_empty(w, 1, w.d), ws)
+    B.moe_expert_ffn_bwd(cfg, rows_d, rows_h, act_empty(w, 1, w.d), offsets, dev_act(I["W1"], w), dev_act(I["W2"], w),
+                         act_empty(w, 1, w.d), dW1, db1, dW2, db2, ws)
+    assert B.moe_check_status(ws) == 0
+    for name, g in (("dW1", dW1), ("db1", db1), ("dW2", dW2), ("db2", db2)):
+        assert float(g.float().abs().max()) == 0.0, name
 
 
 def test_empty_batch():
