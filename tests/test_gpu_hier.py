@@ -21,6 +21,9 @@ HIER = [
     small_workload("hier-wide-bf16", T=777, d=128, h=64, n=96, k=6, a=3, k1=2, b=32, k2=3, act="bf16", seed=34),
     # both gating levels wide enough for the tensor-core gate backward (2a and 2b multiples of 64)
     small_workload("hier-tc-bf16", T=2100, d=64, h=64, n=1024, k=4, a=32, k1=2, b=32, k2=2, act="bf16", seed=35),
+    # few tokens over many groups: some groups get no token at all (|X^(i)| = 0: zero Load_H row, zero gradients)
+    small_workload("hier-empty-groups-f32", T=40, d=32, h=16, n=128, k=4, a=32, k1=2, b=4, k2=2, seed=38),
+    small_workload("hier-empty-groups-bf16", T=48, d=64, h=64, n=1024, k=4, a=32, k1=2, b=32, k2=2, act="bf16", seed=39),
     # primary gate wide enough for the routing screen, secondary gates too narrow for it
     small_workload("hier-primary-screen-bf16", T=1024, d=64, h=64, n=256, k=4, a=32, k1=2, b=8, k2=2, act="bf16", seed=37),
 ]
@@ -40,6 +43,12 @@ def case(request):
     I = synth.make_all(w)
     F, Bk = oracle_run(w, I)
     return w, I, F, Bk, device_inputs(w, I), cfg_of(w)
+
+
+def test_the_empty_group_cases_do_have_empty_groups(case):
+    w, I, F, _, D, cfg = case
+    if "empty-groups" in w.name:
+        assert (np.asarray(F.LS.cnt) == 0).any()
 
 
 def test_hier_gate(case):
