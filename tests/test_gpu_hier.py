@@ -161,3 +161,29 @@ def test_hier_secondary_ties_take_every_column_through_the_chain():
     assert (host(idx) == want["topk_idx"]).all()
     assert (host(ki) == want["kth_idx"]).all()
     assert_close(host(gates), want["gates"], TOL_F32, "gates")
+
+
+def test_hier_screened_routing_equals_pure_chain_routing():
+    """Both gating levels screened on the tensor cores against every slot through the fma chain (c4's shape, 8192 tokens):
+    the flat expert ids and both levels' k-th / (k+1)-th indices must be identical."""
+    import os
+    from dataclasses import replace
+    for seed in range(3):
+        w = replace(synth.CONFIGS["c4"], T=8192, seed=synth.BASE_SEED + 700 + seed, name=f"c4-seed{seed}")
+        cfg = cfg_of(w)
+        S = B.moe_query_sizes(cfg)
+        x = dev_act(synth.make_x(w), w)
+        Wg, Wn, noise = [dev(cat_parts(a)) for a in synth.make_gate(w)]
+        out = []
+        for screen in ("1", "0"):
+            os.environ["MOE_GATE_SCREEN"] = screen
+            ws = B.empty_bytes(B.moe_query_sizes(cfg).ws_bytes)
+            idx, gates = i32(w.T, w.k), f32(S.gates_elems)
+            clean, raw = f32(S.logits_elems), f32(S.logits_elems)
+            kv, ki = f32(S.kth_elems), i32(S.kth_elems)
+            B.moe_gate(cfg, x, Wg, Wn, noise, idx, gates, clean, raw, kv, ki, ws)
+            assert B.moe_check_status(ws) == 0
+            out.append((idx, ki, gates))
+        os.environ["MOE_GATE_SCREEN"] = "1"
+        assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
+        assert_close(host(out[0][2]), host(out[1][2]), TOL_F32, "gates")

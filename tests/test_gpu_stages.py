@@ -156,6 +156,37 @@ def test_screened_routing_equals_pure_chain_routing_on_many_batches():
         assert_close(host(out[0][3]), host(out[1][3]), TOL_F32, "clean")
 
 
+def test_screened_routing_equals_pure_chain_routing_on_badly_scaled_inputs():
+    """The same property where the screen's error model is stressed: features and weight rows spanning six orders of
+    magnitude, heavy-tailed activations, large noise, cancelling logits (so the intervals are wide against the gaps)."""
+    from dataclasses import replace
+    base = replace(synth.CONFIGS["c5"], T=8192, skew="none")
+    for seed in range(4):
+        w = replace(base, seed=synth.BASE_SEED + 600 + seed, name=f"c5-rough{seed}")
+        rng = np.random.default_rng(900 + seed)
+        x = synth.make_x(w).astype(np.float32)
+        Wg, Wn, noise = [np.array(a, np.float32) for a in synth.make_gate(w)]
+        scale = (10.0 ** rng.uniform(-3, 3, size=w.d)).astype(np.float32)
+        x = x * scale * (1.0 + 5.0 * (rng.random(x.shape) < 0.01))          # per-feature scales, 1 % outliers
+        Wg = Wg / scale[:, None]; Wn = Wn / scale[:, None]                    # logits stay O(1): sums of huge and tiny terms
+        if seed & 1:
+            Wg[:, 1::2] = Wg[:, 0::2] * (1.0 + 1e-7)                          # near-duplicate experts
+        noise = noise * 4.0
+        cfg = cfg_of(w)
+        ws, S = ws_for(cfg)
+        xd, Wgd, Wnd, nd = dev_act(x, w), dev(Wg), dev(Wn), dev(noise)
+        out = []
+        for screen in ("1", "0"):
+            os.environ["MOE_GATE_SCREEN"] = screen
+            idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
+            kv, ki = f32(w.T, 2), i32(w.T, 2)
+            B.moe_gate(cfg, xd, Wgd, Wnd, nd, idx, gates, clean, raw, kv, ki, ws)
+            assert B.moe_check_status(ws) == 0
+            out.append((idx, ki))
+        os.environ["MOE_GATE_SCREEN"] = "1"
+        assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
+
+
 def test_dispatch(case):
     w, I, F, _, D, cfg = case
     ws, S = ws_for(cfg)
