@@ -37,6 +37,8 @@ FLAT = [
     small_workload("skewed-long-bf16", T=4096, d=192, h=256, n=6, k=1, act="bf16", seed=11, skew="zipf", gamma=3.0),
     # SM-pair kernels with a deep model width and a hidden width that is no multiple of the 256-column tile
     small_workload("deep-d-bf16", T=2048, d=2048, h=192, n=4, k=2, act="bf16", seed=14),
+    # a single expert: one long segment, every tile but the last is full
+    small_workload("one-expert-bf16", T=5000, d=64, h=128, n=1, k=1, act="bf16", seed=15),
     # the largest expert count the ABI admits, the largest k: generic (any-n) paths of the gating, loss and routing kernels
     small_workload("max-experts-bf16", T=600, d=64, h=64, n=8192, k=8, act="bf16", seed=13),
     synth.CONFIGS["c1"],
