@@ -98,3 +98,15 @@ def test_fused_is_deterministic():
     a, b = run_fused(w, I), run_fused(w, I)
     for name in ("y", "losses", "importance", "load", "dX", "dWg", "dWnoise", "dW1", "db1", "dW2", "db2"):
         assert torch.equal(a[name], b[name]), name
+
+
+def test_two_runs_give_bitwise_identical_results():
+    """Nothing in the path depends on timing: the tile order is static, sums are taken in fixed orders, the lists of
+    uncertain tokens are only worked through element by element. Two runs on the same inputs must agree bit for bit."""
+    w = synth.CONFIGS["c3"].scaled(8192)
+    I = synth.make_all(w)
+    a, b = run_fused(w, I), run_fused(w, I)
+    for name in ("y", "losses", "importance", "load", "counts", "dX", "dWg", "dWnoise", "dW1", "db1", "dW2", "db2"):
+        assert torch.equal(a[name], b[name]), name
+    for name in ("topk_idx", "gates", "clean", "raw_noise", "hid", "ys"):
+        assert torch.equal(a["ctx"][name], b["ctx"][name]), name
