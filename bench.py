@@ -100,7 +100,8 @@ def run_reference(args, w):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    Ts = cpu_sample_tokens(w, 5.0e11)  # a few seconds per step, so that K + W steps end within minutes
+    # the oracle does about 25 GFLOP/s on these hosts: size a step so that K timed steps + 1 warm-up take about two minutes
+    Ts = cpu_sample_tokens(w, min(1.0e12, 3.0e12 / (args.steps + 1)))
     ws, I = host_inputs_sample(w, Ts)
     for _ in range(min(args.warmup, 1)):
         oracle_step(ws, I)
