@@ -1549,14 +1549,17 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
         CUtensorMap tmA, tmB;
+        const bool pairs = T >= 256 * 74 && getenv("MOE_TC_ONE_CTA") == nullptr;  // enough 256-row tiles for every SM pair
         MOE_TRY(map_rows_kmajor(&tmA, dsplit, T, 3 * n2));
-        MOE_TRY(map_weight_kmajor(&tmB, wsplit, 1, d, 3 * n2));
+        if (pairs) MOE_TRY(map_weight_kmajor_half(&tmB, wsplit, 1, d, 3 * n2));
+        else MOE_TRY(map_weight_kmajor(&tmB, wsplit, 1, d, 3 * n2));
         GemmParams p = default_params();
         p.nseg = 1; p.N = d; p.K = n2; p.R = T; p.out_f32 = dX_gate; p.status = status;
         p.nterms = 6;
         const int32_t at[6] = {2, 0, 1, 0, 1, 0}, bt[6] = {0, 2, 1, 1, 0, 0};  // smallest products first
         for (int i = 0; i < 6; ++i) { p.a_term_col[i] = at[i] * n2; p.b_term_col[i] = bt[i] * n2; }
-        MOE_TRY(launch<ROW_BK>(tmA, tmB, p, cdiv(T, BM) * cdiv(d, BN), st));
+        if (pairs) MOE_TRY(launch2<ROW_BK>(tmA, tmB, p, cdiv(T, 256) * cdiv(d, BN), st));
+        else MOE_TRY(launch<ROW_BK>(tmA, tmB, p, cdiv(T, BM) * cdiv(d, BN), st));
     }
     return MOE_OK;
 }
