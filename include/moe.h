@@ -34,6 +34,10 @@
  *     load         : [a*b] Load_H, then [a] primary Load, [a,b] per-group Load_i(X^(i)), [a] |X^(i)|
  *     dload        : [a] d/d(primary Load), then [a,b] d/d(per-group Load)
  * moe_query_sizes gives the element counts.
+ *
+ * Every call only enqueues work on the given stream: no host synchronisation, no allocation, no device-to-host read.
+ * After one eager call per process and device (function attributes are set on first use) the calls may be recorded
+ * in a CUDA graph by stream capture.
  */
 #ifndef MOE_B200_H
 #define MOE_B200_H

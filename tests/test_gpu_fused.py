@@ -110,3 +110,39 @@ def test_two_runs_give_bitwise_identical_results():
         assert torch.equal(a[name], b[name]), name
     for name in ("topk_idx", "gates", "clean", "raw_noise", "hid", "ys"):
         assert torch.equal(a["ctx"][name], b["ctx"][name]), name
+
+
+def test_the_fused_calls_can_be_captured_in_a_cuda_graph():
+    """moe_forward + moe_backward only enqueue work on the caller's stream (no synchronisation, no allocation), so a
+    stream capture records them; replaying the graph must reproduce the eager results bit for bit."""
+    w = synth.CONFIGS["c2"]
+    I = synth.make_all(w)
+    cfg = cfg_of(w)
+    S = B.moe_query_sizes(cfg)
+    D = device_inputs(w, I)
+    ctx, ws = B.empty_bytes(S.ctx_bytes), B.empty_bytes(max(S.ws_fwd_bytes, S.ws_bwd_bytes))
+    out = dict(y=act_empty(w, w.T, w.d), losses=f32(2), imp=f32(w.n), load=f32(S.load_elems), counts=i32(w.n),
+               dX=act_empty(w, w.T, w.d), dWg=f32(S.wg_elems), dWn=f32(S.wg_elems), dW1=act_empty(w, w.n, w.d, w.h),
+               db1=act_empty(w, w.n, w.h), dW2=act_empty(w, w.n, w.h, w.d), db2=act_empty(w, w.n, w.d))
+
+    def step():
+        B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], out["y"],
+                      out["losses"], out["imp"], out["load"], out["counts"], ctx, ws)
+        B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], ctx,
+                       out["dX"], out["dWg"], out["dWn"], out["dW1"], out["db1"], out["dW2"], out["db2"], ws)
+
+    step()  # eager: also the first-call set-up (function attributes, driver entry points)
+    torch.cuda.synchronize()
+    eager = {k: v.clone() for k, v in out.items()}
+    for v in out.values():
+        v.zero_()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for v in out.values():
+        v.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert B.moe_check_status(ws) == 0
+    for k in out:
+        assert torch.equal(out[k], eager[k]), k
