@@ -69,7 +69,16 @@ typedef struct moe_config {
     int32_t a, k1, b, k2;       /* hierarchical levels; a = 0 selects the flat layer (k1, b, k2 ignored) */
     int32_t act;                /* moe_dtype of the "act" tensors                                        */
     float w_importance, w_load; /* scale factors of Eq. 7 and Eq. 11                                     */
+    int32_t flags;              /* 0, or an OR of the MOE_FLAG_* switches below                          */
 } moe_config;
+
+/* Switches in moe_config.flags (0 = the library chooses by problem size):
+ *   MOE_FLAG_GATE_SCREEN_OFF  every token's routing logits through the fixed fma chain (no tensor-core screen)
+ *   MOE_FLAG_GATE_SCREEN_ON   screen the routing on the tensor cores whenever the shapes allow, however small
+ *   MOE_FLAG_TC_ONE_CTA       one-CTA tensor-core GEMM kernels everywhere (no SM pairs), for A/B comparisons */
+#define MOE_FLAG_GATE_SCREEN_OFF 1
+#define MOE_FLAG_GATE_SCREEN_ON 2
+#define MOE_FLAG_TC_ONE_CTA 4
 
 typedef struct moe_sizes {
     int64_t R;            /* T*k                                                                    */
@@ -133,7 +142,8 @@ int32_t moe_check_status(const void *ws, void *stream);
  * 1e-7 of it). For every other token the columns that can still reach rank k+1 are re-evaluated
  * with the chain and the selection is repeated, so its indices are the chain's too; its other
  * columns keep the tensor-core values.
- * Environment: MOE_GATE_SCREEN=0 disables the screen, =1 uses it whenever the shapes allow.
+ * moe_config.flags: MOE_FLAG_GATE_SCREEN_OFF disables the screen, MOE_FLAG_GATE_SCREEN_ON uses it whenever the
+ * shapes allow; by default it is used when the projection has at least 1e9 multiply-adds.
  * `noise` is an input: standard normal draws, or zeros for noiseless gating.
  * in : x [T,d] act, Wg/Wnoise [d,n], noise [T,n]
  * out: topk_idx [T,k], gates [T,k], clean [T,n], raw_noise [T,n], kth_vals [T,2], kth_idx [T,2] */

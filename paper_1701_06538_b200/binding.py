@@ -16,6 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmoe_b200.so")
 
 MOE_F32, MOE_BF16 = 0, 1
+MOE_FLAG_GATE_SCREEN_OFF, MOE_FLAG_GATE_SCREEN_ON, MOE_FLAG_TC_ONE_CTA = 1, 2, 4
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED", 3: "MOE_ERR_WORKSPACE",
                 4: "MOE_ERR_CUDA", 5: "MOE_ERR_TIMEOUT"}
 
@@ -33,7 +34,7 @@ class MoeError(RuntimeError):
 
 class moe_config(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int32) for name in ("T", "d", "h", "n", "k", "a", "k1", "b", "k2", "act")] + \
-               [("w_importance", ctypes.c_float), ("w_load", ctypes.c_float)]
+               [("w_importance", ctypes.c_float), ("w_load", ctypes.c_float), ("flags", ctypes.c_int32)]
 
 
 class moe_sizes(ctypes.Structure):
@@ -67,9 +68,9 @@ def lib():
     return _lib
 
 
-def make_config(T, d, h, n, k, act, w_importance=0.1, w_load=0.1, a=0, k1=0, b=0, k2=0) -> moe_config:
+def make_config(T, d, h, n, k, act, w_importance=0.1, w_load=0.1, a=0, k1=0, b=0, k2=0, flags=0) -> moe_config:
     act_id = {"f32": MOE_F32, "bf16": MOE_BF16}.get(act, act)
-    return moe_config(T, d, h, n, k, a, k1, b, k2, act_id, w_importance, w_load)
+    return moe_config(T, d, h, n, k, a, k1, b, k2, act_id, w_importance, w_load, flags)
 
 
 def act_dtype(cfg: moe_config):

@@ -17,7 +17,7 @@ struct Dims {
     bool hier;
     int64_t a, k1, b, k2;
     int64_t gate_cols, logits, gates, kth, wg, load, dload;
-    int32_t act;
+    int32_t act, flags;
     size_t esz;
 };
 
@@ -40,6 +40,8 @@ int32_t check_config(const moe_config *c) {
         return MOE_ERR_INVALID_ARG;
     }
     if (!(c->w_importance >= 0.0f) || !(c->w_load >= 0.0f)) return MOE_ERR_INVALID_ARG;
+    if (c->flags & ~(MOE_FLAG_GATE_SCREEN_OFF | MOE_FLAG_GATE_SCREEN_ON | MOE_FLAG_TC_ONE_CTA)) return MOE_ERR_INVALID_ARG;
+    if ((c->flags & MOE_FLAG_GATE_SCREEN_OFF) && (c->flags & MOE_FLAG_GATE_SCREEN_ON)) return MOE_ERR_INVALID_ARG;
     return MOE_OK;
 }
 
@@ -50,6 +52,7 @@ Dims dims_of(const moe_config *c) {
     D.hier = c->a > 0;
     D.a = c->a; D.k1 = c->k1; D.b = c->b; D.k2 = c->k2;
     D.act = c->act;
+    D.flags = c->flags;
     D.esz = act_bytes(c->act);
     if (D.hier) {
         D.gate_cols = D.a + D.k1 * D.b;
@@ -107,7 +110,7 @@ struct GateWs {
         idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
         cr = wnorm = xnorm = wt = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = full_list = nullptr; chain_list = nullptr;
         const int64_t n1 = D.hier ? D.a : D.n;  // width of the (first) gate
-        screen = tc_gate_fwd_supported(D.act, D.T, (int32_t)D.d, (int32_t)n1);
+        screen = tc_gate_fwd_supported(D.act, D.T, (int32_t)D.d, (int32_t)n1, D.flags);
         if (screen) {
             cr = cv.take<float>(D.T * 2 * n1);
             wsplit = cv.take<bf16>(3 * D.d * 2 * n1);
@@ -129,7 +132,7 @@ struct GateWs {
         scratch = cv.take<int32_t>(dispatch_ws_elems(D.T * D.k1, (int32_t)D.a));
         tile_prefix = cv.take<int32_t>(tc_tile_ws_ints(D.T * D.k1, D.a));  // prefix + tile table of the grouped product
         const int64_t P1 = D.T * D.k1;
-        screen2 = tc_gate_fwd_supported(D.act, P1, (int32_t)D.d, (int32_t)D.b);
+        screen2 = tc_gate_fwd_supported(D.act, P1, (int32_t)D.d, (int32_t)D.b, D.flags);
         if (screen2) {
             if (!xnorm) xnorm = cv.take<float>(D.T);
             xs_p = cv.take_bytes(P1 * D.d * (int64_t)D.esz);
@@ -346,7 +349,7 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
         MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, (int32_t)D.b, Wg_s, Wn_s, w.wsplit_s, w.wnorm_s,
                                            w.xnorm, w.unsafe_count_s, w.wt_s, st, (int32_t)D.a, !w.screen));
         MOE_TRY(launch_tc_gate_fwd_grouped(w.xs_p, P1, (int32_t)D.d, (int32_t)D.a, (int32_t)D.b, w.wsplit_s, w.offsets_p,
-                                           w.tile_prefix, w.cr_s, status_word(ws_base), st));
+                                           w.tile_prefix, w.cr_s, status_word(ws_base), st, D.flags));
         MOE_TRY(launch_gate_screen(w.cr_s, noise + lp, w.xnorm, w.wnorm_s, (int32_t)D.d, P1, (int32_t)D.b, (int32_t)D.k2,
                                    w.idx_s, g_s, clean + lp, raw_noise + lp, kth_vals + 2 * D.T, kth_idx + 2 * D.T,
                                    w.unsafe_list_s, w.unsafe_count_s, w.chain_list_s, nullptr, st, w.perm_p,
@@ -511,7 +514,7 @@ int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const flo
                                             nullptr, D.T, (int32_t)D.a, (int32_t)D.k1, nullptr, nullptr, w.dsplit,
                                             nullptr, st));
             MOE_TRY(launch_tc_gate_bwd(x, D.T, (int32_t)D.d, (int32_t)D.a, Wg, Wnoise, w.dsplit, w.wsplit, w.partials,
-                                       dWg, dWnoise, dX_gate, status_word(ws_base), st));
+                                       dWg, dWnoise, dX_gate, status_word(ws_base), st, D.flags));
             MOE_TRY(launch_gate_logit_grads(noise + lp, clean + lp, raw_noise + lp, w.H.idx_s, g_s, kth_vals + 2 * D.T,
                                             kth_idx + 2 * D.T, dg_s, dload + D.a, w.H.idx_p, P1, (int32_t)D.b,
                                             (int32_t)D.k2, nullptr, nullptr, w.dsplit_s, w.H.inv_perm_p, st));
@@ -560,7 +563,7 @@ int32_t do_gate_bwd(const moe_config *c, const Dims &D, const void *x, const flo
                                     st));
     if (w.tc)
         return launch_tc_gate_bwd(x, D.T, (int32_t)D.d, (int32_t)D.n, Wg, Wnoise, w.dsplit, w.wsplit, w.partials, dWg,
-                                  dWnoise, dX_gate, status_word(ws_base), st);
+                                  dWnoise, dX_gate, status_word(ws_base), st, D.flags);
     MOE_TRY(gate_weight_grads(D, x, w.dclean, Wg, D.n, dWg, dX_gate, false, st));
     return gate_weight_grads(D, x, w.draw, Wnoise, D.n, dWnoise, dX_gate, true, st);
 }

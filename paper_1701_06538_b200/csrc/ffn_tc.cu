@@ -1260,9 +1260,8 @@ int64_t tc_tile_ws_ints(int64_t R, int64_t nseg);
 int64_t tc_ffn_ws_bytes(const moe_config &c) { return (tc_tile_ws_ints((int64_t)c.T * c.k, c.n) * 4 + 255) & ~255ll; }
 
 // The 256-row tiles of the two-CTA kernel pay off when the average segment fills them.
-static bool use_two_cta(int64_t R, int32_t nseg) {
-    const char *env = getenv("MOE_TC_ONE_CTA");
-    if (env && env[0] == '1') return false;
+static bool use_two_cta(int64_t R, int32_t nseg, int32_t flags) {
+    if (flags & MOE_FLAG_TC_ONE_CTA) return false;
     return R / (nseg > 0 ? nseg : 1) >= 384;
 }
 
@@ -1378,8 +1377,8 @@ int64_t tc_colsum_part_floats(int64_t R, int32_t nseg, int32_t N) { return (cdiv
 // and reduced into colsum_out [nseg, N]; colsum_part needs tc_colsum_part_floats(R, nseg, N) floats
 int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t *offsets, int32_t nseg, int64_t R,
                     int32_t N, int32_t K, void *out, const void *bias, const void *mask, int relu,
-                    int32_t *tile_prefix, int32_t *status, cudaStream_t st, float *colsum_part = nullptr,
-                    void *colsum_out = nullptr) {
+                    int32_t *tile_prefix, int32_t *status, cudaStream_t st, int32_t flags,
+                    float *colsum_part = nullptr, void *colsum_out = nullptr) {
     if (R == 0) {
         if (colsum_out) MOE_CUDA(cudaMemsetAsync(colsum_out, 0, sizeof(bf16) * (size_t)nseg * N, st));
         return MOE_OK;
@@ -1398,7 +1397,7 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
     p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
     p.colsum_part = colsum_out ? colsum_part : nullptr;
-    if (use_two_cta(R, nseg)) {  // segments long enough to fill 256-row tiles: SM pairs
+    if (use_two_cta(R, nseg, flags)) {  // segments long enough to fill 256-row tiles: SM pairs
         if (transposed) MOE_TRY(map_weight_kmajor_half(&tmB, W, nseg, N, K));
         else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
         MOE_TRY(launch_tile_table(offsets, nseg, 256, R, tile_prefix, st));
@@ -1427,12 +1426,12 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
 
 // dW[e] [M, N] = A_e^T . B_e, contraction over the rows of segment e; A [R, M], B [R, N]
 int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int32_t nseg, int64_t R, int32_t M,
-                      int32_t N, void *out, int32_t *status, cudaStream_t st) {
+                      int32_t N, void *out, int32_t *status, cudaStream_t st, int32_t flags) {
     CUtensorMap tmA, tmB;
     GemmParams p = default_params();
     p.offsets = offsets; p.nseg = nseg; p.M = M; p.N = N; p.R = R;
     p.out = (bf16 *)out; p.status = status;
-    if (use_two_cta(R, nseg) && M >= 256) {  // SM pairs: 256 x 256 tiles, each CTA stages half of A and half of B
+    if (use_two_cta(R, nseg, flags) && M >= 256) {  // SM pairs: 256 x 256 tiles, each CTA stages half of A and half of B
         MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, 2));
         MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, 2));
         return launch2<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, 256) * cdiv(N, BN), st);
@@ -1447,8 +1446,8 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
                       cudaStream_t st) {
     const int64_t R = (int64_t)c.T * c.k;
     int32_t *tile_prefix = static_cast<int32_t *>(ws);
-    MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st));
-    return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st);
+    MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st, c.flags));
+    return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1523,7 +1522,7 @@ int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n) {
 
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
-                           float *dX_gate, int32_t *status, cudaStream_t st) {
+                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags) {
     const int32_t n2 = 2 * n;
     if (T == 0) {
         MOE_CUDA(cudaMemsetAsync(dWg, 0, sizeof(float) * d * n, st));
@@ -1549,7 +1548,7 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
         CUtensorMap tmA, tmB;
-        const bool pairs = T >= 256 * 74 && getenv("MOE_TC_ONE_CTA") == nullptr;  // enough 256-row tiles for every SM pair
+        const bool pairs = T >= 256 * 74 && !(flags & MOE_FLAG_TC_ONE_CTA);  // enough 256-row tiles for every SM pair
         MOE_TRY(map_rows_kmajor(&tmA, dsplit, T, 3 * n2));
         if (pairs) MOE_TRY(map_weight_kmajor_half(&tmB, wsplit, 1, d, 3 * n2));
         else MOE_TRY(map_weight_kmajor(&tmB, wsplit, 1, d, 3 * n2));
@@ -1565,13 +1564,12 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
 }
 
 // Forward gate projection for the routing screen: cr = x . (W_lo + W_mid + W_hi), smallest term first.
-bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n) {
-    // MOE_GATE_SCREEN=0: every token through the fma chain; =1: screen whenever the shapes allow;
-    // unset: screen when the projection is large enough to pay for the extra launches
-    const char *env = getenv("MOE_GATE_SCREEN");
-    if (env && env[0] == '0') return false;
+bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n, int32_t flags) {
+    // MOE_FLAG_GATE_SCREEN_OFF: every token through the fma chain; _ON: screen whenever the shapes allow;
+    // neither: screen when the projection is large enough to pay for the extra launches
+    if (flags & MOE_FLAG_GATE_SCREEN_OFF) return false;
     if (!(act == MOE_BF16 && d % 64 == 0 && (2 * n) % 64 == 0 && T >= 256)) return false;
-    if (env && env[0] == '1') return true;
+    if (flags & MOE_FLAG_GATE_SCREEN_ON) return true;
     return (double)T * d * 2.0 * n >= 1.0e9;
 }
 
@@ -1593,10 +1591,10 @@ int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const
 // cr_s [P1, 2b] comes out in sorted order.
 int32_t launch_tc_gate_fwd_grouped(const void *xs_p, int64_t P1, int32_t d, int32_t a, int32_t b, const void *wsplit_s,
                                    const int32_t *offsets_p, int32_t *tile_prefix, float *cr_s, int32_t *status,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, int32_t flags) {
     if (P1 == 0) return MOE_OK;
     const int32_t n2 = 2 * b;
-    const bool pairs = use_two_cta(P1, a);
+    const bool pairs = use_two_cta(P1, a, flags);
     CUtensorMap tmA, tmB;
     MOE_TRY(map_rows_kmajor(&tmA, xs_p, P1, d));
     {   // the group is the map's last coordinate (stride d rows), the precision term an offset of a * d rows along K
@@ -1664,11 +1662,11 @@ int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, 
                           cudaStream_t st) {
     const int64_t R = (int64_t)c.T * c.k;
     MOE_TRY(launch_segment_colsum(dys, c.act, offsets, c.n, R, c.d, db2, colsum, tile_prefix, st));
-    MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st));
+    MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st, c.flags));
     // db1 = column sums of dz, formed in the epilogue of the GEMM that produces dz
-    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, colsum, db1));
-    MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st));
-    return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st);
+    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, c.flags, colsum, db1));
+    MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st, c.flags));
+    return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
 
 }  // namespace moe

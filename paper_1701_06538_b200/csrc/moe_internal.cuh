@@ -89,7 +89,7 @@ constexpr int SCREEN_MAX_CAND = 16;
 int32_t launch_gate_chains(const void *x, int32_t act, int32_t d, int32_t n, const float *Wt, const void *chain_list,
                            const int32_t *chain_count, float *clean, float *raw, cudaStream_t st,
                            int32_t kdiv = 1);  // Wt [2n, d] (per group); token = output row / kdiv
-bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n);
+bool tc_gate_fwd_supported(int32_t act, int64_t T, int32_t d, int32_t n, int32_t flags);
 // cr [T, 2n] (float) = x . [W_g | W_noise] from the three-term split wsplit [3, d, 2n]
 int32_t launch_tc_gate_fwd(const void *x, int64_t T, int32_t d, int32_t n, const void *wsplit, float *cr,
                            int32_t *status, cudaStream_t st);
@@ -200,10 +200,10 @@ bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n);
 int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n);  // floats of partial-sum scratch
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
-                           float *dX_gate, int32_t *status, cudaStream_t st);
+                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags);
 int32_t launch_tc_gate_fwd_grouped(const void *xs_p, int64_t P1, int32_t d, int32_t a, int32_t b, const void *wsplit_s,
                                    const int32_t *offsets_p, int32_t *tile_prefix, float *cr_s, int32_t *status,
-                                   cudaStream_t st);
+                                   cudaStream_t st, int32_t flags);
 bool tc_hier_gate_bwd_supported(int32_t act, int32_t d, int32_t a, int32_t b);
 int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, void *wsplit_s, const float *Wg_s,
                                      const float *Wn_s, const int32_t *offsets_p, int32_t *tile_prefix, int32_t a,

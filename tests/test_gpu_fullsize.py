@@ -6,9 +6,13 @@ The oracle cannot run the expert GEMMs of these batches in reasonable time, so:
     handles the whole batch;
   - expert-side outputs are compared on samples the oracle computes one by one: y and dX of sampled
     tokens (each token's experts are evaluated on that token alone, which is exact because the
-    experts act row by row), and the complete weight / bias gradients of two small experts
-    (every row of those experts is evaluated);
-  - the gate backward is compared in full through its stage call, fed with the oracle's gate state.
+    experts act row by row), the complete weight / bias gradients of two small experts (every row
+    of those experts is evaluated), and, for the LARGEST expert (the longest contraction the weight-gradient
+    GEMMs see), the gradients of a sample of its hidden units spread over every 256-wide tile: the expert
+    restricted to those units is itself a one-hidden-layer expert whose hid, dW1[:, J], db1[J], dW2[J, :]
+    and db2 are exactly the full expert's slices, so the oracle evaluates that smaller network on all rows;
+  - the gate backward is compared in full through its stage call, fed with the oracle's gate state
+    (flat and hierarchical).
 """
 import numpy as np
 import pytest
@@ -25,6 +29,8 @@ from test_gpu_hier import gate_tensors
 pytestmark = pytest.mark.gpu
 
 N_TOKENS = 48
+MAX_FLIP_RATE = 2e-5   # share of ReLU decisions that may differ (pre-activation within rounding of zero)
+UNITS_PER_TILE = 16    # hidden units of the largest expert sampled in every 256-wide tile
 
 
 def slice_gate(G, rows):
@@ -99,47 +105,77 @@ def test_full_size_fused(name):
     got_hid = host(V["hid"][torch.from_numpy(Dp.inv_perm.reshape(w.T, w.k)[toks].reshape(-1).astype(np.int64)).cuda()])
     want_hid = np.asarray(hid)[Ds.inv_perm]
     assert_close(got_hid, want_hid, TOL_BF16, "hid (sampled rows)")
-    clean_rows = ((got_hid > 0) == (want_hid > 0)).reshape(len(toks), -1).all(axis=1)  # no ReLU decision at rounding of 0
-    assert clean_rows.mean() > 0.5
+    flips = (got_hid > 0) != (want_hid > 0)   # ReLU decisions within rounding of 0: rare, and their tokens set aside
+    assert flips.sum() <= max(2, MAX_FLIP_RATE * flips.size), int(flips.sum())
+    clean_rows = ~flips.reshape(len(toks), -1).any(axis=1)
     assert_close(host(D["dX"])[toks][clean_rows], dX[clean_rows], TOL_BF16, "dX (sampled tokens)")
 
-    # ---------------- two small non-empty experts: their complete weight and bias gradients
+    # ---------------- experts: two small ones and an empty one in full, the largest one on sampled hidden units
     order = np.argsort(Dp.counts, kind="stable")
     small = [int(e) for e in order if Dp.counts[e] > 0][:2]
-    for e in small + [int(e) for e in order if Dp.counts[e] == 0][:1]:
+    largest = int(np.argmax(Dp.counts))
+    gu = np.random.default_rng(9)
+    units_big = np.unique(np.concatenate([np.concatenate([[c0, c0 + 255], c0 + gu.choice(256, UNITS_PER_TILE - 2, False)])
+                                          for c0 in range(0, w.h, 256)]))
+    for e, units in [(e, None) for e in small + [int(e) for e in order if Dp.counts[e] == 0][:1]] + [(largest, units_big)]:
         got = {k2: host(D[k2][e]) for k2 in ("dW1", "db1", "dW2", "db2")}
         if Dp.counts[e] == 0:
             assert all(np.abs(v).max() == 0 for v in got.values()), "an expert without rows has zero gradients"
             continue
         slots = Dp.perm[Dp.offsets[e]:Dp.offsets[e + 1]]
         t_e, s_e = slots // w.k, slots % w.k
-        We = synth.make_expert(w, e)
+        W1e, b1e, W2e, b2e = synth.make_expert(w, e)
+        if units is None:
+            units = np.arange(w.h)
+        W1e, b1e, W2e = W1e[:, units], b1e[units], W2e[units, :]   # the expert restricted to these hidden units
         offs = np.array([0, len(slots)], np.int32)
-        hid_e, _ = O.expert_ffn(x[t_e], offs, We[0][None], We[1][None], We[2][None], We[3][None], "bf16")
+        hid_e, _ = O.expert_ffn(x[t_e], offs, W1e[None], b1e[None], W2e[None], b2e[None], "bf16")
         dys_e = O.store(np.asarray(G.gates, np.float64)[t_e, s_e][:, None] * dY[t_e].astype(np.float64), "bf16", True)
-        Ee = O.expert_ffn_bwd(x[t_e], hid_e, dys_e, offs, We[0][None], We[2][None], "bf16")
-        got_hid_e = host(V["hid"][int(Dp.offsets[e]):int(Dp.offsets[e + 1])])
-        keep_cols = ((got_hid_e > 0) == (np.asarray(hid_e) > 0)).all(axis=0)
-        assert keep_cols.mean() > 0.9
-        assert_close(got["dW2"], Ee.dW2[0], TOL_BF16, f"dW2[{e}]")
+        Ee = O.expert_ffn_bwd(x[t_e], hid_e, dys_e, offs, W1e[None], W2e[None], "bf16")
+        got_hid_e = host(V["hid"][int(Dp.offsets[e]):int(Dp.offsets[e + 1])])[:, units]
+        assert_close(got_hid_e, hid_e, TOL_BF16, f"hid[{e}]")
+        flips_e = (got_hid_e > 0) != (np.asarray(hid_e) > 0)
+        assert flips_e.sum() <= max(2, MAX_FLIP_RATE * flips_e.size), (e, int(flips_e.sum()))
+        keep_cols = ~flips_e.any(axis=0)
+        assert_close(got["dW2"][units, :], Ee.dW2[0], TOL_BF16, f"dW2[{e}]")
         assert_close(got["db2"], Ee.db2[0], TOL_BF16, f"db2[{e}]")
-        assert_close(got["dW1"][:, keep_cols], Ee.dW1[0][:, keep_cols], TOL_BF16, f"dW1[{e}]")
-        assert_close(got["db1"][keep_cols], Ee.db1[0][keep_cols], TOL_BF16, f"db1[{e}]")
+        assert_close(got["dW1"][:, units][:, keep_cols], Ee.dW1[0][:, keep_cols], TOL_BF16, f"dW1[{e}]")
+        assert_close(got["db1"][units][keep_cols], Ee.db1[0][keep_cols], TOL_BF16, f"db1[{e}]")
 
     # ---------------- gate backward in full, through its stage call, fed with the oracle's gate state
+    gd = np.random.default_rng(8)
+    dgates = gd.standard_normal((w.T, w.k)).astype(np.float32)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    dWg, dWn, dXg_d = f32(S.wg_elems), f32(S.wg_elems), f32(w.T, w.d)
     if hier is None:
-        gd = np.random.default_rng(8)
-        dgates = gd.standard_normal((w.T, w.k)).astype(np.float32)
         dload = (gd.standard_normal(w.n) * 1e-3).astype(np.float32)
         GBf = O.gate_bwd(x, Wg, Wn, noise, G.clean, G.raw, G.idx, G.gates, G.kth_val, G.kth_idx, dgates, dload, "bf16")
-        dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
-        dWg, dWn, dXg_d = f32(w.d, w.n), f32(w.d, w.n), f32(w.T, w.d)
         B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], dev(G.clean), dev(G.raw), dev(G.idx),
                        dev(G.gates), dev(G.kth_val), dev(G.kth_idx), dev(dgates), dev(dload), dWg, dWn, dXg_d, D["ws"])
-        assert B.moe_check_status(D["ws"]) == 0
-        assert_close(host(dWg), GBf.dWg, TOL_F32, "dWg (full)")
-        assert_close(host(dWn), GBf.dWnoise, TOL_F32, "dWnoise (full)")
-        # The uneven-load workloads route a constant feature through W_g[0, :] with offsets up to ~4 while
-        # sum_j dclean_j ~ 0: that column of dX_gate is a cancelling sum, and fp32 accumulation (any order)
-        # leaves ~1e-5 of the result there; the mean error stays at the 1e-7 level.
-        assert_close(host(dXg_d), GBf.dX_gate, dict(max=5e-5, mean=1e-6), "dX_gate (full)")
+        want_dWg, want_dWn, want_dXg = GBf.dWg, GBf.dWnoise, GBf.dX_gate
+    else:
+        # both levels: the upstream gradients of the stage call are the oracle's own (product-gate gradient with the
+        # Importance term added, d/dLoad of both levels from Eq. 14), so the gate backward is compared alone
+        a_, b_ = w.a, w.b
+        dI = w.w_importance * O.cv_squared_grad(LS.importance)
+        dLH = (w.w_load * O.cv_squared_grad(LS.load)).reshape(a_, b_)
+        safe = np.where(LS.cnt > 0, LS.cnt, 1.0)
+        live = (LS.cnt > 0)[:, None]
+        dload = np.concatenate([np.where(live, dLH * LS.load_s / safe[:, None], 0).sum(1),
+                                np.where(live, dLH * LS.load_p[:, None] / safe[:, None], 0).reshape(-1)]).astype(np.float32)
+        GBh = O.gate_h_bwd(x, Wg[0], Wn[0], noise[0], Wg[1], Wn[1], noise[1], G, LS, dgates, w.w_importance, w.w_load,
+                           "bf16")
+        dg = torch.zeros(S.gates_elems, device="cuda")
+        dg[:w.T * w.k] = dev((dgates.astype(np.float64) + dI[G.idx]).astype(np.float32)).reshape(-1)
+        B.moe_gate_bwd(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], dev(GT["clean"]), dev(GT["raw"]),
+                       dev(GT["topk_idx"]), dev(GT["gates"]), dev(GT["kth_vals"]), dev(GT["kth_idx"]), dg, dev(dload),
+                       dWg, dWn, dXg_d, D["ws"])
+        want_dWg, want_dWn = cat_parts((GBh.dWg_p, GBh.dWg_s)), cat_parts((GBh.dWn_p, GBh.dWn_s))
+        want_dXg = GBh.dX_gate
+    assert B.moe_check_status(D["ws"]) == 0
+    assert_close(host(dWg), want_dWg, TOL_F32, "dWg (full)")
+    assert_close(host(dWn), want_dWn, TOL_F32, "dWnoise (full)")
+    # The uneven-load workloads route a constant feature through W_g[0, :] with offsets up to ~4 while
+    # sum_j dclean_j ~ 0: that column of dX_gate is a cancelling sum, and fp32 accumulation (any order)
+    # leaves ~1e-5 of the result there; the mean error stays at the 1e-7 level.
+    assert_close(host(dXg_d), want_dXg, dict(max=5e-5, mean=1e-6), "dX_gate (full)")
