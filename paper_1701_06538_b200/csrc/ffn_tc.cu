@@ -41,7 +41,7 @@ constexpr int EPI_STAGE_BYTES = 8 * 4096;  // per epilogue warp: a 32 x 128 B sl
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_STAGE_BYTES;
 constexpr int TMEM_COLS = 512;
 constexpr int NTHREADS = 320;   // TMA warp, MMA warp, 8 epilogue warps
-constexpr int NTHREADS2 = 352;  // two-CTA kernel: + one warp that fixes the ragged K tail of the wgrad ahead of the MMAs
+constexpr int NTHREADS2 = 384;  // two-CTA kernel: + one warp that fixes the ragged K tail of the wgrad ahead of the MMAs, + the tile scheduler warp
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Kind { ROW_BMN = 0, ROW_BK = 1, WGRAD = 2 };
@@ -81,7 +81,28 @@ struct GemmParams {
     // columns a_term_col[i] + [0, K) and B columns b_term_col[i] + [0, K)
     int32_t nterms;
     int32_t a_term_col[MAX_TERMS], b_term_col[MAX_TERMS];
+    // two-CTA kernels over ragged segments: tiles are handed out at run time (see PairTiles). sched_counter = next tile
+    // id; sched_table[id / sched_group] = {segment, first row, end row, 0} (segment -1: no more tiles). WGRAD: the
+    // segments in descending size, sched_group = tiles per segment; ROW_*: tile_info, sched_group = N tiles per M tile
+    const int4 *sched_table;
+    int32_t *sched_counter;
+    int32_t sched_group;
+    int32_t trace;  // diagnostics build only: this launch records the tile trace
 };
+
+// Diagnostics build (-DMOE_TILE_TRACE): the first CTA records, per tile, when each warp role started, finished and how
+// long it waited; read back with moe_debug_tile_trace. Compiled out otherwise.
+#ifdef MOE_TILE_TRACE
+__device__ long long g_tile_trace[3][256][4];
+#define TILE_TRACE_SET(role, tile, field, val) do { if (p.trace && blockIdx.x == 0 && (tile) < 256) g_tile_trace[role][tile][field] = (val); } while (0)
+#define TILE_TRACE_ADD(role, tile, field, val) do { if (p.trace && blockIdx.x == 0 && (tile) < 256) g_tile_trace[role][tile][field] += (val); } while (0)
+#define TILE_CLOCK() clock64()
+static int g_trace_launch_no = 0;
+#else
+#define TILE_TRACE_SET(role, tile, field, val) do {} while (0)
+#define TILE_TRACE_ADD(role, tile, field, val) do {} while (0)
+#define TILE_CLOCK() 0ll
+#endif
 
 // ------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -658,7 +679,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 constexpr int STAGES2 = 6;
 constexpr int A2_BYTES = 128 * BK * 2, B2_BYTES = 128 * BK * 2, STAGE2_BYTES = A2_BYTES + B2_BYTES;
 constexpr int DATA2_BYTES = STAGES2 * STAGE2_BYTES + EPI_STAGE_BYTES;  // 224 KiB: 6 stages + float staging, or 5 stages + mask tile
-constexpr int SMEM2_BYTES = DATA2_BYTES + 1024 + 256;
+constexpr int SMEM2_BYTES = DATA2_BYTES + 1024 + 512;  // + alignment slack, barriers, scheduler ring
 constexpr uint32_t PEER_BIT_MASK = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address of the pair
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -720,6 +741,72 @@ __host__ __device__ constexpr uint32_t make_idesc2(int a_mn, int b_mn) {  // M 2
            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
+// Tile source of the two-CTA kernel. Static mode: ids dealt round-robin to the pairs (TileIter). Dynamic mode (ragged
+// segments): a fixed deal leaves pairs idle at the end, because the tiles of a weight-gradient GEMM differ in length by
+// the ratio of the largest to the smallest expert, and because SM pairs do not all run at the same speed (distance to
+// the L2 slices, the two dies). The scheduler warp of the even CTA draws tile ids from a global counter (WGRAD: in
+// descending order of segment size, longest first) and publishes one 16-byte record per tile {segment, first row,
+// end row, tile id} in a four-slot ring in the shared memory of BOTH CTAs; every warp role of both CTAs reads the
+// same sequence of records. A record with segment -1 ends the sequence. Which pair computes a tile does not change
+// the tile's result, so the output stays bit-reproducible.
+constexpr int SCHED_SLOTS = 4;
+__device__ __forceinline__ uint32_t peer_smem_addr(uint32_t addr, uint32_t cta) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, const int4 &v) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster_addr(uint32_t cluster_addr) {  // release at cluster scope
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+template <int KIND> struct PairTiles {
+    const GemmParams &p;
+    TileIter<KIND, 256> fixed;
+    const bool dyn, warp_wide, arrives;
+    const uint32_t ring, full0, empty0;
+    volatile int *abort_flag;
+    int i;
+    // warp_wide: all 32 lanes of the warp call next() together; arrives: this thread reports the slot as read
+    __device__ __forceinline__ PairTiles(const GemmParams &p_, bool dyn_, int32_t first, int32_t stride, uint32_t ring_,
+                                         uint32_t full0_, uint32_t empty0_, volatile int *abort_, bool warp_wide_, bool arrives_)
+        : p(p_), fixed(p_, dyn_ ? p_.total_tiles : first, stride), dyn(dyn_), warp_wide(warp_wide_), arrives(arrives_),
+          ring(ring_), full0(full0_), empty0(empty0_), abort_flag(abort_), i(0) {}
+    __device__ __forceinline__ bool next(Tile &t) {
+        if (!dyn) return fixed.next(t);
+        const int slot = i & (SCHED_SLOTS - 1);
+        const uint32_t par = (uint32_t)(i / SCHED_SLOTS) & 1u;
+        if (!mbar_wait(full0 + 8u * slot, par, abort_flag, p.status)) return false;
+        mbar_try_wait_cluster(full0 + 8u * slot, par);  // acquire at cluster scope: the record came from the other CTA's thread
+        int4 rec;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rec.x), "=r"(rec.y), "=r"(rec.z), "=r"(rec.w)
+                     : "r"(ring + 16u * slot) : "memory");
+        if (warp_wide) __syncwarp();  // every lane has its copy before the slot is reported as read
+        if (arrives) mbar_arrive_leader_relaxed(empty0 + 8u * slot);
+        ++i;
+        if (rec.x < 0) return false;
+        t.e = rec.x; t.row0 = rec.y; t.row_end = rec.z;
+        const int32_t grp = rec.w / p.sched_group, rem = rec.w - grp * p.sched_group;  // rec.w: the tile id
+        if (KIND == WGRAD) {
+            const int32_t tm = rem / p.tiles_n;
+            t.mt = 0;
+            t.m0 = tm * 256;
+            t.n0 = (rem - tm * p.tiles_n) * BN;
+            t.b_chunk = t.n0 / 64;
+            t.kblocks = (t.row_end - t.row0 + BK - 1) / BK;
+        } else {
+            t.mt = grp;
+            t.m0 = 0;
+            t.b_chunk = 0;
+            t.n0 = rem * BN;
+            t.kblocks = p.kblocks_row;
+        }
+        return true;
+    }
+};
+
 // MASKT: the ReLU mask of the dgrad GEMM is not read row by row from global memory by the epilogue but
 // fetched as a 128 x 256 tile by TMA (one stage fewer in exchange for the 64 KiB it occupies).
 template <int KIND, bool MASKT>
@@ -743,6 +830,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     auto afull_bar = [&](int s) { return bars + 8u * (2 * NST + 4 + s); };
     auto ready_bar = [&](int s) { return bars + 8u * (3 * NST + 4 + s); };
     const uint32_t mfull_bar = bars + 8u * 28, mempty_bar = bars + 8u * 29;  // mask tile landed / read by all 8 epilogue warps
+    // dynamic tile scheduling (WGRAD): record published / record read by every role of both CTAs (barrier in the even CTA)
+    const uint32_t sched_full0 = bars + 256, sched_empty0 = bars + 256 + 8u * SCHED_SLOTS, sched_ring = bars + 384;
+    const bool dyn = p.sched_counter != nullptr;
     const uint32_t mask_smem = base + NST * STAGE2_BYTES;                     // 4 blocks of [128 rows][64 columns], 128-B swizzle
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + DATA2_BYTES + 240);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + DATA2_BYTES + 248);
@@ -758,6 +848,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 16); }
         mbar_init(mfull_bar, 1); mbar_init(mempty_bar, 8);
+        // readers of a scheduler record: producer, 8 epilogue warps (WGRAD: + tail warp) in each CTA, the MMA thread in the even one
+        for (int q = 0; q < SCHED_SLOTS; ++q) { mbar_init(sched_full0 + 8u * q, 1); mbar_init(sched_empty0 + 8u * q, KIND == WGRAD ? 21 : 19); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
@@ -795,7 +887,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int s = 0;
             uint32_t ph = 0, mask_ph = 0;
             bool ok = true;
-            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            PairTiles<KIND> it(p, dyn, (int32_t)cluster_id, (int32_t)n_clusters, sched_ring, sched_full0, sched_empty0, abort_flag, false, true);
             Tile t;
             // MASKT: the mask tile of a row tile can only land after the epilogue has read the previous one, which
             // happens while the next tile's K blocks are already being loaded: the load stays "due" and is issued
@@ -816,12 +908,19 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 mask_due = false;
                 return true;
             };
+            int trace_tile = -1;
             while (ok && it.next(t)) {
                 int term = 0, kk = 0;  // ROW_*: piece of the contraction and column inside it
+                ++trace_tile;
+                TILE_TRACE_SET(0, trace_tile, 1, 0);
                 for (int kb = 0; kb < t.kblocks && ok; ++kb) {
                     if (MASKT && mask_due) load_mask(false);
+                    const long long tw0 = TILE_CLOCK();
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
+                    TILE_TRACE_ADD(0, trace_tile, 1, TILE_CLOCK() - tw0);
+                    if (kb == 0) TILE_TRACE_SET(0, trace_tile, 0, TILE_CLOCK());
+                    if (kb == t.kblocks - 1) TILE_TRACE_SET(0, trace_tile, 2, TILE_CLOCK());
                     const uint32_t a_dst = base + s * STAGE2_BYTES, b_dst = a_dst + A2_BYTES;
                     if (KIND == WGRAD) {
                         const int r = t.row0 + kb * BK;
@@ -857,48 +956,83 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even CTA only)
-        if (rank == 0) {
+        // One thread runs the whole loop: nothing in it needs the other lanes, and a single-thread loop has no
+        // divergence / reconvergence around the issue of every K block.
+        if (rank == 0 && lane == 0) {
             constexpr uint32_t idesc = make_idesc2(KIND == WGRAD ? 1 : 0, KIND == ROW_BK ? 0 : 1);
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0, tail_ph = 0;  // tail_ph: one phase bit per stage for afull / ready
             bool ok = true;
-            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            PairTiles<KIND> it(p, dyn, (int32_t)cluster_id, (int32_t)n_clusters, sched_ring, sched_full0, sched_empty0, abort_flag, false, true);
             Tile t;
+            int trace_tile = -1;
             while (ok && it.next(t)) {
+                ++trace_tile;
                 if (t.kblocks == 0) continue;  // empty segment (WGRAD): the epilogue writes zeros
+                TILE_TRACE_SET(1, trace_tile, 0, TILE_CLOCK());
                 ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
+                TILE_TRACE_SET(1, trace_tile, 1, TILE_CLOCK());
+                TILE_TRACE_SET(1, trace_tile, 2, 0);
                 const uint32_t d_tmem = tmem_base + acc * BN;
+                const int tail_valid = KIND == WGRAD ? (t.row_end - t.row0) - (t.kblocks - 1) * BK : BK;  // rows of the last block
                 for (int kb = 0; kb < t.kblocks; ++kb) {
-                    if (KIND == WGRAD) {
-                        const int valid = t.row_end - (t.row0 + kb * BK);
-                        if (valid < BK) {
-                            const uint32_t tp = (tail_ph >> s) & 1u;  // fixed by warp 10 of both CTAs, ahead of time
-                            ok = mbar_wait(ready_bar(s), tp, abort_flag, p.status) && mbar_try_wait_cluster(ready_bar(s), tp);
-                            if (!ok) break;
-                            tail_ph ^= 1u << s;
-                        }
+                    if (KIND == WGRAD && kb == t.kblocks - 1 && tail_valid < BK) {
+                        const uint32_t tp = (tail_ph >> s) & 1u;  // fixed by warp 10 of both CTAs, ahead of time
+                        ok = mbar_wait(ready_bar(s), tp, abort_flag, p.status) && mbar_try_wait_cluster(ready_bar(s), tp);
+                        if (!ok) break;
+                        tail_ph ^= 1u << s;
                     }
+                    const long long tw0 = TILE_CLOCK();
                     ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
+                    TILE_TRACE_ADD(1, trace_tile, 2, TILE_CLOCK() - tw0);
                     const uint32_t a_src = base + s * STAGE2_BYTES, b_src = a_src + A2_BYTES;
-                    if (lane == 0) {
+                    const long long ti0 = TILE_CLOCK();
+                    const uint64_t ad0 = KIND == WGRAD ? desc_mnmajor(a_src) : desc_kmajor(a_src);
+                    const uint64_t bd0 = KIND == ROW_BK ? desc_kmajor(b_src) : desc_mnmajor(b_src);
+                    // a K step of 16 advances the start address (low descriptor bits, in 16-byte units) by 32 bytes in a
+                    // K-major tile and by 16 rows of 128 bytes in an MN-major one; the sum never leaves the address field
+                    constexpr uint64_t a_step = KIND == WGRAD ? (16 * 128) >> 4 : 32 >> 4;
+                    constexpr uint64_t b_step = KIND == ROW_BK ? 32 >> 4 : (16 * 128) >> 4;
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k) {
-                            const uint64_t ad = KIND == WGRAD ? desc_mnmajor(a_src + k * 16 * 128) : desc_kmajor(a_src + k * 32);
-                            const uint64_t bd = KIND == ROW_BK ? desc_kmajor(b_src + k * 32) : desc_mnmajor(b_src + k * 16 * 128);
-                            tc_mma2_bf16(d_tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                        }
-                        tc_commit2(empty_bar(s));
-                    }
-                    __syncwarp();
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma2_bf16(d_tmem, ad0 + k * a_step, bd0 + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    tc_commit2(empty_bar(s));
+                    if (kb == 0) TILE_TRACE_SET(0, trace_tile, 3, 0);
+                    TILE_TRACE_ADD(0, trace_tile, 3, TILE_CLOCK() - ti0);
                     if (++s == NST) { s = 0; ph ^= 1u; }
                 }
-                if (ok && lane == 0) tc_commit2(tfull_bar(acc));
-                __syncwarp();
+                if (ok) tc_commit2(tfull_bar(acc));
+                TILE_TRACE_SET(1, trace_tile, 3, TILE_CLOCK());
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    } else if (warp == 11) {
+        // ------------------------------------------------------------------ tile scheduler (even CTA, one thread)
+        if (dyn && rank == 0 && lane == 0) {
+            const uint32_t peer_ring = peer_smem_addr(sched_ring, 1), peer_full0 = peer_smem_addr(sched_full0, 1);
+            bool ok = true;
+            for (int i = 0; ok; ++i) {
+                const int slot = i & (SCHED_SLOTS - 1);
+                if (i >= SCHED_SLOTS) {  // every reader of the record this slot held has its copy
+                    const uint32_t par = (uint32_t)(i / SCHED_SLOTS - 1) & 1u;
+                    ok = mbar_wait(sched_empty0 + 8u * slot, par, abort_flag, p.status) && mbar_try_wait_cluster(sched_empty0 + 8u * slot, par);
+                    if (!ok) break;
+                }
+                const int32_t id = atomicAdd(p.sched_counter, 1);
+                int4 rec = make_int4(-1, 0, 0, 0);
+                if (id < p.total_tiles) {
+                    rec = p.sched_table[id / p.sched_group];
+                    rec.w = id;
+                }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sched_ring + 16u * slot), "r"(rec.x), "r"(rec.y), "r"(rec.z), "r"(rec.w) : "memory");
+                st_cluster_v4(peer_ring + 16u * slot, rec);
+                mbar_arrive(sched_full0 + 8u * slot);
+                mbar_arrive_cluster_addr(peer_full0 + 8u * slot);
+                if (rec.x < 0) break;
             }
         }
     } else if (warp == 10) {
@@ -909,7 +1043,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int s = 0;
             uint32_t tail_ph = 0;
             bool ok = true;
-            TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+            PairTiles<KIND> it(p, dyn, (int32_t)cluster_id, (int32_t)n_clusters, sched_ring, sched_full0, sched_empty0, abort_flag, true, lane == 0);
             Tile t;
             while (ok && it.next(t)) {
                 for (int kb = 0; kb < t.kblocks; ++kb) {
@@ -934,15 +1068,19 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
-        TileIter<KIND, 256> it(p, (int32_t)cluster_id, (int32_t)n_clusters);
+        PairTiles<KIND> it(p, dyn, (int32_t)cluster_id, (int32_t)n_clusters, sched_ring, sched_full0, sched_empty0, abort_flag, true, lane == 0);
         Tile t;
+        int trace_tile = -1;
         while (ok && it.next(t)) {
             const bool have_acc = t.kblocks > 0;
+            ++trace_tile;
+            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 0, TILE_CLOCK());
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
             }
+            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 1, TILE_CLOCK());
             int64_t tile_row0, out_off = 0;
             int32_t rows_valid;
             if (KIND == WGRAD) {
@@ -975,8 +1113,13 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (col0 >= p.N) break;
                 uint32_t v[32];
                 if (have_acc) {
+                    const long long tl0 = TILE_CLOCK();
                     tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
                     tc_ld_wait();
+                    if (warp == 2 && lane == 0) {
+                        if (c == half * (BN / 64)) TILE_TRACE_SET(2, trace_tile, 3, 0);
+                        TILE_TRACE_ADD(2, trace_tile, 3, TILE_CLOCK() - tl0);
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
@@ -1064,6 +1207,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (lane == 0) mbar_arrive_leader_relaxed(tempty_bar(acc));
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
+            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 2, TILE_CLOCK());
             if (MASKT) {  // the next mask tile may land once this warp's boxes have been read out
                 __syncwarp();
                 if (lane == 0) {
@@ -1244,6 +1388,13 @@ int32_t launch2(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams
         max_clusters = n;
     }
     if (max_tiles <= 0) return MOE_OK;
+#ifdef MOE_TILE_TRACE
+    {   // the launch whose index (counted over the two-CTA launches of the process) equals MOE_TRACE_LAUNCH records
+        const char *env = getenv("MOE_TRACE_LAUNCH");
+        p.trace = env && atoi(env) == g_trace_launch_no;
+        ++g_trace_launch_no;
+    }
+#endif
     cfg.gridDim = dim3(2 * (unsigned)imin(max_tiles, max_clusters));
     MOE_CUDA(cudaLaunchKernelEx(&cfg, grouped_gemm2_kernel<KIND, MASKT>, tmA, tmB, tmM ? *tmM : tmA, tmO ? *tmO : tmA, p));
     MOE_LAUNCHED();
@@ -1272,7 +1423,7 @@ static bool use_two_cta(int64_t R, int32_t nseg, int32_t flags) {
 // the last tile carry segment -1. One block.
 __global__ void __launch_bounds__(1024) tile_table_kernel(const int32_t *__restrict__ offsets, int32_t n, int32_t tm,
                                                           int32_t max_m, int32_t *__restrict__ tile_prefix,
-                                                          int4 *__restrict__ info) {
+                                                          int4 *__restrict__ info, int32_t *__restrict__ counter) {
     __shared__ int32_t warp_sum[32];
     __shared__ int32_t carry;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -1307,6 +1458,7 @@ __global__ void __launch_bounds__(1024) tile_table_kernel(const int32_t *__restr
         __syncthreads();
     }
     if (threadIdx.x == 0) tile_prefix[n] = carry;
+    if (threadIdx.x == 0 && counter) *counter = 0;  // run-time tile counter of the GEMM that follows
     __syncthreads();  // the prefix (global memory, this block's own writes) is complete
     const int32_t total = carry;
     for (int32_t mt = threadIdx.x; mt < max_m; mt += 1024) {
@@ -1325,10 +1477,14 @@ int64_t tc_tile_ws_ints(int64_t R, int64_t nseg) { return ((nseg + 1 + 3) & ~(in
 static int4 *tile_info_of(int32_t *tile_prefix, int32_t nseg) {
     return reinterpret_cast<int4 *>(tile_prefix + ((nseg + 1 + 3) & ~3));
 }
+// the int32 behind the last record of a table of tm = 256-row tiles (the table is sized for 128-row tiles)
+static int32_t *tile_counter_of(int32_t *tile_prefix, int32_t nseg, int64_t R) {
+    return reinterpret_cast<int32_t *>(tile_info_of(tile_prefix, nseg) + cdiv(R, 256) + nseg);
+}
 static int32_t launch_tile_table(const int32_t *offsets, int32_t nseg, int32_t tm, int64_t R, int32_t *tile_prefix,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, int32_t *counter = nullptr) {
     tile_table_kernel<<<1, 1024, 0, st>>>(offsets, nseg, tm, (int32_t)(cdiv(R, tm) + nseg), tile_prefix,
-                                          tile_info_of(tile_prefix, nseg));
+                                          tile_info_of(tile_prefix, nseg), counter);
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -1400,7 +1556,10 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     if (use_two_cta(R, nseg, flags)) {  // segments long enough to fill 256-row tiles: SM pairs
         if (transposed) MOE_TRY(map_weight_kmajor_half(&tmB, W, nseg, N, K));
         else MOE_TRY(map_weight_mnmajor_half(&tmB, W, nseg, K, N));
-        MOE_TRY(launch_tile_table(offsets, nseg, 256, R, tile_prefix, st));
+        p.sched_counter = tile_counter_of(tile_prefix, nseg, R);  // tiles handed out at run time
+        p.sched_table = p.tile_info;
+        p.sched_group = (int32_t)cdiv(N, BN);
+        MOE_TRY(launch_tile_table(offsets, nseg, 256, R, tile_prefix, st, p.sched_counter));
         const int64_t max_tiles2 = (cdiv(R, 256) + nseg) * cdiv(N, BN);
         CUtensorMap tmO;  // output rows as [32][64] boxes
         {
@@ -1424,9 +1583,27 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     return finish(transposed ? launch<ROW_BK>(tmA, tmB, p, max_tiles, st) : launch<ROW_BMN>(tmA, tmB, p, max_tiles, st), 4);
 }
 
-// dW[e] [M, N] = A_e^T . B_e, contraction over the rows of segment e; A [R, M], B [R, N]
+// Order in which the two-CTA weight-gradient GEMM hands out its tiles: seg[r] = {e, first row, end row, 0} for the
+// segment of rank r by descending size (equal sizes by index), and the tile counter reset. One thread per segment.
+constexpr int SCHED_MAX_SEG = 8192;
+__global__ void __launch_bounds__(256) wgrad_schedule_kernel(const int32_t *__restrict__ offsets, int32_t n,
+                                                             int4 *__restrict__ seg, int32_t *__restrict__ counter) {
+    __shared__ int32_t cnt[SCHED_MAX_SEG];
+    for (int32_t e = threadIdx.x; e < n; e += blockDim.x) cnt[e] = offsets[e + 1] - offsets[e];
+    __syncthreads();
+    const int32_t e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e == 0) *counter = 0;
+    if (e >= n) return;
+    const int32_t mine = cnt[e];
+    int32_t rank = 0;
+    for (int32_t o = 0; o < n; ++o) rank += (cnt[o] > mine || (cnt[o] == mine && o < e)) ? 1 : 0;
+    seg[rank] = make_int4(e, offsets[e], offsets[e + 1], 0);
+}
+
+// dW[e] [M, N] = A_e^T . B_e, contraction over the rows of segment e; A [R, M], B [R, N].
+// sched_ws: 4 + 4 * nseg ints (16-byte aligned) for the run-time tile order of the two-CTA kernel, or nullptr.
 int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int32_t nseg, int64_t R, int32_t M,
-                      int32_t N, void *out, int32_t *status, cudaStream_t st, int32_t flags) {
+                      int32_t N, void *out, int32_t *status, cudaStream_t st, int32_t flags, int32_t *sched_ws) {
     CUtensorMap tmA, tmB;
     GemmParams p = default_params();
     p.offsets = offsets; p.nseg = nseg; p.M = M; p.N = N; p.R = R;
@@ -1434,6 +1611,14 @@ int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int3
     if (use_two_cta(R, nseg, flags) && M >= 256) {  // SM pairs: 256 x 256 tiles, each CTA stages half of A and half of B
         MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, 2));
         MOE_TRY(map_rows_mnmajor(&tmB, B, R > 0 ? R : 1, N, 2));
+        if (sched_ws && nseg > 1 && nseg <= SCHED_MAX_SEG) {  // tiles of unequal length: longest first, handed out at run time
+            p.sched_counter = sched_ws;
+            p.sched_table = reinterpret_cast<const int4 *>(sched_ws + 4);
+            p.sched_group = (int32_t)(cdiv(M, 256) * cdiv(N, BN));
+            wgrad_schedule_kernel<<<(unsigned)cdiv(nseg, 256), 256, 0, st>>>(offsets, nseg, reinterpret_cast<int4 *>(sched_ws + 4),
+                                                                          sched_ws);
+            MOE_LAUNCHED();
+        }
         return launch2<WGRAD>(tmA, tmB, p, (int64_t)nseg * cdiv(M, 256) * cdiv(N, BN), st);
     }
     MOE_TRY(map_rows_mnmajor(&tmA, A, R > 0 ? R : 1, M, BM / 64));
@@ -1662,11 +1847,17 @@ int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, 
                           cudaStream_t st) {
     const int64_t R = (int64_t)c.T * c.k;
     MOE_TRY(launch_segment_colsum(dys, c.act, offsets, c.n, R, c.d, db2, colsum, tile_prefix, st));
-    MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st, c.flags));
+    MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st, c.flags, tile_prefix));
     // db1 = column sums of dz, formed in the epilogue of the GEMM that produces dz
     MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, c.flags, colsum, db1));
-    MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st, c.flags));
+    MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st, c.flags, tile_prefix));
     return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
 
 }  // namespace moe
+
+#ifdef MOE_TILE_TRACE
+extern "C" int32_t moe_debug_tile_trace(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, moe::g_tile_trace, sizeof(moe::g_tile_trace)) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+#endif

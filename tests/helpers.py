@@ -40,8 +40,28 @@ def tol_act(w):
     return TOL_BF16 if w.act == "bf16" else TOL_F32
 
 
-def cfg_of(w):
-    return B.make_config(w.T, w.d, w.h, w.n, w.k, w.act, w.w_importance, w.w_load, w.a, w.k1, w.b, w.k2)
+SCREEN_ON, SCREEN_OFF = B.MOE_FLAG_GATE_SCREEN_ON, B.MOE_FLAG_GATE_SCREEN_OFF
+
+
+def cfg_of(w, flags=0):
+    """flags = 0 is what a user (and bench.py) gets: the library chooses its kernels by problem size."""
+    return B.make_config(w.T, w.d, w.h, w.n, w.k, w.act, w.w_importance, w.w_load, w.a, w.k1, w.b, w.k2, flags)
+
+
+def screened(w, flags=SCREEN_ON):
+    """True where moe_gate screens the routing on the tensor cores: bf16, widths that are multiples of 64, and
+    either forced (MOE_FLAG_GATE_SCREEN_ON) or a projection of at least 1e9 multiply-adds."""
+    if flags & SCREEN_OFF:
+        return False
+
+    def level(rows, width):
+        ok = w.act == "bf16" and rows >= 256 and w.d % 64 == 0 and (2 * width) % 64 == 0
+        return ok and (bool(flags & SCREEN_ON) or float(rows) * w.d * 2.0 * width >= 1.0e9)
+
+    first = level(w.T, w.a if w.a else w.n)
+    # the secondary gates of the hierarchical layer are screened on their own (rows = T * k1 slots, width b)
+    second = bool(w.a) and level(w.T * w.k1, w.b)
+    return first or second
 
 
 def cat_parts(parts):

@@ -6,8 +6,8 @@ import torch
 from paper_1701_06538_b200 import binding as B
 from paper_1701_06538_b200 import synth
 
-from helpers import (TOL_F32, act_empty, assert_close, assert_expert_backward_close, cat_parts, cfg_of,
-                     device_inputs, f32, host, i32, oracle_run, small_workload, tol_act)
+from helpers import (SCREEN_ON, TOL_F32, act_empty, assert_close, assert_expert_backward_close, cat_parts, cfg_of,
+                     device_inputs, f32, host, i32, oracle_run, screened, small_workload, tol_act)
 
 pytestmark = pytest.mark.gpu
 
@@ -20,8 +20,8 @@ CASES = [
 ]
 
 
-def run_fused(w, I):
-    cfg = cfg_of(w)
+def run_fused(w, I, flags=0):
+    cfg = cfg_of(w, flags)
     S = B.moe_query_sizes(cfg)
     D = device_inputs(w, I)
     ctx = B.empty_bytes(S.ctx_bytes)
@@ -43,11 +43,25 @@ def run_fused(w, I):
                 db1=db1, dW2=dW2, db2=db2, ctx=V)
 
 
+_ORACLE = {}
+
+
+def oracle_cached(w):
+    if w.name not in _ORACLE:
+        I = synth.make_all(w)
+        _ORACLE[w.name] = (I,) + tuple(oracle_run(w, I))
+    return _ORACLE[w.name]
+
+
+# flags 0: the kernels the library picks by itself (what bench.py runs); SCREEN_ON: the routing screen forced on
+# for these small shapes (it only applies to bf16 layers whose widths are multiples of 64)
+@pytest.mark.parametrize("flags", [0, SCREEN_ON], ids=["default", "screen-on"])
 @pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
-def test_fused_forward_backward(w):
-    I = synth.make_all(w)
-    F, Bk = oracle_run(w, I)
-    G = run_fused(w, I)
+def test_fused_forward_backward(w, flags):
+    if flags and not screened(w, flags):
+        pytest.skip("the routing screen does not apply to this shape")
+    I, F, Bk = oracle_cached(w)
+    G = run_fused(w, I, flags)
     V = G["ctx"]
     # routing: bit-exact
     assert (host(V["topk_idx"]) == F.G.idx).all()

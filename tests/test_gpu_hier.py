@@ -7,10 +7,8 @@ from oracle import moe_oracle as O
 from paper_1701_06538_b200 import binding as B
 from paper_1701_06538_b200 import synth
 
-from helpers import (TOL_F32, act_empty, assert_close, assert_expert_backward_close, cat_parts, cfg_of, dev,
-                     dev_act, device_inputs, f32, host, i32, oracle_run, prec_of, small_workload, tol_act)
-
-from test_gpu_stages import screened
+from helpers import (SCREEN_OFF, SCREEN_ON, TOL_F32, act_empty, assert_close, assert_expert_backward_close, cat_parts, cfg_of, dev,
+                     dev_act, device_inputs, f32, host, i32, oracle_run, prec_of, screened, small_workload, tol_act)
 
 pytestmark = pytest.mark.gpu
 
@@ -42,7 +40,7 @@ def case(request):
     w = request.param
     I = synth.make_all(w)
     F, Bk = oracle_run(w, I)
-    return w, I, F, Bk, device_inputs(w, I), cfg_of(w)
+    return w, I, F, Bk, device_inputs(w, I), cfg_of(w, SCREEN_ON)
 
 
 def test_the_empty_group_cases_do_have_empty_groups(case):
@@ -111,10 +109,13 @@ def test_hier_losses_and_backward_stages(case):
     assert_close(host(dXg), GB.dX_gate, tol, "dX_gate")
 
 
-def test_hier_fused(case):
+@pytest.mark.parametrize("flags", [0, SCREEN_ON], ids=["default", "screen-on"])
+def test_hier_fused(case, flags):
     from test_gpu_fused import run_fused
     w, I, F, Bk, D, cfg = case
-    G = run_fused(w, I)
+    if flags and not screened(w, flags):
+        pytest.skip("the routing screen does not apply to this shape")
+    G = run_fused(w, I, flags)
     V = G["ctx"]
     want = gate_tensors(F.G)
     assert (host(V["topk_idx"]) == F.G.idx).all()
@@ -146,7 +147,7 @@ def test_hier_secondary_ties_take_every_column_through_the_chain():
     n_s[:] = 0.0
     assert screened(w)
     F, _ = oracle_run(w, I, backward=False)
-    D, cfg = device_inputs(w, I), cfg_of(w)
+    D, cfg = device_inputs(w, I), cfg_of(w, SCREEN_ON)
     S = B.moe_query_sizes(cfg)
     ws = B.empty_bytes(S.ws_bytes)
     idx, gates = i32(w.T, w.k), f32(S.gates_elems)
@@ -165,24 +166,21 @@ def test_hier_secondary_ties_take_every_column_through_the_chain():
 def test_hier_screened_routing_equals_pure_chain_routing():
     """Both gating levels screened on the tensor cores against every slot through the fma chain (c4's shape, 8192 tokens):
     the flat expert ids and both levels' k-th / (k+1)-th indices must be identical."""
-    import os
     from dataclasses import replace
     for seed in range(3):
         w = replace(synth.CONFIGS["c4"], T=8192, seed=synth.BASE_SEED + 700 + seed, name=f"c4-seed{seed}")
-        cfg = cfg_of(w)
-        S = B.moe_query_sizes(cfg)
         x = dev_act(synth.make_x(w), w)
         Wg, Wn, noise = [dev(cat_parts(a)) for a in synth.make_gate(w)]
         out = []
-        for screen in ("1", "0"):
-            os.environ["MOE_GATE_SCREEN"] = screen
-            ws = B.empty_bytes(B.moe_query_sizes(cfg).ws_bytes)
+        for flags in (SCREEN_ON, SCREEN_OFF):
+            cfg = cfg_of(w, flags)
+            S = B.moe_query_sizes(cfg)
+            ws = B.empty_bytes(S.ws_bytes)
             idx, gates = i32(w.T, w.k), f32(S.gates_elems)
             clean, raw = f32(S.logits_elems), f32(S.logits_elems)
             kv, ki = f32(S.kth_elems), i32(S.kth_elems)
             B.moe_gate(cfg, x, Wg, Wn, noise, idx, gates, clean, raw, kv, ki, ws)
             assert B.moe_check_status(ws) == 0
             out.append((idx, ki, gates))
-        os.environ["MOE_GATE_SCREEN"] = "1"
         assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
         assert_close(host(out[0][2]), host(out[1][2]), TOL_F32, "gates")

@@ -6,7 +6,6 @@ indices and permutations bit-exact, fp32 gating tensors within 1e-5, expert-side
 helpers.rel_err.
 """
 import dataclasses
-import os
 
 import numpy as np
 import pytest
@@ -16,8 +15,8 @@ from oracle import moe_oracle as O
 from paper_1701_06538_b200 import binding as B
 from paper_1701_06538_b200 import synth
 
-from helpers import (TOL_F32, act_empty, assert_close, cfg_of, dev, dev_act, device_inputs, f32, host, i32,
-                     oracle_run, prec_of, small_workload, tol_act)
+from helpers import (SCREEN_OFF, SCREEN_ON, TOL_F32, act_empty, assert_close, cfg_of, dev, dev_act, device_inputs, f32, host, i32,
+                     oracle_run, prec_of, screened, small_workload, tol_act)
 
 pytestmark = pytest.mark.gpu
 
@@ -50,20 +49,8 @@ def case(request):
     w = request.param
     I = synth.make_all(w)
     F, Bk = oracle_run(w, I)
-    return w, I, F, Bk, device_inputs(w, I), cfg_of(w)
-
-
-def screened(w):
-    """True where moe_gate screens the routing on the tensor cores: bf16, widths that are multiples of 64, and
-    either forced (MOE_GATE_SCREEN=1, set by this test session) or a projection of at least 1e9 multiply-adds."""
-    n1 = w.a if w.a else w.n
-    first = w.act == "bf16" and w.T >= 256 and w.d % 64 == 0 and (2 * n1) % 64 == 0
-    # the secondary gates of the hierarchical layer are screened on their own (rows = T * k1 slots, width b)
-    second = bool(w.a) and w.act == "bf16" and w.T * w.k1 >= 256 and w.d % 64 == 0 and (2 * w.b) % 64 == 0
-    return first or second
-
-
-os.environ["MOE_GATE_SCREEN"] = "1"  # small test shapes would otherwise stay below the automatic threshold
+    # small test shapes would otherwise stay below the automatic threshold of the routing screen
+    return w, I, F, Bk, device_inputs(w, I), cfg_of(w, SCREEN_ON)
 
 
 def ws_for(cfg):
@@ -120,7 +107,7 @@ def test_gate_screen_sends_ties_and_near_ties_to_the_exact_chain():
         I[name][:, 1::2] = I[name][:, 0::2]
     I["Wg"][:, 2] = I["Wg"][:, 0] * np.float32(1 + 2 ** -20)  # and a near-tie far below any provable gap
     G = O.gate(I["x"], I["Wg"], I["Wnoise"], I["noise"], w.k, "bf16")
-    cfg = cfg_of(w)
+    cfg = cfg_of(w, SCREEN_ON)
     ws, S = ws_for(cfg)
     D = device_inputs(w, I)
     idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
@@ -135,24 +122,22 @@ def test_gate_screen_sends_ties_and_near_ties_to_the_exact_chain():
 
 
 def test_screened_routing_equals_pure_chain_routing_on_many_batches():
-    """The screen must never change the routing: with MOE_GATE_SCREEN=0 every token goes through the fma
+    """The screen must never change the routing: with MOE_FLAG_GATE_SCREEN_OFF every token goes through the fma
     chain; both runs must give identical indices on fresh batches of a wide, skewed gate (c5's shape)."""
     from dataclasses import replace
     base = replace(synth.CONFIGS["c5"], T=16384)
     for seed in range(6):
         w = replace(base, seed=synth.BASE_SEED + 500 + seed, name=f"c5-seed{seed}")
-        cfg = cfg_of(w)
-        ws, S = ws_for(cfg)
         x, (Wg, Wn, noise) = dev_act(synth.make_x(w), w), [dev(a) for a in synth.make_gate(w)]
         out = []
-        for screen in ("1", "0"):
-            os.environ["MOE_GATE_SCREEN"] = screen
+        for flags in (SCREEN_ON, SCREEN_OFF):
+            cfg = cfg_of(w, flags)
+            ws, S = ws_for(cfg)
             idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
             kv, ki = f32(w.T, 2), i32(w.T, 2)
             B.moe_gate(cfg, x, Wg, Wn, noise, idx, gates, clean, raw, kv, ki, ws)
             assert B.moe_check_status(ws) == 0
             out.append((idx, ki, gates, clean))
-        os.environ["MOE_GATE_SCREEN"] = "1"
         assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
         assert_close(host(out[0][2]), host(out[1][2]), TOL_F32, "gates")
         assert_close(host(out[0][3]), host(out[1][3]), TOL_F32, "clean")
@@ -174,18 +159,16 @@ def test_screened_routing_equals_pure_chain_routing_on_badly_scaled_inputs():
         if seed & 1:
             Wg[:, 1::2] = Wg[:, 0::2] * (1.0 + 1e-7)                          # near-duplicate experts
         noise = noise * 4.0
-        cfg = cfg_of(w)
-        ws, S = ws_for(cfg)
         xd, Wgd, Wnd, nd = dev_act(x, w), dev(Wg), dev(Wn), dev(noise)
         out = []
-        for screen in ("1", "0"):
-            os.environ["MOE_GATE_SCREEN"] = screen
+        for flags in (SCREEN_ON, SCREEN_OFF):
+            cfg = cfg_of(w, flags)
+            ws, S = ws_for(cfg)
             idx, gates, clean, raw = i32(w.T, w.k), f32(w.T, w.k), f32(w.T, w.n), f32(w.T, w.n)
             kv, ki = f32(w.T, 2), i32(w.T, 2)
             B.moe_gate(cfg, xd, Wgd, Wnd, nd, idx, gates, clean, raw, kv, ki, ws)
             assert B.moe_check_status(ws) == 0
             out.append((idx, ki))
-        os.environ["MOE_GATE_SCREEN"] = "1"
         assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1]), seed
 
 
