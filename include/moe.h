@@ -62,6 +62,7 @@ typedef enum { MOE_F32 = 0, MOE_BF16 = 1 } moe_dtype;
 
 #define MOE_MAX_K 8          /* k, k1, k2 and k1*k2 are at most this                 */
 #define MOE_MAX_EXPERTS 8192 /* n (flat) and a, b (hierarchical levels) are at most this */
+#define MOE_MAX_FLAT_EXPERTS 12288 /* hierarchical: a*b beyond this is MOE_ERR_UNSUPPORTED (one int32 per expert in shared memory) */
 
 typedef struct moe_config {
     int32_t T, d, h;            /* tokens, model width, expert hidden width                              */

@@ -36,6 +36,8 @@ int32_t check_config(const moe_config *c) {
         if ((int64_t)c->a * c->b != c->n || c->k1 * c->k2 != c->k) return MOE_ERR_INVALID_ARG;
         if (c->a > MOE_MAX_EXPERTS || c->b > MOE_MAX_EXPERTS) return MOE_ERR_INVALID_ARG;
         if ((int64_t)c->a * c->b > (int64_t)1 << 20) return MOE_ERR_INVALID_ARG;
+        // the routing kernels keep one int32 per expert in (default-size) shared memory
+        if ((int64_t)c->a * c->b > MOE_MAX_FLAT_EXPERTS) return MOE_ERR_UNSUPPORTED;
     } else if (c->n > MOE_MAX_EXPERTS) {
         return MOE_ERR_INVALID_ARG;
     }

@@ -17,7 +17,7 @@
 //            dz = (dys.W2^T) * [hid > 0],  dxs = dz.W1^T
 //   WGRAD    contraction over the rows of a segment, both operands MN-major:
 //            dW2 = hid^T.dys,  dW1 = xs^T.dz. The last K block of a segment is ragged: the rows
-//            past the segment end are zeroed in shared memory (A operand only: 0 x finite = 0).
+//            past the segment end are zeroed in shared memory in both operands.
 // Weights are addressed through one tensor map with the expert as a coordinate, segment bounds
 // are read on the device: no per-expert descriptors and no host synchronisation.
 //
@@ -93,14 +93,13 @@ struct GemmParams {
 // Diagnostics build (-DMOE_TILE_TRACE): the first CTA records, per tile, when each warp role started, finished and how
 // long it waited; read back with moe_debug_tile_trace. Compiled out otherwise.
 #ifdef MOE_TILE_TRACE
-__device__ long long g_tile_trace[3][256][4];
+__device__ long long g_tile_trace[3][256][6];
 #define TILE_TRACE_SET(role, tile, field, val) do { if (p.trace && blockIdx.x == 0 && (tile) < 256) g_tile_trace[role][tile][field] = (val); } while (0)
-#define TILE_TRACE_ADD(role, tile, field, val) do { if (p.trace && blockIdx.x == 0 && (tile) < 256) g_tile_trace[role][tile][field] += (val); } while (0)
+
 #define TILE_CLOCK() clock64()
 static int g_trace_launch_no = 0;
 #else
 #define TILE_TRACE_SET(role, tile, field, val) do {} while (0)
-#define TILE_TRACE_ADD(role, tile, field, val) do {} while (0)
 #define TILE_CLOCK() 0ll
 #endif
 
@@ -252,6 +251,43 @@ __device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
         }
     }
     return a[0];
+}
+
+// Epilogue arithmetic of one thread's 32 accumulator columns: bias, ReLU, ReLU mask, rounding to bf16. The three
+// options are template parameters so that the loop body has no branches (with run-time flags every element pair became
+// its own basic block and the chain add -> max -> convert ran serially, 16 times).
+template <bool BIAS, bool RELU, bool MASK>
+__device__ __forceinline__ void pack32_mode(const uint32_t (&v)[32], const uint4 (&bias_raw)[4], const uint4 (&mask_raw)[4],
+                                            uint4 (&packed)[4]) {
+    const uint32_t *bw = reinterpret_cast<const uint32_t *>(bias_raw);
+    const uint32_t *mw = reinterpret_cast<const uint32_t *>(mask_raw);
+    uint32_t *out = reinterpret_cast<uint32_t *>(packed);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
+        if (BIAS) { x0 += __uint_as_float(bw[j] << 16); x1 += __uint_as_float(bw[j] & 0xffff0000u); }
+        if (RELU) { x0 = fmaxf(x0, 0.0f); x1 = fmaxf(x1, 0.0f); }
+        if (MASK) {
+            if (!(__uint_as_float(mw[j] << 16) > 0.0f)) x0 = 0.0f;
+            if (!(__uint_as_float(mw[j] & 0xffff0000u) > 0.0f)) x1 = 0.0f;
+        }
+        const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+        out[j] = *reinterpret_cast<const uint32_t *>(&h);
+    }
+}
+// mode: bit 0 bias, bit 1 ReLU, bit 2 mask (the combinations the layer uses are specialised)
+__device__ __forceinline__ void pack32(int mode, const uint32_t (&v)[32], const uint4 (&bias_raw)[4],
+                                       const uint4 (&mask_raw)[4], uint4 (&packed)[4]) {
+    switch (mode) {
+        case 0: pack32_mode<false, false, false>(v, bias_raw, mask_raw, packed); break;
+        case 1: pack32_mode<true, false, false>(v, bias_raw, mask_raw, packed); break;
+        case 3: pack32_mode<true, true, false>(v, bias_raw, mask_raw, packed); break;
+        case 4: pack32_mode<false, false, true>(v, bias_raw, mask_raw, packed); break;
+        case 2: pack32_mode<false, true, false>(v, bias_raw, mask_raw, packed); break;
+        case 5: pack32_mode<true, false, true>(v, bias_raw, mask_raw, packed); break;
+        case 6: pack32_mode<false, true, true>(v, bias_raw, mask_raw, packed); break;
+        default: pack32_mode<true, true, true>(v, bias_raw, mask_raw, packed); break;
+    }
 }
 
 struct Tile {
@@ -459,8 +495,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (KIND == WGRAD && kb == t.kblocks - 1) {
                     const int valid = t.row_end - (t.row0 + kb * BK);  // rows of this block inside the segment
                     if (valid < BK) {
-                        // zero K rows [valid, BK) of A: 128-B lines, in both 64-column chunks
-                        const int lines = (BK - valid) * (BM / 64);
+                        // zero K rows [valid, BK) of A and of B (they belong to the next segment: a non-finite value
+                        // there must not reach this segment's sums): 128-B lines in all 64-column chunks; the A tile's
+                        // two chunks are directly followed by the B tile's four
+                        const int lines = (BK - valid) * ((BM + BN) / 64);
                         for (int u = lane; u < lines * 8; u += 32) {
                             const int line = u >> 3, part = u & 7;
                             const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
@@ -500,6 +538,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter + 31 belong to this warp
+        const int pack_mode = (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
@@ -616,20 +655,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
                     }
-                    const bf16 *bias_h = reinterpret_cast<const bf16 *>(bias_raw);
-                    const bf16 *mask_h = reinterpret_cast<const bf16 *>(mask_raw);
-                    __nv_bfloat162 *ph2 = reinterpret_cast<__nv_bfloat162 *>(packed);
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-                        if (p.bias) { x0 += __bfloat162float(bias_h[j]); x1 += __bfloat162float(bias_h[j + 1]); }
-                        if (p.relu) { x0 = fmaxf(x0, 0.0f); x1 = fmaxf(x1, 0.0f); }
-                        if (p.mask) {
-                            if (!(__bfloat162float(mask_h[j]) > 0.0f)) x0 = 0.0f;
-                            if (!(__bfloat162float(mask_h[j + 1]) > 0.0f)) x1 = 0.0f;
-                        }
-                        ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
-                    }
+                    pack32(pack_mode, v, bias_raw, mask_raw, packed);
                     if (row_ok) {
                         uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
                         st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
@@ -825,8 +851,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     auto empty_bar = [&](int s) { return bars + 8u * (NST + s); };
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * NST + a); };
     auto tempty_bar = [&](int a) { return bars + 8u * (2 * NST + 2 + a); };
-    // WGRAD only: afull = this CTA's own A tile has landed (its ragged K tail is zeroed before use);
-    // ready (even CTA) = both CTAs' A tiles are landed and fixed
+    // WGRAD only: afull = this CTA's own tiles of a ragged last K block have landed (the tail rows are zeroed before use);
+    // ready (even CTA) = both CTAs' tiles are landed and fixed
     auto afull_bar = [&](int s) { return bars + 8u * (2 * NST + 4 + s); };
     auto ready_bar = [&](int s) { return bars + 8u * (3 * NST + 4 + s); };
     const uint32_t mfull_bar = bars + 8u * 28, mempty_bar = bars + 8u * 29;  // mask tile landed / read by all 8 epilogue warps
@@ -869,9 +895,11 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // rows [valid, 64) of stage s's A tile (K rows past the segment end, both 64-column chunks) := 0
+    // rows [valid, 64) of stage s's A and B tiles (K rows past the segment end; two 64-column chunks each, the B tile
+    // directly behind the A tile) := 0. Zeroing A alone would do for finite data (0 x finite = 0); B as well keeps a
+    // non-finite value of the next segment out of this segment's sums.
     auto zero_tail = [&](int s, int valid) {
-        const int lines = (BK - valid) * 2;
+        const int lines = (BK - valid) * 4;
         for (int u = lane; u < lines * 8; u += 32) {
             const int line = u >> 3, part = u & 7;
             const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
@@ -912,27 +940,29 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             while (ok && it.next(t)) {
                 int term = 0, kk = 0;  // ROW_*: piece of the contraction and column inside it
                 ++trace_tile;
-                TILE_TRACE_SET(0, trace_tile, 1, 0);
+                long long tr_empty = 0;
                 for (int kb = 0; kb < t.kblocks && ok; ++kb) {
                     if (MASKT && mask_due) load_mask(false);
                     const long long tw0 = TILE_CLOCK();
                     ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status);
                     if (!ok) break;
-                    TILE_TRACE_ADD(0, trace_tile, 1, TILE_CLOCK() - tw0);
+                    tr_empty += TILE_CLOCK() - tw0;
                     if (kb == 0) TILE_TRACE_SET(0, trace_tile, 0, TILE_CLOCK());
-                    if (kb == t.kblocks - 1) TILE_TRACE_SET(0, trace_tile, 2, TILE_CLOCK());
+                    if (kb == t.kblocks - 1) { TILE_TRACE_SET(0, trace_tile, 2, TILE_CLOCK()); TILE_TRACE_SET(0, trace_tile, 1, tr_empty); }
                     const uint32_t a_dst = base + s * STAGE2_BYTES, b_dst = a_dst + A2_BYTES;
                     if (KIND == WGRAD) {
                         const int r = t.row0 + kb * BK;
-                        if (t.row_end - r < BK) {  // ragged last block: A lands on this CTA's own barrier first
-                            if (rank == 0) mbar_expect_tx(full_bar(s), 2 * B2_BYTES);
-                            mbar_expect_tx(afull_bar(s), A2_BYTES);
+                        if (t.row_end - r < BK) {  // ragged last block: both tiles land on this CTA's own barrier first
+                            if (rank == 0) mbar_expect_tx(full_bar(s), 0);  // nothing counts on the pair's barrier: the
+                                                                            // "ready" barrier gates this stage
+                            mbar_expect_tx(afull_bar(s), STAGE2_BYTES);
                             tma_load_3d(a_dst, &tmA, afull_bar(s), 0, r, t.m0 / 64 + 2 * (int)rank);
+                            tma_load_3d(b_dst, &tmB, afull_bar(s), 0, r, t.b_chunk + 2 * (int)rank);
                         } else {
                             if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
                             tma2_load_3d(a_dst, &tmA, full_bar(s), 0, r, t.m0 / 64 + 2 * (int)rank);
+                            tma2_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk + 2 * (int)rank);
                         }
-                        tma2_load_3d(b_dst, &tmB, full_bar(s), 0, r, t.b_chunk + 2 * (int)rank);
                     } else {
                         if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE2_BYTES);
                         tma2_load_2d(a_dst, &tmA, full_bar(s), p.a_term_col[term] + kk, t.row0 + 128 * (int)rank);
@@ -974,7 +1004,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (!ok) break;
                 tc_fence_after();
                 TILE_TRACE_SET(1, trace_tile, 1, TILE_CLOCK());
-                TILE_TRACE_SET(1, trace_tile, 2, 0);
+                long long tr_wait = 0, tr_issue = 0;
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 const int tail_valid = KIND == WGRAD ? (t.row_end - t.row0) - (t.kblocks - 1) * BK : BK;  // rows of the last block
                 for (int kb = 0; kb < t.kblocks; ++kb) {
@@ -988,7 +1018,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     ok = mbar_wait(full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    TILE_TRACE_ADD(1, trace_tile, 2, TILE_CLOCK() - tw0);
+                    tr_wait += TILE_CLOCK() - tw0;
                     const uint32_t a_src = base + s * STAGE2_BYTES, b_src = a_src + A2_BYTES;
                     const long long ti0 = TILE_CLOCK();
                     const uint64_t ad0 = KIND == WGRAD ? desc_mnmajor(a_src) : desc_kmajor(a_src);
@@ -1001,12 +1031,12 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     for (int k = 0; k < BK / 16; ++k)
                         tc_mma2_bf16(d_tmem, ad0 + k * a_step, bd0 + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit2(empty_bar(s));
-                    if (kb == 0) TILE_TRACE_SET(0, trace_tile, 3, 0);
-                    TILE_TRACE_ADD(0, trace_tile, 3, TILE_CLOCK() - ti0);
+                    tr_issue += TILE_CLOCK() - ti0;
                     if (++s == NST) { s = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit2(tfull_bar(acc));
                 TILE_TRACE_SET(1, trace_tile, 3, TILE_CLOCK());
+                TILE_TRACE_SET(1, trace_tile, 2, tr_wait); TILE_TRACE_SET(0, trace_tile, 3, tr_issue);
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
         }
@@ -1063,6 +1093,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int pack_mode = (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
         uint8_t *stage_o = smem + NST * STAGE2_BYTES + (warp - 2) * 4096;
         uint32_t mask_ph = 0;
         int acc = 0;
@@ -1081,6 +1112,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 tc_fence_after();
             }
             if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 1, TILE_CLOCK());
+            long long tr_ld = 0, tr_st = 0, tr_pack = 0;
             int64_t tile_row0, out_off = 0;
             int32_t rows_valid;
             if (KIND == WGRAD) {
@@ -1116,10 +1148,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const long long tl0 = TILE_CLOCK();
                     tc_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c * 32, v);
                     tc_ld_wait();
-                    if (warp == 2 && lane == 0) {
-                        if (c == half * (BN / 64)) TILE_TRACE_SET(2, trace_tile, 3, 0);
-                        TILE_TRACE_ADD(2, trace_tile, 3, TILE_CLOCK() - tl0);
-                    }
+                    tr_ld += TILE_CLOCK() - tl0;
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
@@ -1156,20 +1185,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
                     }
-                    const bf16 *bias_h = reinterpret_cast<const bf16 *>(bias_raw);
-                    const bf16 *mask_h = reinterpret_cast<const bf16 *>(mask_raw);
-                    __nv_bfloat162 *ph2 = reinterpret_cast<__nv_bfloat162 *>(packed);
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        float x0 = __uint_as_float(v[j]), x1 = __uint_as_float(v[j + 1]);
-                        if (p.bias) { x0 += __bfloat162float(bias_h[j]); x1 += __bfloat162float(bias_h[j + 1]); }
-                        if (p.relu) { x0 = fmaxf(x0, 0.0f); x1 = fmaxf(x1, 0.0f); }
-                        if (p.mask) {
-                            if (!(__bfloat162float(mask_h[j]) > 0.0f)) x0 = 0.0f;
-                            if (!(__bfloat162float(mask_h[j + 1]) > 0.0f)) x1 = 0.0f;
-                        }
-                        ph2[j >> 1] = __floats2bfloat162_rn(x0, x1);
-                    }
+                    const long long tp0 = TILE_CLOCK();
+                    pack32(pack_mode, v, bias_raw, mask_raw, packed);
+                    tr_pack += TILE_CLOCK() - tp0;
                     if (staged) {
                         uint8_t *blk = smem + NST * STAGE2_BYTES + (c >> 1) * 16384;
 #pragma unroll
@@ -1184,9 +1202,11 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             }
                         }
                     } else if (row_ok) {
+                        const long long ts0 = TILE_CLOCK();
                         uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
                         st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
                         st_global_32B(dst + 2, packed[2], packed[3]);
+                        tr_st += TILE_CLOCK() - ts0;
                     }
                     if (p.colsum_part) {  // sums of the rounded values, rows past the segment end count as 0
                         float a[32];
@@ -1207,7 +1227,10 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 if (lane == 0) mbar_arrive_leader_relaxed(tempty_bar(acc));
                 if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
             }
-            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 2, TILE_CLOCK());
+            if (warp == 2 && lane == 0) {
+                TILE_TRACE_SET(2, trace_tile, 2, TILE_CLOCK());
+                TILE_TRACE_SET(2, trace_tile, 3, tr_ld); TILE_TRACE_SET(2, trace_tile, 4, tr_st); TILE_TRACE_SET(2, trace_tile, 5, tr_pack);
+            }
             if (MASKT) {  // the next mask tile may land once this warp's boxes have been read out
                 __syncwarp();
                 if (lane == 0) {

@@ -228,11 +228,12 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
         const double rd = (double)r[j];
         const float sigma = (float)(fmax(rd, 0.0) + log1p(exp(-fabs(rd))));
         float v = fmaf(e[j], sigma, c[j]);
+        if (!(v == v)) v = -CUDART_INF_F;  // a NaN logit ranks last: the selection stays total, indices stay in [0, n)
         int32_t id = j;
         bool shifting = false;
 #pragma unroll
         for (int s = 0; s < KL; ++s) {
-            if (shifting || v > lv[s]) {
+            if (shifting || v > lv[s] || li[s] == INT32_MAX) {  // an empty slot takes anything, -inf included
                 float tv = lv[s]; int32_t ti = li[s];
                 lv[s] = v; li[s] = id; v = tv; id = ti;
                 shifting = true;

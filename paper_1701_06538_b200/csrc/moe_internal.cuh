@@ -21,7 +21,7 @@
 #define MOE_LAUNCHED()                                           \
     do {                                                         \
         ::moe::count_launch();                                   \
-        if (cudaPeekAtLastError() != cudaSuccess) return MOE_ERR_CUDA; \
+        if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA; /* consumed: reported once */ \
     } while (0)
 
 namespace moe {

@@ -136,6 +136,8 @@ __global__ void __launch_bounds__(32) dispatch_rank_kernel(const int32_t *__rest
             const int32_t r = start + rank;
             perm[r] = (int32_t)p;
             inv_perm[p] = r;
+        } else if (live) {
+            inv_perm[p] = -1;  // expert id outside [0, n): the slot is dropped; the row movers skip negative rows
         }
         __syncwarp();
     }
@@ -224,6 +226,7 @@ __global__ void __launch_bounds__(256) dispatch_rows_kernel(const XT *__restrict
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int nvec = d / VN;
+    const int64_t R = T * k;  // a row index outside [0, R) (dropped slot, or a caller's bad inv_perm) is skipped, never followed
     for (int64_t t = warp; t < T; t += nwarps) {
         int32_t rows[MOE_MAX_K];
 #pragma unroll
@@ -233,7 +236,7 @@ __global__ void __launch_bounds__(256) dispatch_rows_kernel(const XT *__restrict
             const uint4 val = src[v];
 #pragma unroll
             for (int s = 0; s < MOE_MAX_K; ++s)
-                if (s < k) reinterpret_cast<uint4 *>(xs + (int64_t)rows[s] * d)[v] = val;
+                if (s < k && (uint32_t)rows[s] < (uint32_t)R) reinterpret_cast<uint4 *>(xs + (int64_t)rows[s] * d)[v] = val;
         }
     }
 }
@@ -276,8 +279,11 @@ __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys,
         float g[KT];
 #pragma unroll
         for (int s = 0; s < KT; ++s) {
-            rowp[s] = reinterpret_cast<const uint4 *>(ys + (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d);
-            g[s] = s < k ? gates[t * k + s] : 0.0f;
+            int32_t row = s < k ? inv_perm[t * k + s] : 0;
+            const bool valid = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot contributes nothing
+            if (!valid) row = 0;
+            rowp[s] = reinterpret_cast<const uint4 *>(ys + (int64_t)row * d);
+            g[s] = (s < k && valid) ? gates[t * k + s] : 0.0f;
         }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
             Vec16<XT> in[KT][VB];
@@ -337,9 +343,12 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
     for (int64_t t = warp; t < T; t += nwarps) {
         int64_t rowo[KT];
         float g[KT], dot[KT];
+        bool valid[KT];
 #pragma unroll
         for (int s = 0; s < KT; ++s) {
-            rowo[s] = (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d;
+            const int32_t row = s < k ? inv_perm[t * k + s] : -1;
+            valid[s] = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot: zero gate gradient, no row written
+            rowo[s] = (int64_t)(valid[s] ? row : 0) * d;
             g[s] = s < k ? gates[t * k + s] : 0.0f;
             dot[s] = 0.0f;
         }
@@ -351,7 +360,7 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
                     dy[b].raw = reinterpret_cast<const uint4 *>(dY + t * d)[v0 + 32 * b];
 #pragma unroll
                     for (int s = 0; s < KT; ++s)
-                        if (s < k) in[s][b].raw = reinterpret_cast<const uint4 *>(ys + rowo[s])[v0 + 32 * b];
+                        if (s < k) in[s][b].raw = reinterpret_cast<const uint4 *>(ys + rowo[s])[v0 + 32 * b];  // row 0 for a dropped slot
                 }
             }
 #pragma unroll
@@ -366,7 +375,7 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
                             dot[s] = fmaf(dy[b].get(i), in[s][b].get(i), dot[s]);
                             out.set(i, g[s] * dy[b].get(i));
                         }
-                        reinterpret_cast<uint4 *>(dys + rowo[s])[v0 + 32 * b] = out.raw;
+                        if (valid[s]) reinterpret_cast<uint4 *>(dys + rowo[s])[v0 + 32 * b] = out.raw;
                     }
                 }
             }
@@ -377,7 +386,7 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
                 float v = dot[s];
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-                if (lane == 0) dgates[t * k + s] = v;
+                if (lane == 0) dgates[t * k + s] = valid[s] ? v : 0.0f;
             }
         }
     }
@@ -414,9 +423,13 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
     const int nvec = d / VN;
     for (int64_t t = warp; t < T; t += nwarps) {
         const uint4 *rowp[KT];
+        bool valid[KT];
 #pragma unroll
-        for (int s = 0; s < KT; ++s)
-            rowp[s] = reinterpret_cast<const uint4 *>(dxs + (int64_t)(s < k ? inv_perm[t * k + s] : 0) * d);
+        for (int s = 0; s < KT; ++s) {
+            const int32_t row = s < k ? inv_perm[t * k + s] : -1;
+            valid[s] = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot contributes nothing
+            rowp[s] = reinterpret_cast<const uint4 *>(dxs + (int64_t)(valid[s] ? row : 0) * d);
+        }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
             Vec16<XT> in[KT][VB];
             float4 addv[VB][VN / 4];
@@ -425,7 +438,7 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
                 if (v0 + 32 * b < nvec) {
 #pragma unroll
                     for (int s = 0; s < KT; ++s)
-                        if (s < k) in[s][b].raw = rowp[s][v0 + 32 * b];
+                        if (s < k) in[s][b].raw = valid[s] ? rowp[s][v0 + 32 * b] : make_uint4(0, 0, 0, 0);
                     if (add) {
 #pragma unroll
                         for (int q = 0; q < VN / 4; ++q)

@@ -53,6 +53,8 @@ def test_validate_accepts_the_five_workloads_and_rejects_bad_ones(lib):
     for kw in bad:
         assert B.moe_validate(B.make_config(**kw)) == 1, kw
     assert B.moe_validate(B.make_config(**dict(ok, a=2, b=4, k1=1, k2=2))) == 0
+    # a hierarchical layer with more experts than the routing kernels hold in shared memory: refused up front
+    assert B.moe_validate(B.make_config(**dict(ok, T=64, n=128 * 128, k=4, a=128, b=128, k1=2, k2=2))) == 2
     assert lib.moe_validate(None) == 1
     assert lib.moe_status_string(5) == b"device-side wait timed out"
 

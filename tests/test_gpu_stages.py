@@ -292,3 +292,102 @@ def test_empty_batch():
     B.moe_dispatch(cfg, act_empty(w, 1, w.d), i32(1), act_empty(w, 1, w.d), i32(1), i32(1), counts, offsets, ws)
     torch.cuda.synchronize()
     assert host(counts).sum() == 0 and host(offsets).sum() == 0
+
+
+def test_non_finite_inputs_never_leave_the_index_range():
+    """A token full of NaN (and one with an infinite feature) gives NaN logits: the selection must still return k
+    distinct experts in [0, n), so that nothing downstream follows a bad index; the whole layer then runs without a
+    fault and the other tokens' routing is the oracle's."""
+    for flags, T in ((SCREEN_ON, 1024), (SCREEN_OFF, 300)):
+        w = small_workload("nan-token", T=T, d=64, h=64, n=32, k=2, act="bf16", seed=21)
+        I = synth.make_all(w)
+        I["x"][5, :] = np.nan
+        I["x"][9, 3] = np.inf
+        cfg = cfg_of(w, flags)
+        S = B.moe_query_sizes(cfg)
+        D = device_inputs(w, I)
+        ctx, ws = B.empty_bytes(S.ctx_bytes), B.empty_bytes(max(S.ws_fwd_bytes, S.ws_bwd_bytes))
+        ctx.fill_(0xFF)  # stale context: any index taken from it would be far out of range
+        y, losses, imp, load, counts = act_empty(w, w.T, w.d), f32(2), f32(w.n), f32(S.load_elems), i32(w.n)
+        B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], y, losses, imp,
+                      load, counts, ctx, ws)
+        dX, dWg, dWn = act_empty(w, w.T, w.d), f32(S.wg_elems), f32(S.wg_elems)
+        dW1, db1 = act_empty(w, w.n, w.d, w.h), act_empty(w, w.n, w.h)
+        dW2, db2 = act_empty(w, w.n, w.h, w.d), act_empty(w, w.n, w.d)
+        B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], ctx,
+                       dX, dWg, dWn, dW1, db1, dW2, db2, ws)
+        assert B.moe_check_status(ws) == 0
+        V = B.ctx_views(cfg, ctx)
+        idx = host(V["topk_idx"])
+        assert idx.min() >= 0 and idx.max() < w.n
+        assert (idx[:, 0] != idx[:, 1]).all()
+        inv = host(V["inv_perm"])
+        assert inv.min() >= 0 and inv.max() < S.R and int(host(counts).sum()) == S.R
+        good = np.ones(w.T, bool)
+        good[[5, 9]] = False
+        I2 = dict(I, x=np.where(np.isfinite(I["x"]), I["x"], 0.0).astype(np.float32))
+        G = O.gate(I2["x"], I["Wg"], I["Wnoise"], I["noise"], w.k, "bf16")
+        assert (idx[good] == G.idx[good]).all()
+        assert np.isfinite(host(y)[good]).all()
+
+
+def test_dispatch_drops_expert_ids_outside_the_range():
+    """moe_dispatch with caller-made indices: ids outside [0, n) are dropped (inv_perm -1), the row movers skip them."""
+    w = small_workload("bad-ids", T=200, d=32, h=16, n=6, k=2, act="f32", seed=22)
+    cfg = cfg_of(w)
+    ws, S = ws_for(cfg)
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, w.n, size=(w.T, w.k)).astype(np.int32)
+    idx[7, 1] = w.n + 3
+    idx[11, 0] = -2
+    idx[100, 1] = 2 ** 31 - 1
+    x = dev_act(synth.make_x(w), w)
+    xs, perm, inv = act_empty(w, S.R, w.d), i32(S.R), i32(S.R)
+    xs.fill_(-7.0)
+    counts, offsets = i32(w.n), i32(w.n + 1)
+    B.moe_dispatch(cfg, x, dev(idx), xs, perm, inv, counts, offsets, ws)
+    inv_h = host(inv).reshape(w.T, w.k)
+    assert inv_h[7, 1] == -1 and inv_h[11, 0] == -1 and inv_h[100, 1] == -1
+    assert int(host(counts).sum()) == S.R - 3 and (np.sort(inv_h[inv_h >= 0]) == np.arange(S.R - 3)).all()
+    gates = dev(np.full((w.T, w.k), 0.5, np.float32))
+    y = act_empty(w, w.T, w.d)
+    B.moe_combine(cfg, xs, gates, inv, y)                      # dropped slots contribute nothing
+    xh = host(x)
+    want = xh.copy()
+    want[[7, 11, 100]] *= 0.5
+    assert np.allclose(host(y), want, rtol=1e-6, atol=1e-6)
+    dg, dys = f32(w.T, w.k), act_empty(w, S.R, w.d)
+    B.moe_combine_bwd(cfg, x, xs, gates, inv, dg, dys)
+    assert host(dg)[7, 1] == 0 and host(dg)[11, 0] == 0
+    out = f32(w.T, w.d)
+    B.moe_dispatch_bwd(cfg, xs, inv, out)
+    torch.cuda.synchronize()
+    assert np.isfinite(host(out)).all()
+
+
+def test_non_finite_rows_of_one_expert_do_not_reach_the_others_weight_gradients():
+    """The weight-gradient GEMMs contract over ragged row ranges; the rows behind a segment's end belong to the next
+    expert and are cleared in both operands, so Inf there cannot turn into 0 x Inf = NaN in this expert's sums."""
+    for T, n, d, h in ((3000, 5, 128, 256), (700, 9, 64, 64)):   # SM-pair kernels / one-CTA kernels
+        w = small_workload("inf-rows", T=T, d=d, h=h, n=n, k=2, act="bf16", seed=23)
+        I = synth.make_all(w)
+        F, Bk = oracle_run(w, I)
+        cfg = cfg_of(w)
+        ws, S = ws_for(cfg)
+        bad = 2
+        o0, o1 = int(F.D.offsets[bad]), int(F.D.offsets[bad + 1])
+        assert o1 - o0 > 0 and o0 % 64 != 0
+        dys = np.asarray(Bk.dys, np.float32).copy()
+        dys[o0:o1] = np.inf
+        hid = np.asarray(F.hid, np.float32).copy()
+        hid[o0:o1] = np.inf
+        dxs = act_empty(w, S.R, w.d)
+        dW1, db1 = act_empty(w, w.n, w.d, w.h), act_empty(w, w.n, w.h)
+        dW2, db2 = act_empty(w, w.n, w.h, w.d), act_empty(w, w.n, w.d)
+        D = device_inputs(w, I)
+        B.moe_expert_ffn_bwd(cfg, dev_act(F.D.xs, w), dev_act(hid, w), dev_act(dys, w), dev(F.D.offsets), D["W1"],
+                             D["W2"], dxs, dW1, db1, dW2, db2, ws)
+        assert B.moe_check_status(ws) == 0
+        others = [e for e in range(w.n) if e != bad]
+        for name, got, want in (("dW1", dW1, Bk.dW1), ("dW2", dW2, Bk.dW2), ("db1", db1, Bk.db1), ("db2", db2, Bk.db2)):
+            assert_close(host(got)[others], np.asarray(want)[others], tol_act(w), name)
