@@ -69,7 +69,7 @@ def test_full_size_fused(name):
     assert_close(host(V["gates"]), want_gates, TOL_F32, "gates")
     assert_close(host(D["importance"]), LS.importance, TOL_F32, "importance")
     assert_close(host(D["load"])[:w.n], LS.load, TOL_F32, "load")
-    assert_close(host(D["losses"]), LS.losses, dict(max=2e-4, mean=2e-4), "losses")
+    assert_close(host(D["losses"]), LS.losses, TOL_F32, "losses")
     xs_rows = host(V["xs"][torch.from_numpy(np.arange(0, S.R, max(1, S.R // 97))).cuda()])
     assert (xs_rows == x[Dp.perm[np.arange(0, S.R, max(1, S.R // 97))] // w.k]).all()
 

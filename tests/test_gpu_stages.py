@@ -207,7 +207,7 @@ def test_losses(case):
     B.moe_losses(cfg, dev(F.G.idx), dev(F.G.gates), dev(F.G.clean), dev(F.G.raw), dev(F.G.kth_val), imp, load, L, ws)
     assert_close(host(imp), F.LS.importance, TOL_F32, "importance")
     assert_close(host(load), F.LS.load, TOL_F32, "load")
-    assert_close(host(L), F.LS.losses, dict(max=2e-4, mean=2e-4), "losses")  # CV^2 amplifies by ~mean/std
+    assert_close(host(L), F.LS.losses, TOL_F32, "losses")
 
 
 def test_combine_bwd(case):
@@ -252,7 +252,7 @@ def test_losses_bwd_and_gate_bwd(case):
     dg, dload = dev(np.asarray(Bk.dgates, np.float32)), f32(S.dload_elems)
     B.moe_losses_bwd(cfg, dev(F.LS.importance), dev(F.LS.load), dev(F.G.idx), dg, dload, ws)
     assert_close(host(dg), dg_want, TOL_F32, "dgates+importance")
-    assert_close(host(dload), dload_want, dict(max=1e-4, mean=1e-4), "dload")
+    assert_close(host(dload), dload_want, TOL_F32, "dload")
     GB = O.gate_bwd(I["x"], I["Wg"], I["Wnoise"], I["noise"], F.G.clean, F.G.raw, F.G.idx, F.G.gates, F.G.kth_val,
                     F.G.kth_idx, dg_want, dload_want, prec)
     dWg, dWn, dXg = f32(w.d, w.n), f32(w.d, w.n), f32(w.T, w.d)

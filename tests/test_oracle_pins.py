@@ -207,6 +207,55 @@ def test_bf16_rounding_points():
     assert np.abs(hid - exact).max() <= np.abs(exact).max() * 2.0 ** -8
 
 
+def test_bf16_rounding_points_of_the_backward():
+    """In "bf16" mode every expert-side tensor the backward materialises (dys, dz, dxs, dW1, db1, dW2, db2, dX) is
+    rounded once to bfloat16: each must be representable (checked with the library's rounding, not the oracle's) and
+    within one bf16 unit of the float64-mode value computed from the same rounded inputs; the gating-side tensors
+    (dgates, dWg, dWnoise) stay float32. A forgotten rounding would leave non-representable values behind."""
+    def representable(a):
+        a = np.asarray(a, np.float32)
+        return (torch.from_numpy(np.ascontiguousarray(a)).bfloat16().float().numpy() == a).all()
+
+    g = rng(31)
+    T, d, n, k, h = 48, 16, 4, 2, 24
+    x = O.round_bf16(g.standard_normal((T, d)).astype(np.float32))
+    dY = O.round_bf16(g.standard_normal((T, d)).astype(np.float32))
+    Wg, Wn = (g.standard_normal((d, n)).astype(np.float32) / 4 for _ in range(2))
+    noise = g.standard_normal((T, n)).astype(np.float32)
+    W1 = O.round_bf16(g.standard_normal((n, d, h)).astype(np.float32) / 4)
+    W2 = O.round_bf16(g.standard_normal((n, h, d)).astype(np.float32) / 5)
+    b1 = O.round_bf16(g.standard_normal((n, h)).astype(np.float32) / 3)
+    b2 = O.round_bf16(g.standard_normal((n, d)).astype(np.float32) / 3)
+    F = O.forward(x, Wg, Wn, noise, W1, b1, W2, b2, k, 0.1, 0.1, "bf16")
+    Bk = O.backward(dY, x, Wg, Wn, noise, W1, b1, W2, b2, F, 0.1, 0.1, "bf16")
+    for name in ("dys", "dz", "dxs", "dW1", "db1", "dW2", "db2", "dX"):
+        assert representable(getattr(Bk, name)), name
+    for name in ("dgates", "dWg", "dWnoise"):   # fp32 gating path: not squeezed into bf16
+        assert not representable(getattr(Bk, name)), name
+    # one rounding each: against float64 evaluations of the single steps on the same (rounded) inputs
+    ulp = 2.0 ** -8  # half-ulp relative error of round-to-nearest is 2^-9; one unit leaves room for the rms floor below
+
+    def one_rounding(got, exact, name):
+        got, exact = np.asarray(got, f64), np.asarray(exact, f64)
+        assert np.abs(got - exact).max() <= ulp * np.abs(exact).max(), name
+        assert (np.abs(got - exact) <= ulp * np.abs(exact) + 1e-30).all(), name
+
+    rows = F.D.inv_perm.reshape(T, k)
+    for s_ in range(k):
+        one_rounding(Bk.dys[rows[:, s_]], np.asarray(F.G.gates, f64)[:, s_, None] * dY.astype(f64), "dys")
+    E64 = O.expert_ffn_bwd(F.D.xs, F.hid, Bk.dys, F.D.offsets, W1, W2, "f64")
+    one_rounding(Bk.dz, E64.dz, "dz")
+    one_rounding(Bk.dW2, E64.dW2, "dW2")
+    one_rounding(Bk.db2, E64.db2, "db2")
+    for e in range(n):   # the steps behind dz take the ROUNDED dz as their input
+        o0, o1 = int(F.D.offsets[e]), int(F.D.offsets[e + 1])
+        dz = np.asarray(Bk.dz[o0:o1], f64)
+        one_rounding(Bk.db1[e], dz.sum(axis=0), "db1")
+        one_rounding(Bk.dW1[e], np.asarray(F.D.xs[o0:o1], f64).T @ dz, "dW1")
+        one_rounding(Bk.dxs[o0:o1], dz @ W1[e].astype(f64).T, "dxs")
+    one_rounding(Bk.dX, np.asarray(Bk.dX_expert, f64) + np.asarray(Bk.dX_gate, f64), "dX")
+
+
 # ---------------------------------------------------------------- dispatch / combine
 def test_dispatch_is_stable_counting_sort_and_round_trips():
     g = rng(10)
