@@ -27,7 +27,8 @@ CV^2 closed forms; P(x, i) against Monte-Carlo on its definition, against a
 delete-and-sort kth_excluding, and against the zero-initialisation closed form;
 hierarchical reductions to the flat layer; every backward against central finite
 differences of the forward in float64; the single-precision chain against an
-exact rational emulation. The table of trained-model balance metrics in the
+exact rational emulation; the layer epilogue (sigmoid, dropout, residual) against its
+closed forms and finite differences. The table of trained-model balance metrics in the
 paper's Appendix A cannot be reproduced without the trained model: for those
 printed values parity is unpinned; the metric definitions themselves are pinned
 by the CV^2 closed forms.
@@ -234,6 +235,48 @@ def combine(ys, gates, inv_perm, prec):
     for s in range(k):
         y = y + np.asarray(gates[:, s], f64)[:, None] * np.asarray(ys[rows[:, s]], f64)
     return store(y, prec, expert_side=True)
+
+
+def unpack_keep(keep_bits, d):
+    """Dropout keep mask [T, d] (bool) from its packed form: bit (q % 8) of byte q // 8 of a row is column q."""
+    bits = np.unpackbits(np.asarray(keep_bits, np.uint8), axis=1, bitorder="little")
+    return bits[:, :d].astype(bool)
+
+
+def combine_layer(ys, gates, inv_perm, x, keep, drop_prob, prec):
+    """The MoE layer as it sits in the paper's models (Appendix C, model and MoE layer architecture): the MoE output
+    y of Eq. 1 goes through a sigmoid, then dropout (each activation dropped with probability DropProb, the kept
+    ones divided by 1 - DropProb), then the layer's input is added (residual connection):
+        out = x + keep * sigmoid(y) / (1 - DropProb).
+    `keep` [T, d] is the 0/1 dropout mask, an input (drawn by the caller, like the gating noise). Only `out` is
+    materialised (one rounding); y stays in working precision."""
+    T, k = gates.shape
+    rows = inv_perm.reshape(T, k).astype(np.int64)
+    y = np.zeros((T, ys.shape[1]), f64)
+    for s in range(k):
+        y = y + np.asarray(gates[:, s], f64)[:, None] * np.asarray(ys[rows[:, s]], f64)
+    sig = 1.0 / (1.0 + np.exp(-y))
+    out = np.asarray(x, f64) + np.asarray(keep, f64) * sig / (1.0 - drop_prob)
+    return store(out, prec, expert_side=True)
+
+
+def combine_layer_bwd(dOut, ys, gates, inv_perm, keep, drop_prob, prec):
+    """Adjoint of combine_layer. Through the residual connection dOut reaches the layer input unchanged (the
+    caller adds it to dX); through dropout and the sigmoid dy = dOut * keep / (1 - DropProb) * s (1 - s) with
+    s = sigmoid(y), and from there on as in combine_bwd."""
+    T, k = gates.shape
+    rows = inv_perm.reshape(T, k).astype(np.int64)
+    y = np.zeros((T, ys.shape[1]), f64)
+    for s in range(k):
+        y = y + np.asarray(gates[:, s], f64)[:, None] * np.asarray(ys[rows[:, s]], f64)
+    sig = 1.0 / (1.0 + np.exp(-y))
+    dy = np.asarray(dOut, f64) * np.asarray(keep, f64) / (1.0 - drop_prob) * sig * (1.0 - sig)
+    dgates = np.zeros((T, k), f64)
+    dys = np.zeros(ys.shape, f64)
+    for s in range(k):
+        dgates[:, s] = (dy * np.asarray(ys[rows[:, s]], f64)).sum(axis=1)
+        dys[rows[:, s]] = np.asarray(gates[:, s], f64)[:, None] * dy
+    return store(dgates, prec), store(dys, prec, expert_side=True)
 
 
 # --------------------------------------------------------------------------------------
@@ -492,11 +535,12 @@ def gate_h_bwd(x, Wg_p, Wn_p, noise_p, Wg_s, Wn_s, noise_s, G, LS, dgates, w_imp
 # --------------------------------------------------------------------------------------
 # the whole layer
 # --------------------------------------------------------------------------------------
-def forward(x, Wg, Wnoise, noise, W1, b1, W2, b2, k, w_importance, w_load, prec, hier=None):
+def forward(x, Wg, Wnoise, noise, W1, b1, W2, b2, k, w_importance, w_load, prec, hier=None, layer=None):
     """Forward of the layer with both balancing losses.
 
     Flat: Wg, Wnoise [d,n], noise [T,n]. Hierarchical (hier=(a, k1, b, k2)): Wg, Wnoise and
-    noise are pairs (primary, secondary) and k is ignored."""
+    noise are pairs (primary, secondary) and k is ignored. layer=(keep [T,d], drop_prob): the output is
+    that of combine_layer (sigmoid, dropout, residual) instead of the plain mixture of Eq. 1."""
     n = W1.shape[0]
     if hier is None:
         G = gate(x, Wg, Wnoise, noise, k, prec)
@@ -507,15 +551,22 @@ def forward(x, Wg, Wnoise, noise, W1, b1, W2, b2, k, w_importance, w_load, prec,
         LS = losses_h(G, a, b, w_importance, w_load, prec)
     D = dispatch(x, G.idx, n)
     hid, ys = expert_ffn(D.xs, D.offsets, W1, b1, W2, b2, prec)
-    y = combine(ys, G.gates, D.inv_perm, prec)
+    if layer is None:
+        y = combine(ys, G.gates, D.inv_perm, prec)
+    else:
+        y = combine_layer(ys, G.gates, D.inv_perm, x, layer[0], layer[1], prec)
     return SimpleNamespace(y=y, G=G, D=D, LS=LS, hid=hid, ys=ys)
 
 
-def backward(dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, F, w_importance, w_load, prec, hier=None):
+def backward(dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, F, w_importance, w_load, prec, hier=None, layer=None):
     """Backward of the layer; both balancing losses enter with upstream gradient 1
-    (they are added to the model's loss, Section 4)."""
+    (they are added to the model's loss, Section 4). With layer=(keep, drop_prob) dY is the gradient of
+    combine_layer's output and also reaches dX directly through the residual connection."""
     T, k = F.G.idx.shape
-    dgates, dys = combine_bwd(dY, F.ys, F.G.gates, F.D.inv_perm, prec)
+    if layer is None:
+        dgates, dys = combine_bwd(dY, F.ys, F.G.gates, F.D.inv_perm, prec)
+    else:
+        dgates, dys = combine_layer_bwd(dY, F.ys, F.G.gates, F.D.inv_perm, layer[0], layer[1], prec)
     E = expert_ffn_bwd(F.D.xs, F.hid, dys, F.D.offsets, W1, W2, prec)
     dX_exp = dispatch_bwd(E.dxs, F.D.inv_perm, T, k, prec)
     if hier is None:
@@ -527,6 +578,9 @@ def backward(dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, F, w_importance, w_load, 
         GB = gate_h_bwd(x, Wg[0], Wnoise[0], noise[0], Wg[1], Wnoise[1], noise[1], F.G, F.LS, dgates,
                         w_importance, w_load, prec)
         dWg, dWn = (GB.dWg_p, GB.dWg_s), (GB.dWn_p, GB.dWn_s)
-    dX = store(np.asarray(dX_exp, f64) + np.asarray(GB.dX_gate, f64), prec, expert_side=True)
+    dX_sum = np.asarray(dX_exp, f64) + np.asarray(GB.dX_gate, f64)
+    if layer is not None:
+        dX_sum = dX_sum + np.asarray(dY, f64)  # residual connection
+    dX = store(dX_sum, prec, expert_side=True)
     return SimpleNamespace(dX=dX, dWg=dWg, dWnoise=dWn, dW1=E.dW1, db1=E.db1, dW2=E.dW2, db2=E.db2,
                            dgates=dgates, dys=dys, dxs=E.dxs, dz=E.dz, dX_expert=dX_exp, dX_gate=GB.dX_gate)

@@ -508,3 +508,72 @@ def test_rounded_modes_stay_close_to_float64():
     for name in ("dX", "dWg", "dWnoise", "dW1", "dW2"):
         ref = getattr(out["f64"][1], name)
         assert np.abs(getattr(out["f32"][1], name) - ref).max() <= 1e-5 * (np.abs(ref).max() + 1)
+
+
+# ---------------------------------------------------------------- layer epilogue: sigmoid, dropout, residual (Appendix C)
+def test_layer_epilogue_closed_forms():
+    g = rng(40)
+    T, k, d = 9, 2, 16
+    ys = g.standard_normal((T * k, d))
+    gates = g.random((T, k)); gates /= gates.sum(axis=1, keepdims=True)
+    inv = g.permutation(T * k).astype(np.int32)
+    x = g.standard_normal((T, d))
+    y = np.asarray(O.combine(ys, gates, inv, "f64"))
+    ones = np.ones((T, d), bool)
+    # no dropout: out - x is the logistic function of the mixture; textbook values of the logistic function
+    out = O.combine_layer(ys, gates, inv, x, ones, 0.0, "f64")
+    assert np.allclose(out - x, 1.0 / (1.0 + np.exp(-y)), rtol=1e-14)
+    assert np.allclose(out - x + (O.combine_layer(-ys, gates, inv, x, ones, 0.0, "f64") - x), 1.0, rtol=1e-13)  # s(y)+s(-y)=1
+    zero = O.combine_layer(np.zeros_like(ys), gates, inv, x, ones, 0.0, "f64")
+    assert np.allclose(zero - x, 0.5, rtol=1e-15)
+    # everything dropped: the residual alone; everything kept with DropProb 1/2: twice the sigmoid
+    assert (O.combine_layer(ys, gates, inv, x, ~ones, 0.3, "f64") == x).all()
+    assert np.allclose(O.combine_layer(ys, gates, inv, x, ones, 0.5, "f64") - x, 2.0 * (out - x), rtol=1e-14)
+    # dropout is unbiased: averaging over a mask and its complement, each scaled for DropProb 1/2, gives back the sigmoid
+    keep = g.random((T, d)) < 0.5
+    a = O.combine_layer(ys, gates, inv, x, keep, 0.5, "f64") - x
+    b = O.combine_layer(ys, gates, inv, x, ~keep, 0.5, "f64") - x
+    assert np.allclose(0.5 * (a + b), out - x, rtol=1e-13)
+    # the packed mask format
+    bits = np.packbits(keep, axis=1, bitorder="little")
+    assert (O.unpack_keep(bits, d) == keep).all()
+    assert O.unpack_keep(np.array([[0b00000101]], np.uint8), 8).tolist() == [[True, False, True] + [False] * 5]
+
+
+def test_layer_epilogue_backward_matches_finite_differences():
+    p = tiny(41)
+    T, d = p["x"].shape
+    g = rng(42)
+    keep = g.random((T, d)) < 0.7
+    layer = (keep, 0.3)
+    dOut = g.standard_normal((T, d))
+    k, wi, wl = 3, 0.1, 0.2
+
+    def loss():
+        F = O.forward(p["x"], p["Wg"], p["Wnoise"], p["noise"], p["W1"], p["b1"], p["W2"], p["b2"], k, wi, wl, "f64",
+                      layer=layer)
+        return float((F.y * dOut).sum() + F.LS.losses.sum()), F
+
+    base, F = loss()
+    Bk = O.backward(dOut, p["x"], p["Wg"], p["Wnoise"], p["noise"], p["W1"], p["b1"], p["W2"], p["b2"], F, wi, wl, "f64",
+                    layer=layer)
+    step = 1e-6
+    for name, grad, arr in flat_names(p, Bk):
+        flat = arr.reshape(-1)
+        scale = max(np.abs(grad).max(), 1e-3)
+        for pos in g.choice(flat.size, size=min(10, flat.size), replace=False):
+            old = flat[pos]
+            flat[pos] = old + step
+            up, Fu = loss()
+            flat[pos] = old - step
+            dn, Fd = loss()
+            flat[pos] = old
+            assert (Fu.G.idx == F.G.idx).all() and (Fd.G.idx == F.G.idx).all()
+            assert abs((up - dn) / (2 * step) - grad.reshape(-1)[pos]) / scale < 2e-6, (name, pos)
+    # dropped activations pass no gradient into the experts: with everything dropped only the residual and the
+    # balancing losses are left
+    none = (np.zeros((T, d), bool), 0.3)
+    F0 = O.forward(p["x"], p["Wg"], p["Wnoise"], p["noise"], p["W1"], p["b1"], p["W2"], p["b2"], k, wi, wl, "f64", layer=none)
+    B0 = O.backward(dOut, p["x"], p["Wg"], p["Wnoise"], p["noise"], p["W1"], p["b1"], p["W2"], p["b2"], F0, wi, wl, "f64",
+                    layer=none)
+    assert np.abs(B0.dW1).max() == 0 and np.abs(B0.dW2).max() == 0 and np.abs(B0.dys).max() == 0
