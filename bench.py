@@ -447,6 +447,16 @@ def stage_timings(B, cfg, S, D, w, timed, K, peaks):
                      8.0 * T * d * gate_cols, T * d * (esz + 4) + 5 * 4 * T * gate_cols),
         "dispatch_bwd": (lambda: B.moe_dispatch_bwd(cfg, dxs, V["inv_perm"], dXe), 0.0, k * T * d * esz + T * d * 4),
     }
+    if d % 8 == 0:
+        # the layer as it sits in the paper's models (sigmoid, dropout, residual fused into the combine kernels): timed
+        # beside the plain stages, not part of the step; the keep mask is one bit per activation
+        keep = torch.from_numpy(synth.make_keep_bits(w, 0.3)).cuda()
+        out_layer = e(T, d, dt=adt)
+        calls["combine_layer"] = (lambda: B.moe_combine_layer(cfg, V["ys"], V["gates"], V["inv_perm"], D["x"], keep, 0.3,
+                                                              out_layer), 0.0, (k + 2) * T * d * esz + T * d // 8 + 8 * R)
+        calls["combine_layer_bwd"] = (lambda: B.moe_combine_layer_bwd(cfg, D["dY"], V["ys"], V["gates"], V["inv_perm"],
+                                                                      keep, 0.3, dgates, dys), 0.0,
+                                      (1 + 2 * k) * T * d * esz + T * d // 8 + 12 * R)
     out = {}
     for name, (fn, flop, byts) in calls.items():
         fn()

@@ -258,6 +258,41 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
                      const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
                      void *db2, void *ws, void *stream);
 
+/* ------------------------------------------------------------------------------------------
+ * The layer inside the paper's models (Appendix C, "Model Architecture" and "MoE Layer Architecture"):
+ * the MoE output goes through a sigmoid, then dropout (each activation dropped with probability
+ * drop_prob, the kept ones divided by 1 - drop_prob), then the layer's input is added (residual):
+ *     out[t] = x[t] + keep[t] * sigmoid(y[t]) / (1 - drop_prob),   y[t] = sum_s gates[t,s] * ys[row(t,s)]  (Eq. 1)
+ * fused into the combine kernels, so y makes no round trip through memory (it is never stored; the
+ * backward recomputes it from the ys rows it gathers anyway).
+ * keep_bits [T, d/8] uint8 is the dropout mask, an INPUT drawn by the caller like the gating noise:
+ * bit (q % 8) of byte q / 8 of a token's row is 1 where column q is kept. Needs d % 8 == 0 and
+ * 0 <= drop_prob < 1 (MOE_ERR_INVALID_ARG otherwise).
+ * ------------------------------------------------------------------------------------------ */
+
+/* Combine with the layer epilogue.   in: ys, gates [T,k], inv_perm, x [T,d] act   out: out [T,d] act */
+int32_t moe_combine_layer(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm,
+                          const void *x, const uint8_t *keep_bits, float drop_prob, void *out, void *stream);
+
+/* Its adjoint: dy = dOut * keep / (1 - drop_prob) * s (1 - s) with s = sigmoid(y), then as moe_combine_bwd:
+ * dgates [T,k] = <dy[t], ys[row]>, dys [R,d] act = gates[t,s] * dy[t]. The gradient through the residual
+ * connection is dOut itself: the caller adds it to dX (moe_layer_backward does). */
+int32_t moe_combine_layer_bwd(const moe_config *cfg, const void *dOut, const void *ys, const float *gates,
+                              const int32_t *inv_perm, const uint8_t *keep_bits, float drop_prob, float *dgates,
+                              void *dys, void *stream);
+
+/* moe_forward / moe_backward with the layer epilogue: `out` replaces y, dOut replaces dY, and dX also
+ * receives dOut through the residual connection. Same context and workspaces as the plain calls. */
+int32_t moe_layer_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise,
+                          const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                          const uint8_t *keep_bits, float drop_prob, void *out, float *losses, float *importance,
+                          float *load, int32_t *counts, void *ctx, void *ws, void *stream);
+int32_t moe_layer_backward(const moe_config *cfg, const void *dOut, const void *x, const float *Wg,
+                           const float *Wnoise, const float *noise, const void *W1, const void *b1, const void *W2,
+                           const void *b2, const uint8_t *keep_bits, float drop_prob, const void *ctx, void *dX,
+                           float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2, void *db2, void *ws,
+                           void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED",
 EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_workspace_bytes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
            "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
-           "moe_backward"]
+           "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward"]
 
 
 class MoeError(RuntimeError):
@@ -89,7 +89,8 @@ def _stream():
 
 
 def _call(name, cfg, *tensors, stream=True):
-    args = [ctypes.byref(cfg)] + [_p(t) for t in tensors]
+    # device tensors become pointers; a Python float is a `float` argument passed by value
+    args = [ctypes.byref(cfg)] + [ctypes.c_float(t) if isinstance(t, float) else _p(t) for t in tensors]
     if stream:
         args.append(_stream())
     status = getattr(lib(), name)(*args)
@@ -189,6 +190,26 @@ def moe_forward(cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, y, losses, importance
 def moe_backward(cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2, ws):
     _call("moe_backward", cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2,
           ws)
+
+
+def moe_combine_layer(cfg, ys, gates, inv_perm, x, keep_bits, drop_prob, out):
+    _call("moe_combine_layer", cfg, ys, gates, inv_perm, x, keep_bits, float(drop_prob), out)
+
+
+def moe_combine_layer_bwd(cfg, dOut, ys, gates, inv_perm, keep_bits, drop_prob, dgates, dys):
+    _call("moe_combine_layer_bwd", cfg, dOut, ys, gates, inv_perm, keep_bits, float(drop_prob), dgates, dys)
+
+
+def moe_layer_forward(cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, drop_prob, out, losses, importance, load,
+                      counts, ctx, ws):
+    _call("moe_layer_forward", cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, float(drop_prob), out, losses,
+          importance, load, counts, ctx, ws)
+
+
+def moe_layer_backward(cfg, dOut, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, drop_prob, ctx, dX, dWg, dWnoise,
+                       dW1, db1, dW2, db2, ws):
+    _call("moe_layer_backward", cfg, dOut, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, float(drop_prob), ctx, dX,
+          dWg, dWnoise, dW1, db1, dW2, db2, ws)
 
 
 # ----------------------------------------------------------------------------------------------

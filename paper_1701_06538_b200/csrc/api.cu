@@ -83,6 +83,13 @@ bool bad_ptr(const void *p) { return p == nullptr || !aligned16(p); }
             if (bad_ptr(ps_[i_])) return MOE_ERR_INVALID_ARG;         \
     } while (0)
 
+// arguments of the layer epilogue: packed keep bits [T, d/8] and the dropout probability
+int32_t check_layer(const moe_config *c, const uint8_t *keep_bits, float drop_prob) {
+    if (bad_ptr(keep_bits) || c->d % 8 != 0) return MOE_ERR_INVALID_ARG;
+    if (!(drop_prob >= 0.0f) || !(drop_prob < 1.0f)) return MOE_ERR_INVALID_ARG;
+    return MOE_OK;
+}
+
 cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
 
 int32_t *status_word(void *ws) { return static_cast<int32_t *>(ws); }
@@ -751,11 +758,14 @@ int32_t moe_gate_bwd(const moe_config *cfg, const void *x, const float *Wg, cons
                        dload, dWg, dWnoise, dX_gate, ws, cv, as_stream(stream));
 }
 
-int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
-                    const void *W1, const void *b1, const void *W2, const void *b2, void *y, float *losses,
-                    float *importance, float *load, int32_t *counts, void *ctx, void *ws, void *stream) {
+// keep_bits != nullptr: the output is that of the layer epilogue (sigmoid, dropout, residual) instead of Eq. 1 alone
+static int32_t forward_impl(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise,
+                            const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                            const uint8_t *keep_bits, float drop_prob, void *y, float *losses, float *importance,
+                            float *load, int32_t *counts, void *ctx, void *ws, void *stream) {
     MOE_TRY(check_config(cfg));
     REQUIRE_PTRS(x, Wg, Wnoise, noise, W1, b1, W2, b2, y, losses, importance, load, counts, ctx, ws);
+    if (keep_bits) MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
     const Dims D = dims_of(cfg);
     cudaStream_t st = as_stream(stream);
     Ctx C(ctx, D);
@@ -768,7 +778,8 @@ int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const
       MOE_TRY(do_dispatch(D, x, C.topk_idx, C.xs, C.perm, C.inv_perm, C.counts, C.offsets, cv, st)); }
     { Carver cv = fresh();
       MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st)); }
-    MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st));
+    MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st,
+                           keep_bits ? x : nullptr, keep_bits, keep_bits ? 1.0f / (1.0f - drop_prob) : 1.0f));
     { Carver cv = fresh();
       MOE_TRY(do_losses(cfg, D, C.topk_idx, C.gates, C.clean, C.raw_noise, C.kth_vals, C.importance, C.load,
                         C.losses, C.perm, C.offsets, cv, st)); }
@@ -779,12 +790,30 @@ int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const
     return MOE_OK;
 }
 
-int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const float *Wg, const float *Wnoise,
-                     const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
-                     const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
-                     void *db2, void *ws, void *stream) {
+int32_t moe_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise, const float *noise,
+                    const void *W1, const void *b1, const void *W2, const void *b2, void *y, float *losses,
+                    float *importance, float *load, int32_t *counts, void *ctx, void *ws, void *stream) {
+    return forward_impl(cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, nullptr, 0.0f, y, losses, importance, load, counts,
+                        ctx, ws, stream);
+}
+
+int32_t moe_layer_forward(const moe_config *cfg, const void *x, const float *Wg, const float *Wnoise,
+                          const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                          const uint8_t *keep_bits, float drop_prob, void *out, float *losses, float *importance,
+                          float *load, int32_t *counts, void *ctx, void *ws, void *stream) {
+    if (!keep_bits) return MOE_ERR_INVALID_ARG;
+    return forward_impl(cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, drop_prob, out, losses, importance, load,
+                        counts, ctx, ws, stream);
+}
+
+static int32_t backward_impl(const moe_config *cfg, const void *dY, const void *x, const float *Wg,
+                             const float *Wnoise, const float *noise, const void *W1, const void *b1, const void *W2,
+                             const void *b2, const uint8_t *keep_bits, float drop_prob, const void *ctx, void *dX,
+                             float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2, void *db2, void *ws,
+                             void *stream) {
     MOE_TRY(check_config(cfg));
     REQUIRE_PTRS(dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2, ws);
+    if (keep_bits) MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
     const Dims D = dims_of(cfg);
     cudaStream_t st = as_stream(stream);
     Ctx C(const_cast<void *>(ctx), D);
@@ -794,7 +823,7 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
     BwdWs B(base, D);
     auto fresh = [&]() { return base; };  // stage scratch starts after the tensors that live across stages
     MOE_TRY(launch_combine_bwd(dY, C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dgates,
-                               B.dys, st));
+                               B.dys, st, keep_bits, keep_bits ? 1.0f / (1.0f - drop_prob) : 1.0f));
     { Carver cv = fresh();
       MOE_TRY(do_expert_ffn_bwd(cfg, D, C.xs, C.hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, ws, cv,
                                 st)); }
@@ -803,8 +832,46 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
     { Carver cv = fresh();
       MOE_TRY(do_gate_bwd(cfg, D, x, Wg, Wnoise, noise, C.clean, C.raw_noise, C.topk_idx, C.gates, C.kth_vals,
                           C.kth_idx, B.dgates, B.dload, dWg, dWnoise, B.dX_gate, ws, cv, st)); }
+    // dX = expert path + gating path (+ the upstream gradient itself through the residual connection)
     return launch_dispatch_bwd(B.dxs, D.act, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dX_gate, nullptr, dX,
-                               st);
+                               st, keep_bits ? dY : nullptr);
+}
+
+int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const float *Wg, const float *Wnoise,
+                     const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
+                     const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
+                     void *db2, void *ws, void *stream) {
+    return backward_impl(cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, nullptr, 0.0f, ctx, dX, dWg, dWnoise, dW1, db1,
+                         dW2, db2, ws, stream);
+}
+
+int32_t moe_layer_backward(const moe_config *cfg, const void *dOut, const void *x, const float *Wg,
+                           const float *Wnoise, const float *noise, const void *W1, const void *b1, const void *W2,
+                           const void *b2, const uint8_t *keep_bits, float drop_prob, const void *ctx, void *dX,
+                           float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2, void *db2, void *ws,
+                           void *stream) {
+    if (!keep_bits) return MOE_ERR_INVALID_ARG;
+    return backward_impl(cfg, dOut, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, drop_prob, ctx, dX, dWg, dWnoise,
+                         dW1, db1, dW2, db2, ws, stream);
+}
+
+int32_t moe_combine_layer(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm,
+                          const void *x, const uint8_t *keep_bits, float drop_prob, void *out, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(ys, gates, inv_perm, x, out);
+    MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
+    return launch_combine(ys, cfg->act, gates, inv_perm, cfg->T, cfg->k, cfg->d, out, as_stream(stream), x, keep_bits,
+                          1.0f / (1.0f - drop_prob));
+}
+
+int32_t moe_combine_layer_bwd(const moe_config *cfg, const void *dOut, const void *ys, const float *gates,
+                              const int32_t *inv_perm, const uint8_t *keep_bits, float drop_prob, float *dgates,
+                              void *dys, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(dOut, ys, gates, inv_perm, dgates, dys);
+    MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
+    return launch_combine_bwd(dOut, ys, cfg->act, gates, inv_perm, cfg->T, cfg->k, cfg->d, dgates, dys,
+                              as_stream(stream), keep_bits, 1.0f / (1.0f - drop_prob));
 }
 
 }  // extern "C"

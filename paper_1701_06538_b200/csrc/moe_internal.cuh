@@ -103,15 +103,19 @@ int32_t launch_dispatch_index(const int32_t *topk_idx, int64_t R, int32_t n, int
                               int32_t *counts, int32_t *offsets, int32_t *scratch, cudaStream_t st);
 int32_t launch_dispatch_rows(const void *x, int32_t act, int64_t T, int32_t k, int32_t d, const int32_t *inv_perm,
                              void *xs, cudaStream_t st);
+// keep != nullptr: the layer epilogue of Appendix C (sigmoid, dropout through the packed keep bits [T, d/8] with the
+// kept activations scaled by keep_scale = 1 / (1 - DropProb), residual xres added); see route.cu
 int32_t launch_combine(const void *ys, int32_t act, const float *gates, const int32_t *inv_perm, int64_t T,
-                       int32_t k, int32_t d, void *y, cudaStream_t st);
+                       int32_t k, int32_t d, void *y, cudaStream_t st, const void *xres = nullptr,
+                       const uint8_t *keep = nullptr, float keep_scale = 1.0f);
 int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const float *gates,
                            const int32_t *inv_perm, int64_t T, int32_t k, int32_t d, float *dgates, void *dys,
-                           cudaStream_t st);
+                           cudaStream_t st, const uint8_t *keep = nullptr, float keep_scale = 1.0f);
 // out_f32 = sum_s dxs[inv_perm[t*k+s]] (+ add_f32 if given); written as float or, if out_act
 // is given instead, rounded to the act type.
 int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_perm, int64_t T, int32_t k,
-                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st);
+                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st,
+                            const void *add_act = nullptr);
 // tile_prefix[e] = sum_{e' < e} ceil(count_e' / bm), e = 0..n
 int32_t launch_tile_prefix(const int32_t *offsets, int32_t n, int32_t bm, int32_t *tile_prefix, cudaStream_t st);
 

@@ -264,11 +264,22 @@ int32_t launch_dispatch_rows(const void *x, int32_t act, int64_t T, int32_t k, i
         else { CALL(8, 1); }               \
     } while (0)
 
-// y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]]   (Eq. 1), float sum in slot order
-template <typename XT, int KT, int VB>
-__global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys, const float *__restrict__ gates,
+// Dropout keep bit of column q of a token row: bit q % 8 of byte q / 8. A 16-byte vector holds VN = 8 (bf16) or 4
+// (float) consecutive columns starting at a multiple of VN: its bits are one byte, or one half of a byte.
+template <int VN> __device__ __forceinline__ uint32_t keep_bits_of(const uint8_t *row_bits, int v) {
+    return VN == 8 ? (uint32_t)row_bits[v] : ((uint32_t)row_bits[v >> 1] >> ((v & 1) * 4)) & 0xFu;
+}
+// 1 / (1 + e^-y) with the hardware exponential and reciprocal (a few 1e-7 of relative error, far inside the tolerance of
+// the float layer; the IEEE division and the full-range expf made the fused kernels arithmetic-bound)
+__device__ __forceinline__ float logistic(float y) { return __fdividef(1.0f, 1.0f + __expf(-y)); }
+
+// y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]]   (Eq. 1), float sum in slot order.
+// LAYER (Appendix C): out[t] = x[t] + keep[t] * sigmoid(y[t]) * keep_scale, y itself is not stored.
+template <typename XT, int KT, int VB, bool LAYER>
+__global__ void __launch_bounds__(256, LAYER ? 3 : 1) combine_kernel(const XT *__restrict__ ys, const float *__restrict__ gates,
                                                       const int32_t *__restrict__ inv_perm, int64_t T, int32_t k,
-                                                      int32_t d, XT *__restrict__ y) {
+                                                      int32_t d, XT *__restrict__ y, const XT *__restrict__ xres,
+                                                      const uint8_t *__restrict__ keep, float keep_scale) {
     constexpr int VN = 16 / sizeof(XT);
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -286,12 +297,18 @@ __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys,
             g[s] = (s < k && valid) ? gates[t * k + s] : 0.0f;
         }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
-            Vec16<XT> in[KT][VB];
+            Vec16<XT> in[KT][VB], xr[VB];
+            uint32_t kb[VB];
 #pragma unroll
-            for (int b = 0; b < VB; ++b)
+            for (int b = 0; b < VB; ++b) {
 #pragma unroll
                 for (int s = 0; s < KT; ++s)
                     if (s < k && v0 + 32 * b < nvec) in[s][b].raw = rowp[s][v0 + 32 * b];
+                if (LAYER && v0 + 32 * b < nvec) {
+                    xr[b].raw = reinterpret_cast<const uint4 *>(xres + t * d)[v0 + 32 * b];
+                    kb[b] = keep_bits_of<VN>(keep + t * (d / 8), v0 + 32 * b);
+                }
+            }
 #pragma unroll
             for (int b = 0; b < VB; ++b) {
                 if (v0 + 32 * b >= nvec) break;
@@ -304,6 +321,11 @@ __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys,
 #pragma unroll
                         for (int i = 0; i < VN; ++i) acc[i] = fmaf(g[s], in[s][b].get(i), acc[i]);
                     }
+                if (LAYER) {
+#pragma unroll
+                    for (int i = 0; i < VN; ++i)
+                        acc[i] = fmaf(((kb[b] >> i) & 1u) ? keep_scale : 0.0f, logistic(acc[i]), xr[b].get(i));  // a select, no branch: 0 * s + x = x
+                }
                 Vec16<XT> out;
 #pragma unroll
                 for (int i = 0; i < VN; ++i) out.set(i, acc[i]);
@@ -314,27 +336,37 @@ __global__ void __launch_bounds__(256) combine_kernel(const XT *__restrict__ ys,
 }
 
 int32_t launch_combine(const void *ys, int32_t act, const float *gates, const int32_t *inv_perm, int64_t T,
-                       int32_t k, int32_t d, void *y, cudaStream_t st) {
+                       int32_t k, int32_t d, void *y, cudaStream_t st, const void *xres, const uint8_t *keep,
+                       float keep_scale) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
-#define MOE_CALL(KT, VB)                                                                                          \
-    if (act == MOE_BF16)                                                                                          \
-        combine_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)ys, gates, inv_perm, T, k, d, (bf16 *)y); \
-    else                                                                                                          \
-        combine_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)ys, gates, inv_perm, T, k, d, (float *)y)
+#define MOE_CALL_L(KT, VB, L)                                                                                         \
+    if (act == MOE_BF16)                                                                                              \
+        combine_kernel<bf16, KT, VB, L><<<grid, 256, 0, st>>>((const bf16 *)ys, gates, inv_perm, T, k, d, (bf16 *)y,  \
+                                                              (const bf16 *)xres, keep, keep_scale);                  \
+    else                                                                                                              \
+        combine_kernel<float, KT, VB, L><<<grid, 256, 0, st>>>((const float *)ys, gates, inv_perm, T, k, d, (float *)y, \
+                                                               (const float *)xres, keep, keep_scale)
+#define MOE_CALL(KT, VB)                     \
+    if (keep) { MOE_CALL_L(KT, VB, true); }  \
+    else { MOE_CALL_L(KT, VB, false); }
     MOE_DISPATCH_KT(k, MOE_CALL);
 #undef MOE_CALL
+#undef MOE_CALL_L
     MOE_LAUNCHED();
     return MOE_OK;
 }
 
-// dgates[t,s] = <dY[t], ys[row]>,  dys[row] = gates[t,s] * dY[t]
-template <typename XT, int KT, int VB>
-__global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__ dY, const XT *__restrict__ ys,
+// dgates[t,s] = <dy[t], ys[row]>,  dys[row] = gates[t,s] * dy[t], with dy = dY, or (LAYER: adjoint of the sigmoid and
+// the dropout of Appendix C) dy = dY * keep * keep_scale * s (1 - s), s = sigmoid(y), y recomputed from the ys rows
+// this kernel gathers anyway (same order of operations as the forward, so the same y bit for bit).
+template <typename XT, int KT, int VB, bool LAYER>
+__global__ void __launch_bounds__(256, LAYER ? 3 : 1) combine_bwd_kernel(const XT *__restrict__ dY, const XT *__restrict__ ys,
                                                           const float *__restrict__ gates,
                                                           const int32_t *__restrict__ inv_perm, int64_t T,
                                                           int32_t k, int32_t d, float *__restrict__ dgates,
-                                                          XT *__restrict__ dys) {
+                                                          XT *__restrict__ dys, const uint8_t *__restrict__ keep,
+                                                          float keep_scale) {
     constexpr int VN = 16 / sizeof(XT);
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -354,10 +386,12 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
         }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
             Vec16<XT> dy[VB], in[KT][VB];
+            uint32_t kb[VB];
 #pragma unroll
             for (int b = 0; b < VB; ++b) {
                 if (v0 + 32 * b < nvec) {
                     dy[b].raw = reinterpret_cast<const uint4 *>(dY + t * d)[v0 + 32 * b];
+                    if (LAYER) kb[b] = keep_bits_of<VN>(keep + t * (d / 8), v0 + 32 * b);
 #pragma unroll
                     for (int s = 0; s < KT; ++s)
                         if (s < k) in[s][b].raw = reinterpret_cast<const uint4 *>(ys + rowo[s])[v0 + 32 * b];  // row 0 for a dropped slot
@@ -366,14 +400,28 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
 #pragma unroll
             for (int b = 0; b < VB; ++b) {
                 if (v0 + 32 * b >= nvec) break;
+                float dyv[VN];
+#pragma unroll
+                for (int i = 0; i < VN; ++i) dyv[i] = dy[b].get(i);
+                if (LAYER) {
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) {
+                        float yv = 0.0f;
+#pragma unroll
+                        for (int s = 0; s < KT; ++s)
+                            if (s < k) yv = fmaf(valid[s] ? g[s] : 0.0f, in[s][b].get(i), yv);
+                        const float sg = logistic(yv);
+                        dyv[i] = (((kb[b] >> i) & 1u) ? keep_scale : 0.0f) * (dyv[i] * (sg * (1.0f - sg)));
+                    }
+                }
 #pragma unroll
                 for (int s = 0; s < KT; ++s) {
                     if (s < k) {
                         Vec16<XT> out;
 #pragma unroll
                         for (int i = 0; i < VN; ++i) {
-                            dot[s] = fmaf(dy[b].get(i), in[s][b].get(i), dot[s]);
-                            out.set(i, g[s] * dy[b].get(i));
+                            dot[s] = fmaf(dyv[i], in[s][b].get(i), dot[s]);
+                            out.set(i, g[s] * dyv[i]);
                         }
                         if (valid[s]) reinterpret_cast<uint4 *>(dys + rowo[s])[v0 + 32 * b] = out.raw;
                     }
@@ -394,28 +442,34 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const XT *__restrict__
 
 int32_t launch_combine_bwd(const void *dY, const void *ys, int32_t act, const float *gates,
                            const int32_t *inv_perm, int64_t T, int32_t k, int32_t d, float *dgates, void *dys,
-                           cudaStream_t st) {
+                           cudaStream_t st, const uint8_t *keep, float keep_scale) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
-#define MOE_CALL(KT, VB)                                                                                             \
-    if (act == MOE_BF16)                                                                                             \
-        combine_bwd_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)dY, (const bf16 *)ys, gates, inv_perm, T, \
-                                                                k, d, dgates, (bf16 *)dys);                           \
-    else                                                                                                             \
-        combine_bwd_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)dY, (const float *)ys, gates, inv_perm, \
-                                                                 T, k, d, dgates, (float *)dys)
+#define MOE_CALL_L(KT, VB, L)                                                                                            \
+    if (act == MOE_BF16)                                                                                                 \
+        combine_bwd_kernel<bf16, KT, VB, L><<<grid, 256, 0, st>>>((const bf16 *)dY, (const bf16 *)ys, gates, inv_perm, T, \
+                                                                   k, d, dgates, (bf16 *)dys, keep, keep_scale);          \
+    else                                                                                                                 \
+        combine_bwd_kernel<float, KT, VB, L><<<grid, 256, 0, st>>>((const float *)dY, (const float *)ys, gates, inv_perm, \
+                                                                    T, k, d, dgates, (float *)dys, keep, keep_scale)
+#define MOE_CALL(KT, VB)                     \
+    if (keep) { MOE_CALL_L(KT, VB, true); }  \
+    else { MOE_CALL_L(KT, VB, false); }
     MOE_DISPATCH_KT(k, MOE_CALL);
 #undef MOE_CALL
+#undef MOE_CALL_L
     MOE_LAUNCHED();
     return MOE_OK;
 }
 
-// out[t] = sum_s dxs[inv_perm[t*k+s]] (+ add[t]); float output, or rounded to the act type
+// out[t] = sum_s dxs[inv_perm[t*k+s]] (+ add[t]) (+ add_act[t], a second addend in the act type: the gradient that
+// reaches the layer input through the residual connection); float output, or rounded to the act type
 template <typename XT, int KT, int VB>
 __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict__ dxs,
                                                            const int32_t *__restrict__ inv_perm, int64_t T,
                                                            int32_t k, int32_t d, const float *add,
-                                                           float *out_f32, XT *__restrict__ out_act) {
+                                                           float *out_f32, XT *__restrict__ out_act,
+                                                           const XT *__restrict__ add_act) {
     constexpr int VN = 16 / sizeof(XT);
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -431,7 +485,7 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
             rowp[s] = reinterpret_cast<const uint4 *>(dxs + (int64_t)(valid[s] ? row : 0) * d);
         }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
-            Vec16<XT> in[KT][VB];
+            Vec16<XT> in[KT][VB], res[VB];
             float4 addv[VB][VN / 4];
 #pragma unroll
             for (int b = 0; b < VB; ++b) {
@@ -439,6 +493,7 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
 #pragma unroll
                     for (int s = 0; s < KT; ++s)
                         if (s < k) in[s][b].raw = valid[s] ? rowp[s][v0 + 32 * b] : make_uint4(0, 0, 0, 0);
+                    if (add_act) res[b].raw = reinterpret_cast<const uint4 *>(add_act + t * d)[v0 + 32 * b];
                     if (add) {
 #pragma unroll
                         for (int q = 0; q < VN / 4; ++q)
@@ -465,6 +520,10 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
                         acc[4 * q + 2] += addv[b][q].z; acc[4 * q + 3] += addv[b][q].w;
                     }
                 }
+                if (add_act) {
+#pragma unroll
+                    for (int i = 0; i < VN; ++i) acc[i] += res[b].get(i);
+                }
                 const int64_t at = t * d + (int64_t)(v0 + 32 * b) * VN;
                 if (out_act) {
                     Vec16<XT> out;
@@ -483,16 +542,17 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
 }
 
 int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_perm, int64_t T, int32_t k,
-                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st) {
+                            int32_t d, const float *add_f32, float *out_f32, void *out_act, cudaStream_t st,
+                            const void *add_act) {
     if (T == 0) return MOE_OK;
     const unsigned grid = (unsigned)imin(cdiv(T, 8), 148 * 16);
 #define MOE_CALL(KT, VB)                                                                                              \
     if (act == MOE_BF16)                                                                                              \
         dispatch_bwd_kernel<bf16, KT, VB><<<grid, 256, 0, st>>>((const bf16 *)dxs, inv_perm, T, k, d, add_f32, out_f32, \
-                                                                 (bf16 *)out_act);                                     \
+                                                                 (bf16 *)out_act, (const bf16 *)add_act);              \
     else                                                                                                              \
         dispatch_bwd_kernel<float, KT, VB><<<grid, 256, 0, st>>>((const float *)dxs, inv_perm, T, k, d, add_f32,       \
-                                                                  out_f32, (float *)out_act)
+                                                                  out_f32, (float *)out_act, (const float *)add_act)
     MOE_DISPATCH_KT(k, MOE_CALL);
 #undef MOE_CALL
     MOE_LAUNCHED();

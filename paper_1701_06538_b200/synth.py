@@ -20,7 +20,7 @@ import numpy as np
 BASE_SEED = 0x17010653
 
 # tensor ids of the streams
-_X, _WG, _WN, _NOISE, _W1, _W2, _DY, _BETA, _WG_S, _WN_S, _NOISE_S, _B1, _B2 = range(1, 14)
+_X, _WG, _WN, _NOISE, _W1, _W2, _DY, _BETA, _WG_S, _WN_S, _NOISE_S, _B1, _B2, _KEEP = range(1, 15)
 
 
 @dataclass(frozen=True)
@@ -97,6 +97,13 @@ def make_x(w: Workload) -> np.ndarray:
 
 def make_dY(w: Workload) -> np.ndarray:
     return storage_grid(_normal(w, _DY, (w.T, w.d)), w.act)
+
+
+def make_keep_bits(w: Workload, drop_prob: float) -> np.ndarray:
+    """Dropout keep mask of the layer epilogue, packed: [T, d/8] uint8, bit (q % 8) of byte q // 8 is column q;
+    a column is kept with probability 1 - drop_prob."""
+    keep = _rng(w, _KEEP).random((w.T, w.d), dtype=np.float32) >= np.float32(drop_prob)
+    return np.packbits(keep, axis=1, bitorder="little")
 
 
 def expert_offsets(w: Workload) -> np.ndarray:
