@@ -28,7 +28,8 @@ delete-and-sort kth_excluding, and against the zero-initialisation closed form;
 hierarchical reductions to the flat layer; every backward against central finite
 differences of the forward in float64; the single-precision chain against an
 exact rational emulation; the layer epilogue (sigmoid, dropout, residual) against its
-closed forms and finite differences. The table of trained-model balance metrics in the
+closed forms and finite differences; the factored optimiser step against full Adam
+on rank-one squared gradients and its textbook limits. The table of trained-model balance metrics in the
 paper's Appendix A cannot be reproduced without the trained model: for those
 printed values parity is unpinned; the metric definitions themselves are pinned
 by the CV^2 closed forms.
@@ -530,6 +531,51 @@ def gate_h_bwd(x, Wg_p, Wn_p, noise_p, Wg_s, Wn_s, noise_s, G, LS, dgates, w_imp
             dXg[rows] += dc[rows] @ np.asarray(Wg_s[i], f64).T + dr[rows] @ np.asarray(Wn_s[i], f64).T
     return SimpleNamespace(dWg_p=out.dWg, dWn_p=out.dWnoise, dWg_s=store(dWg_s, prec),
                            dWn_s=store(dWn_s, prec), dX_gate=store(dXg, prec))
+
+
+# --------------------------------------------------------------------------------------
+# optimiser step on the expert parameters (Appendix D, "Training": the memory optimisations)
+# --------------------------------------------------------------------------------------
+def adam_factored_step(W, g, row_avg, col_avg, lr, beta2, eps, step):
+    """One step of Adam with beta1 = 0 (no first-moment estimate: the gradient itself is used) whose second-moment
+    matrix is kept only through its row-wise and column-wise averages: those two vectors are the running averages
+    (decay beta2) of the row / column means of g*g, and the matrix of estimators is taken to be their outer product
+    divided by the mean of either one. Adam's bias correction 1 - beta2^step and its epsilon outside the square root
+    are kept. W, g [rows, cols]; returns (W', row_avg', col_avg')."""
+    g = np.asarray(g, f64)
+    sq = g * g
+    row_avg = beta2 * np.asarray(row_avg, f64) + (1.0 - beta2) * sq.mean(axis=1)
+    col_avg = beta2 * np.asarray(col_avg, f64) + (1.0 - beta2) * sq.mean(axis=0)
+    mean = row_avg.mean()
+    v = np.outer(row_avg, col_avg) / mean if mean > 0 else np.zeros_like(sq)
+    v_hat = v / (1.0 - beta2 ** step)
+    W = np.asarray(W, f64) - lr * g / (np.sqrt(v_hat) + eps)
+    return W, row_avg, col_avg
+
+
+def adam_vector_step(b, g, v, lr, beta2, eps, step):
+    """The same optimiser on a vector of parameters (the expert biases): a vector has no rows and columns to
+    average over, so its second-moment estimate is kept in full (plain Adam with beta1 = 0)."""
+    g = np.asarray(g, f64)
+    v = beta2 * np.asarray(v, f64) + (1.0 - beta2) * g * g
+    b = np.asarray(b, f64) - lr * g / (np.sqrt(v / (1.0 - beta2 ** step)) + eps)
+    return b, v
+
+
+def expert_adam_factored(W1, b1, W2, b2, dW1, db1, dW2, db2, state, lr, beta2, eps, step, prec):
+    """adam_factored_step on every expert's two weight matrices and adam_vector_step on its biases.
+    state = dict(r1 [n,d], c1 [n,h], r2 [n,h], c2 [n,d], vb1 [n,h], vb2 [n,d]) (float), updated in place on a copy.
+    The parameters are rounded once to the layer's storage type, the state to float32."""
+    n = W1.shape[0]
+    out = {k_: np.array(v_, f64) for k_, v_ in state.items()}
+    nW1, nb1, nW2, nb2 = (np.zeros(a.shape, f64) for a in (W1, b1, W2, b2))
+    for e in range(n):
+        nW1[e], out["r1"][e], out["c1"][e] = adam_factored_step(W1[e], dW1[e], out["r1"][e], out["c1"][e], lr, beta2, eps, step)
+        nW2[e], out["r2"][e], out["c2"][e] = adam_factored_step(W2[e], dW2[e], out["r2"][e], out["c2"][e], lr, beta2, eps, step)
+        nb1[e], out["vb1"][e] = adam_vector_step(b1[e], db1[e], out["vb1"][e], lr, beta2, eps, step)
+        nb2[e], out["vb2"][e] = adam_vector_step(b2[e], db2[e], out["vb2"][e], lr, beta2, eps, step)
+    out = {k_: store(v_, prec) for k_, v_ in out.items()}
+    return (store(nW1, prec, True), store(nb1, prec, True), store(nW2, prec, True), store(nb2, prec, True), out)
 
 
 # --------------------------------------------------------------------------------------

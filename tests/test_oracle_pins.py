@@ -577,3 +577,55 @@ def test_layer_epilogue_backward_matches_finite_differences():
     B0 = O.backward(dOut, p["x"], p["Wg"], p["Wnoise"], p["noise"], p["W1"], p["b1"], p["W2"], p["b2"], F0, wi, wl, "f64",
                     layer=none)
     assert np.abs(B0.dW1).max() == 0 and np.abs(B0.dW2).max() == 0 and np.abs(B0.dys).max() == 0
+
+
+# ---------------------------------------------------------------- factored second-moment Adam, beta1 = 0 (Appendix D)
+def full_adam_beta1_zero(W, g, v, lr, beta2, eps, step):
+    """Textbook Adam (Kingma & Ba) with beta1 = 0 and the complete second-moment matrix."""
+    v = beta2 * v + (1 - beta2) * g * g
+    return W - lr * g / (np.sqrt(v / (1 - beta2 ** step)) + eps), v
+
+
+def test_factored_adam_is_full_adam_when_the_squared_gradient_has_rank_one():
+    g_ = rng(60)
+    rows, cols = 7, 5
+    a, b = g_.standard_normal(rows), g_.standard_normal(cols)
+    G = np.outer(a, b)            # G*G = (a*a)(b*b)^T: its row and column averages determine it completely
+    W = g_.standard_normal((rows, cols))
+    r, c, v = np.zeros(rows), np.zeros(cols), np.zeros((rows, cols))
+    for step in (1, 2, 3):
+        Wf, r, c = O.adam_factored_step(W, G, r, c, 1e-2, 0.9, 1e-8, step)
+        Wa, v = full_adam_beta1_zero(W, G, v, 1e-2, 0.9, 1e-8, step)
+        assert np.allclose(Wf, Wa, rtol=1e-12, atol=1e-14)
+        assert np.allclose(np.outer(r, c) / r.mean(), v, rtol=1e-12)
+        assert math.isclose(r.mean(), c.mean(), rel_tol=1e-13)   # "the mean of either one"
+        W = Wf
+        G = G * 1.5               # still rank one, and proportional: the running averages stay rank-one consistent
+
+
+def test_factored_adam_textbook_limits():
+    g_ = rng(61)
+    W = g_.standard_normal((4, 6))
+    # constant-magnitude gradient: v = g^2 everywhere, every entry moves by lr * sign(g) (up to eps), at every step
+    G = 0.3 * np.sign(g_.standard_normal((4, 6)))
+    r, c = np.zeros(4), np.zeros(6)
+    Wn = W
+    for step in (1, 2, 3, 4):
+        Wn, r, c = O.adam_factored_step(Wn, G, r, c, 1e-3, 0.999, 0.0, step)
+        assert np.allclose(W - Wn, step * 1e-3 * np.sign(G), rtol=1e-10)
+    # bias correction: after t identical steps the corrected estimate is exactly the squared gradient's averages
+    assert np.allclose(r / (1 - 0.999 ** 4), 0.09, rtol=1e-12) and np.allclose(c / (1 - 0.999 ** 4), 0.09, rtol=1e-12)
+    # a zero gradient leaves the parameters alone (0 / (0 + eps))
+    W0, _, _ = O.adam_factored_step(W, np.zeros_like(W), np.zeros(4), np.zeros(6), 1e-3, 0.999, 1e-8, 1)
+    assert (W0 == W).all()
+    # the approximation keeps the row and column averages of the true second-moment matrix exactly
+    G = g_.standard_normal((4, 6))
+    _, r, c = O.adam_factored_step(W, G, np.zeros(4), np.zeros(6), 1e-3, 0.0, 1e-8, 1)   # beta2 = 0: averages of G*G
+    V = np.outer(r, c) / r.mean()
+    assert np.allclose(V.mean(axis=1), (G * G).mean(axis=1), rtol=1e-12)
+    assert np.allclose(V.mean(axis=0), (G * G).mean(axis=0), rtol=1e-12)
+    # vectors: plain Adam with beta1 = 0
+    b, gb = g_.standard_normal(5), g_.standard_normal(5)
+    bn, vb = O.adam_vector_step(b, gb, np.zeros(5), 1e-2, 0.9, 1e-8, 1)
+    ba, va = full_adam_beta1_zero(b, gb, np.zeros(5), 1e-2, 0.9, 1e-8, 1)
+    assert np.allclose(bn, ba, rtol=1e-14) and np.allclose(vb, va, rtol=1e-14)
