@@ -457,6 +457,13 @@ def stage_timings(B, cfg, S, D, w, timed, K, peaks):
         calls["combine_layer_bwd"] = (lambda: B.moe_combine_layer_bwd(cfg, D["dY"], V["ys"], V["gates"], V["inv_perm"],
                                                                       keep, 0.3, dgates, dys), 0.0,
                                       (1 + 2 * k) * T * d * esz + T * d // 8 + 12 * R)
+    # the optimiser step of the paper's large models (factored second-moment Adam, beta1 = 0) on the expert parameters:
+    # timed beside the stages, not part of the step; learning rate 0 leaves the weights as they are
+    adam_state = torch.zeros(S.adam_state_elems, device="cuda")
+    adam_ws = B.empty_bytes(S.ws_adam_bytes)
+    calls["adam_factored"] = (lambda: B.moe_expert_adam_factored(cfg, D["W1"], D["b1"], D["W2"], D["b2"], D["dW1"], D["db1"],
+                                                                 D["dW2"], D["db2"], adam_state, 0.0, 0.999, 1e-8, 1, adam_ws),
+                              0.0, 4 * 2 * n * d * h * esz)
     out = {}
     for name, (fn, flop, byts) in calls.items():
         fn()

@@ -80,6 +80,11 @@ typedef struct moe_config {
 #define MOE_FLAG_GATE_SCREEN_OFF 1
 #define MOE_FLAG_GATE_SCREEN_ON 2
 #define MOE_FLAG_TC_ONE_CTA 4
+/*   MOE_FLAG_RECOMPUTE_HID    the hidden activations of the experts are not kept between moe_forward and
+ *                             moe_backward (Appendix D, memory optimisations): the context has no `hid`
+ *                             (moe_ctx_layout.hid is then meaningless, the context R*h elements smaller), the
+ *                             backward runs the first expert GEMM again (2*R*d*h extra flop) into its workspace */
+#define MOE_FLAG_RECOMPUTE_HID 8
 
 typedef struct moe_sizes {
     int64_t R;            /* T*k                                                                    */
@@ -94,6 +99,8 @@ typedef struct moe_sizes {
     int64_t ws_fwd_bytes; /* workspace of moe_forward                                               */
     int64_t ws_bwd_bytes; /* workspace of moe_backward                                              */
     int64_t ctx_bytes;    /* context written by moe_forward and read by moe_backward                */
+    int64_t adam_state_elems; /* floats of optimiser state of moe_expert_adam_factored: n * (3d + 3h)   */
+    int64_t ws_adam_bytes;    /* workspace of moe_expert_adam_factored                                  */
 } moe_sizes;
 
 /* Byte offsets, inside the context of moe_forward, of the tensors it saves (same layouts as
@@ -182,7 +189,8 @@ int32_t moe_dispatch_noalloc(const moe_config *cfg, const void *x, const int32_t
 /* Experts (Section 3.2, Appendix C): on the rows offsets[e] <= r < offsets[e+1],
  *   hid = relu(xs.W1[e] + b1[e]),  ys = hid.W2[e] + b2[e],
  * float accumulation, one rounding to the act type at hid and at ys.
- * in : xs [R,d], offsets [n+1], W1 [n,d,h], b1 [n,h], W2 [n,h,d], b2 [n,d]   out: hid [R,h], ys [R,d] */
+ * in : xs [R,d], offsets [n+1], W1 [n,d,h], b1 [n,h], W2 [n,h,d], b2 [n,d]   out: hid [R,h], ys [R,d]
+ * With MOE_FLAG_RECOMPUTE_HID `hid` may be NULL: the hidden activations then stay in the workspace. */
 int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
                        const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws,
                        void *stream);
@@ -257,6 +265,22 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
                      const float *noise, const void *W1, const void *b1, const void *W2, const void *b2,
                      const void *ctx, void *dX, float *dWg, float *dWnoise, void *dW1, void *db1, void *dW2,
                      void *db2, void *ws, void *stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Optimiser step on the expert parameters (Appendix D, "Training": the memory optimisations): Adam with
+ * beta1 = 0 (no first-moment estimate) and a factored second-moment estimate. For each expert weight matrix
+ * only the running averages (decay beta2) of the row-wise and of the column-wise means of the squared
+ * gradient are kept; the matrix of estimators is their outer product divided by the mean of the row vector.
+ * Adam's bias correction 1 - beta2^step and its epsilon outside the square root are kept:
+ *     W -= lr * g / (sqrt(row_i * col_j / mean(row) / (1 - beta2^step)) + eps)
+ * The biases (vectors) keep a full second-moment estimate. Parameters are updated IN PLACE (one rounding to
+ * the act type). `state` (moe_sizes.adam_state_elems floats, zero before the first step) holds, in this
+ * order: row [n,d] and column [n,h] averages of W1, row [n,h] and column [n,d] averages of W2, second moments
+ * of b1 [n,h] and b2 [n,d]. step >= 1 counts the calls. ws: moe_sizes.ws_adam_bytes.
+ * ------------------------------------------------------------------------------------------ */
+int32_t moe_expert_adam_factored(const moe_config *cfg, void *W1, void *b1, void *W2, void *b2, const void *dW1,
+                                 const void *db1, const void *dW2, const void *db2, float *state, float lr,
+                                 float beta2, float eps, int32_t step, void *ws, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * The layer inside the paper's models (Appendix C, "Model Architecture" and "MoE Layer Architecture"):

@@ -16,14 +16,15 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmoe_b200.so")
 
 MOE_F32, MOE_BF16 = 0, 1
-MOE_FLAG_GATE_SCREEN_OFF, MOE_FLAG_GATE_SCREEN_ON, MOE_FLAG_TC_ONE_CTA = 1, 2, 4
+MOE_FLAG_GATE_SCREEN_OFF, MOE_FLAG_GATE_SCREEN_ON, MOE_FLAG_TC_ONE_CTA, MOE_FLAG_RECOMPUTE_HID = 1, 2, 4, 8
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_UNSUPPORTED", 3: "MOE_ERR_WORKSPACE",
                 4: "MOE_ERR_CUDA", 5: "MOE_ERR_TIMEOUT"}
 
 EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_workspace_bytes", "moe_query_ctx_layout", "moe_status_string", "moe_check_status",
            "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
-           "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward"]
+           "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward",
+           "moe_expert_adam_factored"]
 
 
 class MoeError(RuntimeError):
@@ -40,7 +41,8 @@ class moe_config(ctypes.Structure):
 class moe_sizes(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int64) for name in
                 ("R", "gate_cols", "logits_elems", "gates_elems", "kth_elems", "wg_elems", "load_elems",
-                 "dload_elems", "ws_bytes", "ws_fwd_bytes", "ws_bwd_bytes", "ctx_bytes")]
+                 "dload_elems", "ws_bytes", "ws_fwd_bytes", "ws_bwd_bytes", "ctx_bytes", "adam_state_elems",
+                 "ws_adam_bytes")]
 
 
 class moe_ctx_layout(ctypes.Structure):
@@ -90,7 +92,8 @@ def _stream():
 
 def _call(name, cfg, *tensors, stream=True):
     # device tensors become pointers; a Python float is a `float` argument passed by value
-    args = [ctypes.byref(cfg)] + [ctypes.c_float(t) if isinstance(t, float) else _p(t) for t in tensors]
+    args = [ctypes.byref(cfg)] + [ctypes.c_float(t) if isinstance(t, float) else
+                                  ctypes.c_int32(t) if isinstance(t, int) else _p(t) for t in tensors]
     if stream:
         args.append(_stream())
     status = getattr(lib(), name)(*args)
@@ -192,6 +195,11 @@ def moe_backward(cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dW
           ws)
 
 
+def moe_expert_adam_factored(cfg, W1, b1, W2, b2, dW1, db1, dW2, db2, state, lr, beta2, eps, step, ws):
+    _call("moe_expert_adam_factored", cfg, W1, b1, W2, b2, dW1, db1, dW2, db2, state, float(lr), float(beta2), float(eps),
+          int(step), ws)
+
+
 def moe_combine_layer(cfg, ys, gates, inv_perm, x, keep_bits, drop_prob, out):
     _call("moe_combine_layer", cfg, ys, gates, inv_perm, x, keep_bits, float(drop_prob), out)
 
@@ -230,7 +238,7 @@ def ctx_views(cfg, ctx):
         size = torch.empty((), dtype=dtype).element_size()
         return ctx[off:off + count * size].view(dtype).view(*shape)
 
-    return dict(topk_idx=view(L.topk_idx, R, torch.int32, (T, k)),
+    views = dict(topk_idx=view(L.topk_idx, R, torch.int32, (T, k)),
                 gates=view(L.gates, S.gates_elems, torch.float32, (-1,)),
                 clean=view(L.clean, S.logits_elems, torch.float32, (-1,)),
                 raw_noise=view(L.raw_noise, S.logits_elems, torch.float32, (-1,)),
@@ -238,6 +246,9 @@ def ctx_views(cfg, ctx):
                 kth_idx=view(L.kth_idx, S.kth_elems, torch.int32, (-1, 2)),
                 xs=view(L.xs, R * d, adt, (R, d)), perm=view(L.perm, R, torch.int32, (R,)),
                 inv_perm=view(L.inv_perm, R, torch.int32, (R,)), counts=view(L.counts, n, torch.int32, (n,)),
-                offsets=view(L.offsets, n + 1, torch.int32, (n + 1,)), hid=view(L.hid, R * h, adt, (R, h)),
+                offsets=view(L.offsets, n + 1, torch.int32, (n + 1,)),
                 ys=view(L.ys, R * d, adt, (R, d)), importance=view(L.importance, n, torch.float32, (n,)),
                 load=view(L.load, S.load_elems, torch.float32, (-1,)), losses=view(L.losses, 2, torch.float32, (2,)))
+    if not cfg.flags & MOE_FLAG_RECOMPUTE_HID:  # with the flag the context keeps no hidden activations
+        views["hid"] = view(L.hid, R * h, adt, (R, h))
+    return views

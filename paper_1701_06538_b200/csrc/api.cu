@@ -42,7 +42,8 @@ int32_t check_config(const moe_config *c) {
         return MOE_ERR_INVALID_ARG;
     }
     if (!(c->w_importance >= 0.0f) || !(c->w_load >= 0.0f)) return MOE_ERR_INVALID_ARG;
-    if (c->flags & ~(MOE_FLAG_GATE_SCREEN_OFF | MOE_FLAG_GATE_SCREEN_ON | MOE_FLAG_TC_ONE_CTA)) return MOE_ERR_INVALID_ARG;
+    if (c->flags & ~(MOE_FLAG_GATE_SCREEN_OFF | MOE_FLAG_GATE_SCREEN_ON | MOE_FLAG_TC_ONE_CTA | MOE_FLAG_RECOMPUTE_HID))
+        return MOE_ERR_INVALID_ARG;
     if ((c->flags & MOE_FLAG_GATE_SCREEN_OFF) && (c->flags & MOE_FLAG_GATE_SCREEN_ON)) return MOE_ERR_INVALID_ARG;
     return MOE_OK;
 }
@@ -164,9 +165,11 @@ struct DispatchWs {
 struct FfnWs {
     int32_t *tile_prefix;
     void *tc;
+    void *hid;  // MOE_FLAG_RECOMPUTE_HID: the hidden activations live here instead of in a buffer that is kept
     FfnWs(Carver &cv, const Dims &D, const moe_config *c) {
         tile_prefix = cv.take<int32_t>(D.n + 1);
         tc = tc_ffn_supported(*c) ? cv.take_bytes(tc_ffn_ws_bytes(*c)) : nullptr;
+        hid = (D.flags & MOE_FLAG_RECOMPUTE_HID) ? cv.take_bytes(D.R * D.h * (int64_t)D.esz) : nullptr;
     }
 };
 
@@ -290,7 +293,7 @@ struct Ctx {
         off.inv_perm = at(); inv_perm = cv.take<int32_t>(D.R);
         off.counts = at(); counts = cv.take<int32_t>(D.n);
         off.offsets = at(); offsets = cv.take<int32_t>(D.n + 1);
-        off.hid = at(); hid = cv.take_bytes(D.R * D.h * (int64_t)D.esz);
+        off.hid = at(); hid = (D.flags & MOE_FLAG_RECOMPUTE_HID) ? nullptr : cv.take_bytes(D.R * D.h * (int64_t)D.esz);
         off.ys = at(); ys = cv.take_bytes(D.R * D.d * (int64_t)D.esz);
         off.importance = at(); importance = cv.take<float>(D.n);
         off.load = at(); load = cv.take<float>(D.load);
@@ -392,16 +395,22 @@ SimtGemm base_gemm(const Dims &D) {
     return g;
 }
 
+// hid == nullptr (only with MOE_FLAG_RECOMPUTE_HID): the hidden activations stay in the workspace.
+// first_only: only hid = relu(xs.W1 + b1) is computed (ys is not touched).
 int32_t do_expert_ffn(const moe_config *c, const Dims &D, const void *xs, const int32_t *offsets, const void *W1,
                       const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws_base,
-                      Carver &cv, cudaStream_t st) {
+                      Carver &cv, cudaStream_t st, bool first_only = false, void **hid_used = nullptr) {
     FfnWs w(cv, D, c);
-    if (w.tc) return launch_tc_ffn(*c, xs, offsets, W1, b1, W2, b2, hid, ys, w.tc, status_word(ws_base), st);
+    if (!hid) hid = w.hid;
+    if (!hid) return MOE_ERR_INVALID_ARG;
+    if (hid_used) *hid_used = hid;
+    if (w.tc) return launch_tc_ffn(*c, xs, offsets, W1, b1, W2, b2, hid, ys, w.tc, status_word(ws_base), st, first_only);
     SimtGemm g = base_gemm(D);  // hid = relu(xs.W1 + b1)
     g.A = xs; g.B = W1; g.C = hid; g.bias = b1; g.relu = 1;
     g.sa_i = D.d; g.sa_k = 1; g.sb_k = D.h; g.sb_j = 1; g.sc_i = D.h; g.sc_j = 1;
     g.mode = 0; g.offsets = offsets; g.nseg = (int32_t)D.n; g.M = D.R; g.N = D.h; g.K = D.d; g.b_e = D.d * D.h;
     MOE_TRY(launch_simt_gemm(g, w.tile_prefix, st));
+    if (first_only) return MOE_OK;
     g = base_gemm(D);  // ys = hid.W2 + b2
     g.A = hid; g.B = W2; g.C = ys; g.bias = b2;
     g.sa_i = D.h; g.sa_k = 1; g.sb_k = D.d; g.sb_j = 1; g.sc_i = D.d; g.sc_j = 1;
@@ -626,6 +635,10 @@ int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *out) {
     int64_t stage_bwd = s_fbwd;
     if (s_lbwd > stage_bwd) stage_bwd = s_lbwd;
     if (s_gbwd > stage_bwd) stage_bwd = s_gbwd;
+    const int64_t s_fbwd_recompute = measure([&](Carver &cv) { FfnBwdWs w(cv, D); FfnWs f(cv, D, cfg); (void)w; (void)f; });
+    if ((D.flags & MOE_FLAG_RECOMPUTE_HID) && s_fbwd_recompute > stage_bwd) stage_bwd = s_fbwd_recompute;
+    out->adam_state_elems = D.n * (3 * D.d + 3 * D.h);
+    out->ws_adam_bytes = kWsHeader + ((adam_ws_floats((int32_t)D.n, (int32_t)D.d, (int32_t)D.h) * 4 + 255) & ~(int64_t)255);
     out->ws_bytes = fwd > stage_bwd ? fwd : stage_bwd;
     out->ws_fwd_bytes = fwd;
     out->ws_bwd_bytes = measure([&](Carver &cv) { BwdWs w(cv, D); (void)w; }) + stage_bwd;
@@ -677,7 +690,8 @@ int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *off
                        const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws,
                        void *stream) {
     MOE_TRY(check_config(cfg));
-    REQUIRE_PTRS(xs, offsets, W1, b1, W2, b2, hid, ys, ws);
+    REQUIRE_PTRS(xs, offsets, W1, b1, W2, b2, ys, ws);
+    if (hid ? !aligned16(hid) : !(cfg->flags & MOE_FLAG_RECOMPUTE_HID)) return MOE_ERR_INVALID_ARG;
     const Dims D = dims_of(cfg);
     Carver cv(ws);
     cv.take_bytes(kWsHeader);
@@ -777,7 +791,7 @@ static int32_t forward_impl(const moe_config *cfg, const void *x, const float *W
     { Carver cv = fresh();
       MOE_TRY(do_dispatch(D, x, C.topk_idx, C.xs, C.perm, C.inv_perm, C.counts, C.offsets, cv, st)); }
     { Carver cv = fresh();
-      MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st)); }
+      MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st)); }  // C.hid null: stays in ws
     MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st,
                            keep_bits ? x : nullptr, keep_bits, keep_bits ? 1.0f / (1.0f - drop_prob) : 1.0f));
     { Carver cv = fresh();
@@ -825,7 +839,16 @@ static int32_t backward_impl(const moe_config *cfg, const void *dY, const void *
     MOE_TRY(launch_combine_bwd(dY, C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, B.dgates,
                                B.dys, st, keep_bits, keep_bits ? 1.0f / (1.0f - drop_prob) : 1.0f));
     { Carver cv = fresh();
-      MOE_TRY(do_expert_ffn_bwd(cfg, D, C.xs, C.hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, ws, cv,
+      const void *hid = C.hid;
+      if (!hid) {  // MOE_FLAG_RECOMPUTE_HID: the forward kept no hidden activations; the first GEMM is run again
+          FfnBwdWs skip(cv, D);  // the expert backward's own scratch comes first, the recomputed tensor behind it
+          (void)skip;
+          void *again = nullptr;
+          MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, nullptr, nullptr, ws, cv, st, true, &again));
+          hid = again;
+          cv = fresh();
+      }
+      MOE_TRY(do_expert_ffn_bwd(cfg, D, C.xs, hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, ws, cv,
                                 st)); }
     { Carver cv = fresh();
       MOE_TRY(do_losses_bwd(cfg, D, C.importance, C.load, C.topk_idx, B.dgates, B.dload, cv, st)); }
@@ -853,6 +876,16 @@ int32_t moe_layer_backward(const moe_config *cfg, const void *dOut, const void *
     if (!keep_bits) return MOE_ERR_INVALID_ARG;
     return backward_impl(cfg, dOut, x, Wg, Wnoise, noise, W1, b1, W2, b2, keep_bits, drop_prob, ctx, dX, dWg, dWnoise,
                          dW1, db1, dW2, db2, ws, stream);
+}
+
+int32_t moe_expert_adam_factored(const moe_config *cfg, void *W1, void *b1, void *W2, void *b2, const void *dW1,
+                                 const void *db1, const void *dW2, const void *db2, float *state, float lr,
+                                 float beta2, float eps, int32_t step, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(W1, b1, W2, b2, dW1, db1, dW2, db2, state, ws);
+    if (!(lr >= 0.0f) || !(beta2 >= 0.0f) || !(beta2 < 1.0f) || !(eps >= 0.0f) || step < 1) return MOE_ERR_INVALID_ARG;
+    return launch_expert_adam(cfg->act, cfg->n, cfg->d, cfg->h, W1, b1, W2, b2, dW1, db1, dW2, db2, state, lr, beta2, eps,
+                              step, reinterpret_cast<float *>(static_cast<char *>(ws) + kWsHeader), as_stream(stream));
 }
 
 int32_t moe_combine_layer(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm,

@@ -1651,10 +1651,11 @@ int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int3
 
 int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
-                      cudaStream_t st) {
+                      cudaStream_t st, bool first_only) {
     const int64_t R = (int64_t)c.T * c.k;
     int32_t *tile_prefix = static_cast<int32_t *>(ws);
     MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st, c.flags));
+    if (first_only) return MOE_OK;
     return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
 

@@ -196,9 +196,16 @@ int32_t launch_segment_colsum(const void *in, int32_t act, const int32_t *offset
 // ----------------------------------------------------------------------------- tensor-core experts (ffn_tc.cu)
 bool tc_ffn_supported(const moe_config &c);
 int64_t tc_ffn_ws_bytes(const moe_config &c);
+// first_only: only hid = relu(xs.W1 + b1) (the recomputation of the hidden activations in the backward pass)
 int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
-                      cudaStream_t st);
+                      cudaStream_t st, bool first_only = false);
+
+// ----------------------------------------------------------------------------- optimiser step (optim.cu)
+int64_t adam_ws_floats(int32_t n, int32_t d, int32_t h);
+int32_t launch_expert_adam(int32_t act, int32_t n, int32_t d, int32_t h, void *W1, void *b1, void *W2, void *b2,
+                           const void *dW1, const void *db1, const void *dW2, const void *db2, float *state, float lr,
+                           float beta2, float eps, int32_t step, float *ws, cudaStream_t st);
 
 bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n);
 int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n);  // floats of partial-sum scratch

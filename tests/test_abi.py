@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.moe_config) == 52
-    assert ctypes.sizeof(B.moe_sizes) == 12 * 8
+    assert ctypes.sizeof(B.moe_sizes) == 14 * 8
     assert ctypes.sizeof(B.moe_ctx_layout) == 16 * 8
 
 
@@ -48,7 +48,7 @@ def test_validate_accepts_the_five_workloads_and_rejects_bad_ones(lib):
     ok = dict(T=16, d=64, h=64, n=8, k=2, act="f32")
     bad = [dict(ok, k=0), dict(ok, k=9), dict(ok, k=3, n=2), dict(ok, d=3), dict(ok, h=0), dict(ok, T=-1),
            dict(ok, act=7), dict(ok, n=1 << 20), dict(ok, a=2, b=3, k1=1, k2=1), dict(ok, a=2, b=4, k1=2, k2=2),
-           dict(ok, d=4, act="bf16"), dict(ok, w_load=-1.0), dict(ok, flags=8),
+           dict(ok, d=4, act="bf16"), dict(ok, w_load=-1.0), dict(ok, flags=16),
            dict(ok, flags=B.MOE_FLAG_GATE_SCREEN_ON | B.MOE_FLAG_GATE_SCREEN_OFF)]
     for kw in bad:
         assert B.moe_validate(B.make_config(**kw)) == 1, kw
