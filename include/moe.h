@@ -8,9 +8,14 @@
  *  - Every pointer is a DEVICE pointer except `const moe_config*`, `moe_sizes*`,
  *    `moe_ctx_layout*` and pointers whose name starts with `host_`.
  *  - The caller owns every buffer (inputs, outputs, workspace, context). The library never
- *    allocates or frees device memory, keeps no state between calls and never synchronises
- *    the host with the device (except moe_check_status, which says so). All work is enqueued
+ *    allocates or frees device memory and never synchronises the host with the device (except
+ *    moe_check_status and moe_debug_bounds_violations, which say so). It keeps no state between
+ *    calls, with three small exceptions: a host-side launch counter (diagnostics), function
+ *    attributes set on a kernel's first launch, and moe_dispatch_noalloc (see there: a fixed
+ *    scratch array inside the library's device image and its cached address). All work is enqueued
  *    on `stream` (a cudaStream_t passed as void*; NULL is the default stream).
+ *  - `ws` and `ctx` are bare pointers: a buffer that is too small cannot be detected by the call it
+ *    is passed to. moe_query_sizes gives the sizes, moe_check_buffer_sizes checks one.
  *  - Tensors are row-major, contiguous, and start on a 32-byte boundary (256-byte for the
  *    workspace and the context). Outputs are overwritten, not accumulated into.
  *  - "act" tensors (x, xs, hid, ys, y, W1, b1, W2, b2 and their gradients) have the element
@@ -126,6 +131,29 @@ const char *moe_status_string(int32_t status);
  * (a host-side counter; the one piece of process-wide state the library keeps). */
 int64_t moe_debug_launch_count(void);
 
+/* Is a buffer of `bytes` bytes large enough for its role with this configuration? MOE_OK, or MOE_ERR_WORKSPACE.
+ * The calls themselves take `ws` / `ctx` as bare pointers and cannot see a short buffer: check here first. */
+typedef enum {
+    MOE_BUF_WS_STAGE = 0,    /* ws of any stage call (moe_sizes.ws_bytes)     */
+    MOE_BUF_WS_FORWARD = 1,  /* ws of moe_forward / moe_layer_forward         */
+    MOE_BUF_WS_BACKWARD = 2, /* ws of moe_backward / moe_layer_backward       */
+    MOE_BUF_CONTEXT = 3,     /* ctx of the fused calls                        */
+    MOE_BUF_WS_ADAM = 4      /* ws of moe_expert_adam_factored                */
+} moe_buffer_role;
+int32_t moe_check_buffer_sizes(const moe_config *cfg, int32_t which, size_t bytes);
+
+/* Diagnostics: enqueues a one-thread kernel that waits, with the bounded-wait helper of the tensor-core kernels, for
+ * limit_ns nanoseconds (at most 1e8) on a barrier nobody signals, gives up, and leaves MOE_ERR_TIMEOUT in the status
+ * word of `ws` (read it with moe_check_status). Nothing else is outstanding in that kernel: it returns normally and the
+ * context stays usable. Exists so that the expiry path can be tested without starving a real kernel. */
+int32_t moe_debug_wait_timeout(void *ws, int64_t limit_ns, void *stream);
+
+/* Diagnostics: in the checking build of the library (compiled with -DMOE_BOUNDS_CHECK) the number of values read
+ * from memory that were about to be used as an index outside their range, over all kernels so far (such accesses are
+ * skipped in every build; the checking build also counts them). Always 0 in the regular build; -1 on a CUDA error.
+ * Synchronises the device. */
+int64_t moe_debug_bounds_violations(void);
+
 /* Synchronises `stream`, then reads the status word the kernels of the last call that used
  * `ws` left there. MOE_OK, or MOE_ERR_TIMEOUT if a bounded wait inside a tensor-core kernel
  * gave up (its outputs are then undefined; the context stays usable). */
@@ -177,7 +205,9 @@ int32_t moe_dispatch(const moe_config *cfg, const void *x, const int32_t *topk_i
  *  - Limit: ceil(T*k / 1024) * n + 64 <= MOE_NOALLOC_SCRATCH_INTS, else MOE_ERR_WORKSPACE is
  *    returned and nothing is launched (e.g. T*k = 262144 rows with up to 4096 experts fit).
  *  - The first call on each device looks up the array's device address (with that device
- *    current); make that first call before starting any stream capture.
+ *    current) and keeps it; make that first call before starting any stream capture. The kept
+ *    address belongs to the device's primary context: after a cudaDeviceReset of that device it
+ *    is stale and this entry point must not be called again in the process.
  *  - All calls in the process share the array, which keeps whatever the last call left there
  *    (the kernels overwrite every word before reading it, so nothing needs clearing). Two
  *    calls that overlap on the GPU -- different streams, or different host threads -- race on

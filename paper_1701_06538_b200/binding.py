@@ -24,7 +24,7 @@ EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_wor
            "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward",
-           "moe_expert_adam_factored"]
+           "moe_expert_adam_factored", "moe_check_buffer_sizes", "moe_debug_wait_timeout", "moe_debug_bounds_violations"]
 
 
 class MoeError(RuntimeError):
@@ -58,14 +58,16 @@ def lib():
     """The loaded shared library. Raises if it was not built (python -m paper_1701_06538_b200.build)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1701_06538_b200.build`; "
+        path = os.environ.get("MOE_B200_LIB", LIB_PATH)  # e.g. the checking build (libmoe_b200_check.so), for the test that runs it
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with `python -m paper_1701_06538_b200.build`; "
                               "there is no fallback path")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         for name in EXPORTS:
             getattr(L, name).restype = ctypes.c_int32
         L.moe_status_string.restype = ctypes.c_char_p
         L.moe_debug_launch_count.restype = ctypes.c_int64
+        L.moe_debug_bounds_violations.restype = ctypes.c_int64
         _lib = L
     return _lib
 
@@ -132,6 +134,20 @@ def moe_query_ctx_layout(cfg) -> moe_ctx_layout:
     if status != 0:
         raise MoeError("moe_query_ctx_layout", status)
     return out
+
+
+def moe_check_buffer_sizes(cfg, which, nbytes) -> int:
+    return lib().moe_check_buffer_sizes(ctypes.byref(cfg), ctypes.c_int32(which), ctypes.c_size_t(nbytes))
+
+
+def moe_debug_wait_timeout(ws, limit_ns):
+    status = lib().moe_debug_wait_timeout(_p(ws), ctypes.c_int64(limit_ns), _stream())
+    if status:
+        raise MoeError("moe_debug_wait_timeout", status)
+
+
+def moe_debug_bounds_violations() -> int:
+    return int(lib().moe_debug_bounds_violations())
 
 
 def moe_check_status(ws) -> int:

@@ -189,7 +189,7 @@ struct HierIdxWs {
         tile_prefix = cv.take<int32_t>(tc_tile_ws_ints(D.T * D.k1, D.a));  // prefix + tile table of the secondary-gate GEMMs
     }
     int32_t build(const Dims &D, const int32_t *topk_idx, cudaStream_t st) {
-        MOE_TRY(launch_hier_split_idx(topk_idx, D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.b, idx_p, idx_s, st));
+        MOE_TRY(launch_hier_split_idx(topk_idx, D.T, (int32_t)D.k1, (int32_t)D.k2, (int32_t)D.a, (int32_t)D.b, idx_p, idx_s, st));
         return launch_dispatch_index(idx_p, D.T * D.k1, (int32_t)D.a, perm_p, inv_perm_p, counts_p, offsets_p, scratch,
                                      st);
     }
@@ -487,7 +487,7 @@ int32_t do_losses_bwd(const moe_config *c, const Dims &D, const float *importanc
         return launch_losses_bwd_flat(importance, load, (int32_t)D.n, topk_idx, D.R, c->w_importance, c->w_load,
                                       dgates, dload, w.dimp, st);
     MOE_TRY(launch_cv2_grad(importance, (int32_t)D.n, c->w_importance, w.dimp, st));
-    MOE_TRY(launch_add_gathered(dgates, topk_idx, w.dimp, D.R, st));
+    MOE_TRY(launch_add_gathered(dgates, topk_idx, w.dimp, D.R, (int32_t)D.n, st));
     MOE_TRY(launch_cv2_grad(load, (int32_t)D.n, c->w_load, w.dload_h, st));  // load[0 : a*b] is Load_H
     return launch_load_h_bwd(load, w.dload_h, (int32_t)D.a, (int32_t)D.b, dload, st);
 }
@@ -653,6 +653,38 @@ int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *out) {
     Ctx ctx(nullptr, dims_of(cfg));
     *out = ctx.off;
     return MOE_OK;
+}
+
+int64_t moe_debug_bounds_violations(void) {
+    const unsigned long long parts[] = {bounds_violations_route(), bounds_violations_losses(), bounds_violations_hier(),
+                                        bounds_violations_gate(), bounds_violations_ffn()};
+    unsigned long long sum = 0;
+    for (unsigned long long v : parts) {
+        if (v == ~0ull) return -1;
+        sum += v;
+    }
+    return (int64_t)sum;
+}
+
+int32_t moe_debug_wait_timeout(void *ws, int64_t limit_ns, void *stream) {
+    if (bad_ptr(ws) || limit_ns < 0 || limit_ns > 100000000) return MOE_ERR_INVALID_ARG;  // at most 0.1 s
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return launch_debug_wait(status_word(ws), (unsigned long long)limit_ns, as_stream(stream));
+}
+
+int32_t moe_check_buffer_sizes(const moe_config *cfg, int32_t which, size_t bytes) {
+    moe_sizes s;
+    MOE_TRY(moe_query_sizes(cfg, &s));
+    int64_t need;
+    switch (which) {
+        case MOE_BUF_WS_STAGE: need = s.ws_bytes; break;
+        case MOE_BUF_WS_FORWARD: need = s.ws_fwd_bytes; break;
+        case MOE_BUF_WS_BACKWARD: need = s.ws_bwd_bytes; break;
+        case MOE_BUF_CONTEXT: need = s.ctx_bytes; break;
+        case MOE_BUF_WS_ADAM: need = s.ws_adam_bytes; break;
+        default: return MOE_ERR_INVALID_ARG;
+    }
+    return (int64_t)bytes >= need ? MOE_OK : MOE_ERR_WORKSPACE;
 }
 
 int32_t moe_check_status(const void *ws, void *stream) {

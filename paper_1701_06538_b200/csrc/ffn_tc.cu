@@ -140,18 +140,22 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // Bounded wait. Returns false (and raises the CTA's abort flag + the status word) on expiry.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                                unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        if (global_ns() - t0 > limit_ns) {
             *abort_flag = 1;
             atomicExch(status, (int32_t)MOE_ERR_TIMEOUT);
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+    return mbar_wait_limit(bar, parity, abort_flag, status, WAIT_LIMIT_NS);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1) {
@@ -366,6 +370,7 @@ __device__ __forceinline__ bool tile_decode(const GemmParams &p, int32_t id, con
             return true;
         }
         if (raw.x < 0) return false;  // past the last M tile
+        MOE_BOUNDS_NOTE(raw.x < p.nseg && raw.y >= 0 && raw.y <= raw.z && (int64_t)raw.z <= p.R);
         t.e = raw.x;
         t.row0 = raw.y;
         t.row_end = raw.z;
@@ -813,6 +818,7 @@ template <int KIND> struct PairTiles {
         if (arrives) mbar_arrive_leader_relaxed(empty0 + 8u * slot);
         ++i;
         if (rec.x < 0) return false;
+        MOE_BOUNDS_NOTE(rec.x < p.nseg && rec.y >= 0 && rec.y <= rec.z && (int64_t)rec.z <= p.R);
         t.e = rec.x; t.row0 = rec.y; t.row_end = rec.z;
         const int32_t grp = rec.w / p.sched_group, rem = rec.w - grp * p.sched_group;  // rec.w: the tile id
         if (KIND == WGRAD) {
@@ -1877,6 +1883,28 @@ int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, 
     MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st, c.flags, tile_prefix));
     return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
+
+// ------------------------------------------------------------------------------------------
+// The expiry path of the bounded waits, exercised on its own: one thread waits, with the helper the GEMM kernels use,
+// on an mbarrier nobody arrives at. Nothing asynchronous is outstanding (no copy, no MMA, no tensor memory), so the
+// kernel simply returns once the limit has passed and leaves MOE_ERR_TIMEOUT in the status word.
+// ------------------------------------------------------------------------------------------
+__global__ void debug_wait_kernel(int32_t *status, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait_limit(smem_u32(&bar), 0, &abort_flag, status, limit_ns);
+}
+
+int32_t launch_debug_wait(int32_t *status, unsigned long long limit_ns, cudaStream_t st) {
+    debug_wait_kernel<<<1, 1, 0, st>>>(status, limit_ns);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
+MOE_BOUNDS_READER(bounds_violations_ffn)
 
 }  // namespace moe
 

@@ -767,4 +767,6 @@ int32_t launch_hier_merge(int64_t T, int32_t k1, int32_t k2, int32_t b, const in
     return MOE_OK;
 }
 
+MOE_BOUNDS_READER(bounds_violations_gate)
+
 }  // namespace moe

@@ -5,20 +5,22 @@
 namespace moe {
 
 // idx_p[t, s1] = group of primary slot s1; idx_s[p, s2] = expert inside that group
-__global__ void hier_split_idx_kernel(const int32_t *__restrict__ topk_idx, int64_t total, int32_t k2, int32_t b,
-                                      int32_t *__restrict__ idx_p, int32_t *__restrict__ idx_s) {
+__global__ void hier_split_idx_kernel(const int32_t *__restrict__ topk_idx, int64_t total, int32_t k2, int32_t a,
+                                      int32_t b, int32_t *__restrict__ idx_p, int32_t *__restrict__ idx_s) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // over T*k1*k2
     if (i >= total) return;
-    const int32_t id = topk_idx[i];
+    int32_t id = topk_idx[i];
+    MOE_BOUNDS_NOTE((uint32_t)id < (uint32_t)(a * b));
+    if ((uint32_t)id >= (uint32_t)(a * b)) id = 0;  // a caller's bad id: the group index below stays inside its tables
     idx_s[i] = id % b;
     if (i % k2 == 0) idx_p[i / k2] = id / b;
 }
 
-int32_t launch_hier_split_idx(const int32_t *topk_idx, int64_t T, int32_t k1, int32_t k2, int32_t b, int32_t *idx_p,
-                              int32_t *idx_s, cudaStream_t st) {
+int32_t launch_hier_split_idx(const int32_t *topk_idx, int64_t T, int32_t k1, int32_t k2, int32_t a, int32_t b,
+                              int32_t *idx_p, int32_t *idx_s, cudaStream_t st) {
     const int64_t total = T * k1 * k2;
     if (total == 0) return MOE_OK;
-    hier_split_idx_kernel<<<(unsigned)cdiv(total, 256), 256, 0, st>>>(topk_idx, total, k2, b, idx_p, idx_s);
+    hier_split_idx_kernel<<<(unsigned)cdiv(total, 256), 256, 0, st>>>(topk_idx, total, k2, a, b, idx_p, idx_s);
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -209,5 +211,7 @@ int32_t launch_add_slot_rows(const float *dX_sec, int64_t T, int32_t k1, int32_t
     MOE_LAUNCHED();
     return MOE_OK;
 }
+
+MOE_BOUNDS_READER(bounds_violations_hier)
 
 }  // namespace moe

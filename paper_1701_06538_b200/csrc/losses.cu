@@ -222,9 +222,13 @@ __global__ void __launch_bounds__(256) cv2_grad_kernel(const float *v, int32_t m
         out[i] = (float)((double)scale * c * (((double)v[i] - a.mu) - a.var / a.mu));
 }
 
-__global__ void add_gathered_kernel(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R) {
+// dgates[p] += dimp[topk_idx[p]]; an expert id outside [0, n) adds nothing
+__global__ void add_gathered_kernel(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, int32_t n) {
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p < R) dgates[p] += dimp[topk_idx[p]];
+    if (p >= R) return;
+    const int32_t e = topk_idx[p];
+    MOE_BOUNDS_NOTE((uint32_t)e < (uint32_t)n);
+    if ((uint32_t)e < (uint32_t)n) dgates[p] += dimp[e];
 }
 
 int32_t launch_cv2_grad(const float *v, int32_t m, float scale, float *out, cudaStream_t st) {
@@ -233,9 +237,10 @@ int32_t launch_cv2_grad(const float *v, int32_t m, float scale, float *out, cuda
     return MOE_OK;
 }
 
-int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, cudaStream_t st) {
+int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, int32_t n,
+                            cudaStream_t st) {
     if (R == 0) return MOE_OK;
-    add_gathered_kernel<<<(unsigned)cdiv(R, 256), 256, 0, st>>>(dgates, topk_idx, dimp, R);
+    add_gathered_kernel<<<(unsigned)cdiv(R, 256), 256, 0, st>>>(dgates, topk_idx, dimp, R, n);
     MOE_LAUNCHED();
     return MOE_OK;
 }
@@ -248,10 +253,12 @@ int32_t launch_losses_bwd_flat(const float *importance, const float *load, int32
     cv2_grad_kernel<<<1, 256, 0, st>>>(load, n, w_load, dload);
     MOE_LAUNCHED();
     if (R > 0) {
-        add_gathered_kernel<<<(unsigned)cdiv(R, 256), 256, 0, st>>>(dgates, topk_idx, dimp_tmp, R);
+        add_gathered_kernel<<<(unsigned)cdiv(R, 256), 256, 0, st>>>(dgates, topk_idx, dimp_tmp, R, n);
         MOE_LAUNCHED();
     }
     return MOE_OK;
 }
+
+MOE_BOUNDS_READER(bounds_violations_losses)
 
 }  // namespace moe

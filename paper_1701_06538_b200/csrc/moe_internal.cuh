@@ -24,9 +24,34 @@
         if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA; /* consumed: reported once */ \
     } while (0)
 
+// Checking build (-DMOE_BOUNDS_CHECK, the stand-in for a memory checker): every place where a value read from memory
+// becomes an index reports a value outside its range to a counter of the translation unit (never a trap; the access
+// itself is skipped by the guards that are always compiled in). moe_debug_bounds_violations adds the counters up.
+#ifdef MOE_BOUNDS_CHECK
+static __device__ unsigned long long g_tu_bounds_violations = 0ull;
+#define MOE_BOUNDS_NOTE(ok)                                                  \
+    do {                                                                     \
+        if (!(ok)) atomicAdd(&g_tu_bounds_violations, 1ull);                 \
+    } while (0)
+#define MOE_BOUNDS_READER(fn)                                                                                   \
+    unsigned long long fn() {                                                                                   \
+        unsigned long long v = 0;                                                                               \
+        return cudaMemcpyFromSymbol(&v, g_tu_bounds_violations, sizeof(v)) == cudaSuccess ? v : ~0ull;          \
+    }
+#else
+#define MOE_BOUNDS_NOTE(ok) do {} while (0)
+#define MOE_BOUNDS_READER(fn) unsigned long long fn() { return 0ull; }
+#endif
+
 namespace moe {
 
 void count_launch();  // diagnostics: kernels launched by this library so far (api.cu)
+// per translation unit: out-of-range indices seen by the checking build (0 in the regular build)
+unsigned long long bounds_violations_route();
+unsigned long long bounds_violations_losses();
+unsigned long long bounds_violations_hier();
+unsigned long long bounds_violations_gate();
+unsigned long long bounds_violations_ffn();
 
 typedef __nv_bfloat16 bf16;
 
@@ -134,8 +159,8 @@ int32_t launch_losses_bwd_flat(const float *importance, const float *load, int32
                                cudaStream_t st);
 
 // ----------------------------------------------------------------------------- hierarchical pieces (hier.cu)
-int32_t launch_hier_split_idx(const int32_t *topk_idx, int64_t T, int32_t k1, int32_t k2, int32_t b, int32_t *idx_p,
-                              int32_t *idx_s, cudaStream_t st);
+int32_t launch_hier_split_idx(const int32_t *topk_idx, int64_t T, int32_t k1, int32_t k2, int32_t a, int32_t b,
+                              int32_t *idx_p, int32_t *idx_s, cudaStream_t st);
 int32_t launch_segment_sum(const float *vals, const int32_t *perm, const int32_t *offsets, int32_t nseg, float *out,
                            cudaStream_t st);
 int64_t grouped_sums_ws_floats(int64_t rows, int32_t nseg, int32_t n);
@@ -149,7 +174,8 @@ int32_t launch_hier_gate_product_bwd(const float *gates, float *dgates, int64_t 
                                      cudaStream_t st);
 int32_t launch_add_slot_rows(const float *dX_sec, int64_t T, int32_t k1, int32_t d, float *dX_gate, cudaStream_t st);
 int32_t launch_cv2_grad(const float *v, int32_t m, float scale, float *out, cudaStream_t st);
-int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, cudaStream_t st);
+int32_t launch_add_gathered(float *dgates, const int32_t *topk_idx, const float *dimp, int64_t R, int32_t n,
+                            cudaStream_t st);
 
 // ----------------------------------------------------------------------------- gate backward (gate_bwd.cu)
 // dclean, draw [rows, n] from the saved gate tensors; dload_row_stride = 0 broadcasts dload [n].
@@ -200,6 +226,8 @@ int64_t tc_ffn_ws_bytes(const moe_config &c);
 int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
                       cudaStream_t st, bool first_only = false);
+
+int32_t launch_debug_wait(int32_t *status, unsigned long long limit_ns, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- optimiser step (optim.cu)
 int64_t adam_ws_floats(int32_t n, int32_t d, int32_t h);

@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(32) dispatch_rank_kernel(const int32_t *__rest
         const int64_t p = p0 + i + lane;
         const bool live = p < R;
         int32_t e = live ? topk_idx[p] : -1;
+        MOE_BOUNDS_NOTE(!live || (uint32_t)e < (uint32_t)n);
         if ((uint32_t)e >= (uint32_t)n) e = -1;
         const unsigned peers = __match_any_sync(0xffffffffu, e);
         const int rank = __popc(peers & ((1u << lane) - 1u));
@@ -134,6 +135,7 @@ __global__ void __launch_bounds__(32) dispatch_rank_kernel(const int32_t *__rest
         start = __shfl_sync(0xffffffffu, start, leader);
         if (e >= 0) {
             const int32_t r = start + rank;
+            MOE_BOUNDS_NOTE((uint32_t)r < (uint32_t)R);
             perm[r] = (int32_t)p;
             inv_perm[p] = r;
         } else if (live) {
@@ -230,7 +232,10 @@ __global__ void __launch_bounds__(256) dispatch_rows_kernel(const XT *__restrict
     for (int64_t t = warp; t < T; t += nwarps) {
         int32_t rows[MOE_MAX_K];
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) rows[s] = s < k ? inv_perm[t * k + s] : 0;
+        for (int s = 0; s < MOE_MAX_K; ++s) {
+            rows[s] = s < k ? inv_perm[t * k + s] : 0;
+            MOE_BOUNDS_NOTE((uint32_t)rows[s] < (uint32_t)R);
+        }
         const uint4 *src = reinterpret_cast<const uint4 *>(x + t * d);
         for (int v = lane; v < nvec; v += 32) {
             const uint4 val = src[v];
@@ -292,6 +297,7 @@ __global__ void __launch_bounds__(256, LAYER ? 3 : 1) combine_kernel(const XT *_
         for (int s = 0; s < KT; ++s) {
             int32_t row = s < k ? inv_perm[t * k + s] : 0;
             const bool valid = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot contributes nothing
+            MOE_BOUNDS_NOTE(valid || s >= k);
             if (!valid) row = 0;
             rowp[s] = reinterpret_cast<const uint4 *>(ys + (int64_t)row * d);
             g[s] = (s < k && valid) ? gates[t * k + s] : 0.0f;
@@ -380,6 +386,7 @@ __global__ void __launch_bounds__(256, LAYER ? 3 : 1) combine_bwd_kernel(const X
         for (int s = 0; s < KT; ++s) {
             const int32_t row = s < k ? inv_perm[t * k + s] : -1;
             valid[s] = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot: zero gate gradient, no row written
+            MOE_BOUNDS_NOTE(valid[s] || s >= k);
             rowo[s] = (int64_t)(valid[s] ? row : 0) * d;
             g[s] = s < k ? gates[t * k + s] : 0.0f;
             dot[s] = 0.0f;
@@ -482,6 +489,7 @@ __global__ void __launch_bounds__(256) dispatch_bwd_kernel(const XT *__restrict_
         for (int s = 0; s < KT; ++s) {
             const int32_t row = s < k ? inv_perm[t * k + s] : -1;
             valid[s] = (uint32_t)row < (uint32_t)(T * k);  // a dropped slot contributes nothing
+            MOE_BOUNDS_NOTE(valid[s] || s >= k);
             rowp[s] = reinterpret_cast<const uint4 *>(dxs + (int64_t)(valid[s] ? row : 0) * d);
         }
         for (int v0 = lane; v0 < nvec; v0 += 32 * VB) {
@@ -558,5 +566,7 @@ int32_t launch_dispatch_bwd(const void *dxs, int32_t act, const int32_t *inv_per
     MOE_LAUNCHED();
     return MOE_OK;
 }
+
+MOE_BOUNDS_READER(bounds_violations_route)
 
 }  // namespace moe

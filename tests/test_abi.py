@@ -75,3 +75,13 @@ def test_hierarchical_sizes(lib):
     assert S.gate_cols == 64 + 2 * 64 and S.logits_elems == w.T * 192
     assert S.gates_elems == w.T * (4 + 2 + 4) and S.kth_elems == 2 * w.T * 3
     assert S.wg_elems == 512 * 64 + 64 * 512 * 64 and S.load_elems == 2 * 4096 + 128 and S.dload_elems == 64 + 4096
+
+
+def test_buffer_size_check(lib):
+    w = synth.CONFIGS["c2"]
+    cfg = B.make_config(w.T, w.d, w.h, w.n, w.k, w.act)
+    S = B.moe_query_sizes(cfg)
+    for which, need in enumerate((S.ws_bytes, S.ws_fwd_bytes, S.ws_bwd_bytes, S.ctx_bytes, S.ws_adam_bytes)):
+        assert B.moe_check_buffer_sizes(cfg, which, need) == 0
+        assert B.moe_check_buffer_sizes(cfg, which, need - 1) == 3      # MOE_ERR_WORKSPACE
+    assert B.moe_check_buffer_sizes(cfg, 9, 1 << 40) == 1
