@@ -34,9 +34,28 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 L2_BYTES = 126 * 2 ** 20
 # FP32 FMA peak of a B200 at its maximum SM clock: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
-# dram__bytes_read.sum + dram__bytes_write.sum of the six expert GEMMs of one step, from one ncu capture of the bench
-# command (the summary under profiles/ names it); workloads without a capture report null
-NCU_TRAFFIC_BYTES_PER_STEP = {"c5-wide-zipf-128": 31.80e9}  # profiles/grouped_gemm_c5_full_dram_traffic.txt
+# dram__bytes_read.sum + dram__bytes_write.sum of the six expert GEMMs of one step come from an ncu capture whose summary
+# under profiles/ records the figure per workload together with the hash of the GEMM source it was taken with: a figure
+# taken with another version of the kernels is not reported (null) rather than carried along
+TRAFFIC_SUMMARY = os.path.join(ROOT, "profiles", "grouped_gemm_dram_traffic.txt")
+GEMM_SOURCE = os.path.join(ROOT, "paper_1701_06538_b200", "csrc", "ffn_tc.cu")
+
+
+def ncu_traffic_bytes_per_step(workload_name):
+    """The captured DRAM bytes per step of the expert GEMMs for this workload, or None if there is no capture or the
+    GEMM source has changed since it was taken."""
+    import hashlib
+    import re
+    try:
+        text = open(TRAFFIC_SUMMARY).read()
+        sha = hashlib.sha256(open(GEMM_SOURCE, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    m = re.search(r"^ffn_tc_sha256:\s*([0-9a-f]{64})", text, re.M)
+    if not m or m.group(1) != sha:
+        return None
+    m = re.search(r"^traffic_bytes_per_step\[%s\]:\s*([0-9.eE+]+)" % re.escape(workload_name), text, re.M)
+    return float(m.group(1)) if m else None
 
 
 def load_peaks():
@@ -90,18 +109,21 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def cpu_sample_tokens(w, flop_budget=2.0e12):
-    # flop_budget 2e12: about 10-30 s of oracle work per forward+backward on the host cores
+def cpu_sample_tokens(w, steps):
+    """Tokens of the CPU sample. ONE size for both places the oracle is timed (the cpu_baseline of the GPU arm: one
+    forward+backward; the --impl reference arm: `steps` of them), because the oracle's rate depends on it (every step
+    touches all experts' weights, however few rows an expert gets): about 2e12 flop (10-30 s) per forward+backward, less
+    when `steps` of them would not fit in about four minutes, in multiples of 1024 tokens."""
     per_token_flop = 12.0 * w.k * w.d * w.h + 12.0 * w.d * (w.n if w.a == 0 else w.a + w.k1 * w.b)
-    return int(max(256, min(w.T, 2 ** int(np.log2(flop_budget / per_token_flop)))))
+    budget = min(2.0e12, 1.6e13 / (steps + 1))  # the oracle sustains roughly 1e11 flop/s on these hosts
+    return int(max(256, min(w.T, 1024 * int(budget / per_token_flop / 1024))))
 
 
 def run_reference(args, w):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    # the oracle does about 25 GFLOP/s on these hosts: size a step so that K timed steps + 1 warm-up take about two minutes
-    Ts = cpu_sample_tokens(w, min(1.0e12, 3.0e12 / (args.steps + 1)))
+    Ts = cpu_sample_tokens(w, args.steps)
     ws, I = host_inputs_sample(w, Ts)
     for _ in range(min(args.warmup, 1)):
         oracle_step(ws, I)
@@ -113,7 +135,8 @@ def run_reference(args, w):
     total = sum(times)
     value = ws.T * args.steps / total
     cores = blas_threads()
-    sample = f"first {ws.T} of {w.T} tokens of {w.name}, all {w.n} experts resident, forward+backward per step"
+    sample = (f"first {ws.T} of {w.T} tokens of {w.name}, all {w.n} experts resident, forward+backward per step "
+              f"(the same sample size as the cpu_baseline of the GPU arm at --steps {args.steps})")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
@@ -361,21 +384,27 @@ def run_ours(args, w):
     gemm_ms = stages["expert_ffn"]["ms"] + stages["expert_ffn_bwd"]["ms"]
     achieved = gemm_flop / (gemm_ms / 1e3) / 1e12
     achieved_gbs = gemm_bytes / (gemm_ms / 1e3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_STEP.get(workload_config(w)["workload"])
+    traffic = ncu_traffic_bytes_per_step(workload_config(w)["workload"])
     kernel = "expert grouped GEMMs (moe_expert_ffn + moe_expert_ffn_bwd, 6 launches; achieved = per-step flop or bytes / per-step time)"
     if w.act != "bf16":
         roof = {"bound": "alu", "kernel": "expert grouped GEMMs, fp32 SIMT", "achieved": achieved,
                 "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
                 "peak_kind": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"}
-    elif achieved_gbs / peaks["hbm_gbs"] > achieved / peaks["bf16_tflops_sustained"]:
+    elif achieved_gbs / peaks["hbm_gbs"] > achieved / peaks["bf16_tflops"]:
         roof = {"bound": "hbm", "kernel": kernel, "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": traffic,
                 "peak_kind": f"{peak_kind} copy bandwidth", "tensor_tflops": achieved}
     else:
-        roof = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                "peak_kind": f"{peak_kind} sustained bf16 (kernels timed back to back inside a long loop)",
-                "frac_of_nominal_2250": achieved / 2250.0, "algorithmic_bytes": gemm_bytes}
+        # the stage timers run a few launches back to back (about 0.1 s), not a seconds-long loop under the power cap:
+        # the burst figure is the denominator; the sustained and the nominal one are printed beside it
+        roof = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
+                "peak_kind": f"{peak_kind} burst bf16 (cuBLAS, best of 10)",
+                "frac_of_burst": achieved / peaks["bf16_tflops"],
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal_2250": achieved / 2250.0, "algorithmic_bytes": gemm_bytes,
+                "forward_tflops": 4.0 * w.R * w.d * w.h / stages["expert_ffn"]["ms"] / 1e9,
+                "backward_tflops": 8.0 * w.R * w.d * w.h / stages["expert_ffn_bwd"]["ms"] / 1e9}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -387,14 +416,14 @@ def run_ours(args, w):
            "gpu_launches": launches, "roofline": roof, "stages": stages,
            "balance": balance_metrics(D)}
     if want_cpu:
-        Ts = cpu_sample_tokens(w)
+        Ts = cpu_sample_tokens(w, args.steps)
         wsamp, I = host_inputs_sample(w, Ts, experts=(host["W1"], host["b1"], host["W2"], host["b2"]))
         t0 = time.perf_counter()
         oracle_step(wsamp, I)
         sec = time.perf_counter() - t0
         out["cpu_baseline"] = {"value": wsamp.T / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                "sample": f"first {wsamp.T} of {w.T} tokens, all {w.n} experts, one forward+backward "
-                                         f"({sec:.1f} s)"}
+                                         f"({sec:.1f} s); --impl reference uses the same sample size at --steps {args.steps}"}
     if rank == 0:
         print(json.dumps(out))
     if world > 1:
