@@ -28,7 +28,8 @@ delete-and-sort kth_excluding, and against the zero-initialisation closed form;
 hierarchical reductions to the flat layer; every backward against central finite
 differences of the forward in float64; the single-precision chain against an
 exact rational emulation; the layer epilogue (sigmoid, dropout, residual) against its
-closed forms and finite differences; the factored optimiser step against full Adam
+closed forms and finite differences; strictly balanced gating against brute-force column
+sorts, its counting invariants and finite differences; the factored optimiser step against full Adam
 on rank-one squared gradients and its textbook limits. The table of trained-model balance metrics in the
 paper's Appendix A cannot be reproduced without the trained model: for those
 printed values parity is unpinned; the metric definitions themselves are pinned
@@ -531,6 +532,144 @@ def gate_h_bwd(x, Wg_p, Wn_p, noise_p, Wg_s, Wn_s, noise_s, G, LS, dgates, w_imp
             dXg[rows] += dc[rows] @ np.asarray(Wg_s[i], f64).T + dr[rows] @ np.asarray(Wn_s[i], f64).T
     return SimpleNamespace(dWg_p=out.dWg, dWn_p=out.dWnoise, dWg_s=store(dWg_s, prec),
                            dWn_s=store(dWn_s, prec), dX_gate=store(dXg, prec))
+
+
+# --------------------------------------------------------------------------------------
+# strictly balanced gating (Appendix F, Eq. 15-20)
+# --------------------------------------------------------------------------------------
+def softmax_gate(x, Wg, prec):
+    """G_sigma(x) = Softmax(x . W_g)   (Eq. 15). The logits come from `project` (the fixed single-precision chain in
+    the rounded modes, because the masks below are integer decisions taken on these numbers); the exponentials and
+    their sum are taken in float64, largest logit subtracted first, and the quotient is rounded once."""
+    c = project(x, Wg, prec)
+    c64 = np.asarray(c, f64)
+    e = np.exp(c64 - c64.max(axis=1, keepdims=True))
+    den = np.zeros(c64.shape[0], f64)
+    for i in range(c64.shape[1]):  # ascending expert
+        den = den + e[:, i]
+    p = e / den[:, None]
+    return c, (p if prec == "f64" else p.astype(f32))
+
+
+def batchwise_mask(p, m):
+    """M_batchwise(X, m)   (Eq. 18): for every expert (column) the m largest values over the batch are kept, so that
+    every expert receives exactly m examples; equal values go to the lower token index."""
+    T, n = p.shape
+    assert 0 <= m <= T
+    mask = np.zeros((T, n), bool)
+    for i in range(n):
+        order = np.argsort(-np.asarray(p[:, i]), kind="stable")  # descending value, equal values keep token order
+        mask[order[:m], i] = True
+    return mask
+
+
+def threshold_mask(p, thr):
+    """M_threshold(x, T)_i = 1 if x_i > T_i   (Eq. 19), the mask used when no batch is available (inference)."""
+    return np.asarray(p) > np.asarray(thr)[None, :]
+
+
+def masked_gate(p, mask, prec):
+    """G(x)_i = G_sigma(x)_i M_i / sum_j G_sigma(x)_j M_j   (Eq. 16); an example no expert keeps has G(x) = 0.
+    The denominator is summed in ascending expert order."""
+    p64 = np.asarray(p, f64)
+    den = np.zeros(p64.shape[0], f64)
+    for i in range(p64.shape[1]):
+        den = den + np.where(mask[:, i], p64[:, i], 0.0)
+    safe = np.where(den > 0, den, 1.0)
+    G = np.where(mask, p64 / safe[:, None], 0.0)
+    return store(G, prec), store(den, prec)
+
+
+def batchwise_loss(p, mask_b, thr):
+    """L_batchwise(X, T, m) = sum_j sum_i (M_threshold(x_j, T)_i - M_batchwise(X, m)_{j,i}) (X_{j,i} - T_i)   (Eq. 20):
+    zero exactly when the two masks agree, positive otherwise."""
+    p64, t64 = np.asarray(p, f64), np.asarray(thr, f64)[None, :]
+    diff = threshold_mask(p, thr).astype(f64) - np.asarray(mask_b, f64)
+    return float((diff * (p64 - t64)).sum())
+
+
+def dispatch_balanced(x, mask):
+    """Each expert receives the examples its mask column keeps, in token order: sorted row r belongs to expert
+    r // m when every column keeps m. Returns the token of each row, the expert of each row, offsets and xs."""
+    T, n = mask.shape
+    tok, exp = [], []
+    offsets = np.zeros(n + 1, np.int32)
+    for i in range(n):
+        rows = np.nonzero(mask[:, i])[0]
+        tok.append(rows)
+        exp.append(np.full(rows.size, i))
+        offsets[i + 1] = offsets[i] + rows.size
+    tok = np.concatenate(tok).astype(np.int32) if n else np.zeros(0, np.int32)
+    exp = np.concatenate(exp).astype(np.int32) if n else np.zeros(0, np.int32)
+    return SimpleNamespace(tok_of_row=tok, expert_of_row=exp, offsets=offsets, xs=np.asarray(x)[tok])
+
+
+def combine_balanced(ys, G, tok_of_row, expert_of_row, T, prec):
+    """y = sum_i G(x)_i E_i(x)   (Eq. 1) over however many experts keep the example, in ascending expert order."""
+    y = np.zeros((T, ys.shape[1]), f64)
+    G64 = np.asarray(G, f64)
+    for r in range(len(tok_of_row)):  # rows are sorted by expert, so every token adds its experts in ascending order
+        t, e = int(tok_of_row[r]), int(expert_of_row[r])
+        y[t] += G64[t, e] * np.asarray(ys[r], f64)
+    return store(y, prec, expert_side=True)
+
+
+def combine_balanced_bwd(dY, ys, G, tok_of_row, expert_of_row, prec):
+    """Adjoint of combine_balanced: dG of each row's (token, expert) pair and dys."""
+    dY64, G64 = np.asarray(dY, f64), np.asarray(G, f64)
+    t, e = tok_of_row.astype(np.int64), expert_of_row.astype(np.int64)
+    dG_row = (dY64[t] * np.asarray(ys, f64)).sum(axis=1)
+    dys = G64[t, e][:, None] * dY64[t]
+    return store(dG_row, prec), store(dys, prec, expert_side=True)
+
+
+def gate_balanced_bwd(x, Wg, p, mask_b, thr, dG_row, tok_of_row, expert_of_row, w_batchwise, prec):
+    """Back-propagation through Eq. 16 (the mask is a constant), Eq. 20 scaled by w_batchwise, and the softmax of
+    Eq. 15, to W_g, the layer input and the thresholds."""
+    T, n = p.shape
+    p64 = np.asarray(p, f64)
+    dG = np.zeros((T, n), f64)
+    dG[tok_of_row.astype(np.int64), expert_of_row.astype(np.int64)] = np.asarray(dG_row, f64)
+    den = np.where(mask_b, p64, 0.0).sum(axis=1)
+    safe = np.where(den > 0, den, 1.0)
+    G = np.where(mask_b, p64 / safe[:, None], 0.0)
+    inner = (G * dG).sum(axis=1)
+    dp = np.where(mask_b, (dG - inner[:, None]) / safe[:, None], 0.0)
+    diff = threshold_mask(p, thr).astype(f64) - np.asarray(mask_b, f64)
+    dp = dp + w_batchwise * diff                     # d L_batchwise / d X_{j,i}
+    dthr = -w_batchwise * diff.sum(axis=0)           # d L_batchwise / d T_i
+    dc = p64 * (dp - (dp * p64).sum(axis=1, keepdims=True))
+    x64 = np.asarray(x, f64)
+    return SimpleNamespace(dWg=store(x64.T @ dc, prec), dX_gate=store(dc @ np.asarray(Wg, f64).T, prec),
+                           dthr=store(dthr, prec), dlogits=dc)
+
+
+def forward_balanced(x, Wg, thr, W1, b1, W2, b2, k, prec):
+    """The layer with strictly balanced gating at training time: every expert gets m = k |X| / n examples."""
+    T, n = x.shape[0], W1.shape[0]
+    assert (k * T) % n == 0
+    m = k * T // n
+    c, p = softmax_gate(x, Wg, prec)
+    mask = batchwise_mask(p, m)
+    G, den = masked_gate(p, mask, prec)
+    D = dispatch_balanced(x, mask)
+    hid, ys = expert_ffn(D.xs, D.offsets, W1, b1, W2, b2, prec)
+    y = combine_balanced(ys, G, D.tok_of_row, D.expert_of_row, T, prec)
+    loss = batchwise_loss(p, mask, thr)
+    return SimpleNamespace(y=y, logits=c, p=p, mask=mask, G=G, den=den, D=D, hid=hid, ys=ys, m=m,
+                           loss=store(np.array([loss]), prec), mask_thr=threshold_mask(p, thr))
+
+
+def backward_balanced(dY, x, Wg, thr, W1, b1, W2, b2, F, w_batchwise, prec):
+    T = x.shape[0]
+    dG_row, dys = combine_balanced_bwd(dY, F.ys, F.G, F.D.tok_of_row, F.D.expert_of_row, prec)
+    E = expert_ffn_bwd(F.D.xs, F.hid, dys, F.D.offsets, W1, W2, prec)
+    dX_exp = np.zeros((T, x.shape[1]), f64)
+    np.add.at(dX_exp, F.D.tok_of_row.astype(np.int64), np.asarray(E.dxs, f64))
+    GB = gate_balanced_bwd(x, Wg, F.p, F.mask, thr, dG_row, F.D.tok_of_row, F.D.expert_of_row, w_batchwise, prec)
+    dX = store(dX_exp + np.asarray(GB.dX_gate, f64), prec, expert_side=True)
+    return SimpleNamespace(dX=dX, dWg=GB.dWg, dthr=GB.dthr, dW1=E.dW1, db1=E.db1, dW2=E.dW2, db2=E.db2, dG_row=dG_row,
+                           dys=dys, dxs=E.dxs, dX_gate=GB.dX_gate, dX_expert=store(dX_exp, prec))
 
 
 # --------------------------------------------------------------------------------------

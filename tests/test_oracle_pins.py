@@ -629,3 +629,103 @@ def test_factored_adam_textbook_limits():
     bn, vb = O.adam_vector_step(b, gb, np.zeros(5), 1e-2, 0.9, 1e-8, 1)
     ba, va = full_adam_beta1_zero(b, gb, np.zeros(5), 1e-2, 0.9, 1e-8, 1)
     assert np.allclose(bn, ba, rtol=1e-14) and np.allclose(vb, va, rtol=1e-14)
+
+
+# ---------------------------------------------------------------- strictly balanced gating (Appendix F, Eq. 15-20)
+def balanced_tiny(seed, T=12, d=5, n=6, h=4):
+    g = rng(seed)
+    return dict(x=g.standard_normal((T, d)), Wg=g.standard_normal((d, n)) * 0.8, W1=g.standard_normal((n, d, h)) * 0.6,
+                b1=g.standard_normal((n, h)) * 0.3, W2=g.standard_normal((n, h, d)) * 0.6, b2=g.standard_normal((n, d)) * 0.3)
+
+
+def test_balanced_gating_invariants_and_brute_force():
+    p_ = balanced_tiny(70)
+    k = 2
+    T, n = p_["x"].shape[0], p_["Wg"].shape[1]
+    m = k * T // n
+    thr = np.full(n, 0.2)
+    F = O.forward_balanced(p_["x"], p_["Wg"], thr, p_["W1"], p_["b1"], p_["W2"], p_["b2"], k, "f64")
+    # Eq. 15 is the textbook softmax
+    z = p_["x"] @ p_["Wg"]
+    assert np.allclose(F.p, np.exp(z) / np.exp(z).sum(axis=1, keepdims=True), rtol=1e-13)
+    # every expert receives exactly m examples, on average k per example
+    assert (F.mask.sum(axis=0) == m).all() and F.mask.sum() == k * T
+    assert (np.diff(F.D.offsets) == m).all()
+    # the mask by brute force: per column, pair (value, -token) sorted descending, first m
+    for i in range(n):
+        best = sorted(range(T), key=lambda t: (-F.p[t, i], t))[:m]
+        assert sorted(best) == list(np.nonzero(F.mask[:, i])[0])
+    # kept gates renormalise to one; an example nobody keeps has a zero gate vector and a zero output
+    kept = F.mask.any(axis=1)
+    assert np.allclose(F.G.sum(axis=1)[kept], 1.0, rtol=1e-13) and (F.G[~F.mask] == 0).all()
+    assert (F.G.sum(axis=1)[~kept] == 0).all() and (np.asarray(F.y)[~kept] == 0).all()
+    # the output is the literal double sum of Eq. 1 with these gates
+    want = np.zeros_like(p_["x"])
+    for t in range(T):
+        for i in range(n):
+            if F.mask[t, i]:
+                hidden = np.maximum(p_["x"][t] @ p_["W1"][i] + p_["b1"][i], 0)
+                want[t] += F.G[t, i] * (hidden @ p_["W2"][i] + p_["b2"][i])
+    assert np.allclose(F.y, want, rtol=1e-12, atol=1e-14)
+
+
+def test_balanced_ties_go_to_the_lower_token():
+    p = np.array([[0.5, 0.1], [0.5, 0.3], [0.5, 0.3], [0.2, 0.3]])
+    mask = O.batchwise_mask(p, 2)
+    assert mask[:, 0].tolist() == [True, True, False, False]      # three-way tie at 0.5: tokens 0 and 1
+    assert mask[:, 1].tolist() == [False, True, True, False]      # three-way tie at 0.3: tokens 1 and 2
+
+
+def test_threshold_mask_and_batchwise_loss():
+    p_ = balanced_tiny(71)
+    k = 2
+    T, n = p_["x"].shape[0], p_["Wg"].shape[1]
+    m = k * T // n
+    _, p = O.softmax_gate(p_["x"], p_["Wg"], "f64")
+    mask = O.batchwise_mask(p, m)
+    # thresholds between each column's m-th and (m+1)-th largest value reproduce the batchwise mask: the loss is zero
+    srt = -np.sort(-p, axis=0)
+    thr = 0.5 * (srt[m - 1] + srt[m])
+    assert (O.threshold_mask(p, thr) == mask).all()
+    assert O.batchwise_loss(p, mask, thr) == 0.0
+    # any other thresholds give a positive loss: every disagreeing entry contributes |X - T|
+    for shift in (-0.05, 0.07):
+        thr2 = thr + shift
+        dis = O.threshold_mask(p, thr2) != mask
+        assert dis.any()
+        assert math.isclose(O.batchwise_loss(p, mask, thr2), np.abs(p - thr2[None, :])[dis].sum(), rel_tol=1e-12)
+    # Eq. 19 is a strict inequality
+    assert not O.threshold_mask(np.array([[0.25]]), np.array([0.25]))[0, 0]
+
+
+def test_balanced_backward_matches_finite_differences():
+    p_ = balanced_tiny(72)
+    k, wb = 2, 0.7
+    T, n = p_["x"].shape[0], p_["Wg"].shape[1]
+    g = rng(73)
+    dY = g.standard_normal(p_["x"].shape)
+    thr = np.full(n, 1.0 / n) + 0.02 * g.standard_normal(n)
+    p_["thr"] = thr
+
+    def loss():
+        F = O.forward_balanced(p_["x"], p_["Wg"], p_["thr"], p_["W1"], p_["b1"], p_["W2"], p_["b2"], k, "f64")
+        return float((F.y * dY).sum() + wb * F.loss[0]), F
+
+    base, F = loss()
+    Bk = O.backward_balanced(dY, p_["x"], p_["Wg"], p_["thr"], p_["W1"], p_["b1"], p_["W2"], p_["b2"], F, wb, "f64")
+    step = 1e-6
+    for name, grad in (("x", Bk.dX), ("Wg", Bk.dWg), ("thr", Bk.dthr), ("W1", Bk.dW1), ("b1", Bk.db1), ("W2", Bk.dW2),
+                       ("b2", Bk.db2)):
+        flat = p_[name].reshape(-1)
+        scale = max(np.abs(grad).max(), 1e-3)
+        for pos in g.choice(flat.size, size=min(10, flat.size), replace=False):
+            old = flat[pos]
+            flat[pos] = old + step
+            up, Fu = loss()
+            flat[pos] = old - step
+            dn, Fd = loss()
+            flat[pos] = old
+            same = (Fu.mask == F.mask).all() and (Fd.mask == F.mask).all() and (Fu.mask_thr == F.mask_thr).all() and \
+                (Fd.mask_thr == F.mask_thr).all()
+            assert same, "a mask switched inside the stencil: pick another seed"
+            assert abs((up - dn) / (2 * step) - np.asarray(grad).reshape(-1)[pos]) / scale < 2e-6, (name, pos)
