@@ -430,6 +430,107 @@ def run_ours(args, w):
         torch.distributed.destroy_process_group()
 
 
+def run_balanced(args, w):
+    """The same layer with strictly balanced gating (Appendix F): every expert receives exactly k T / n examples, so
+    the grouped GEMMs run on uniform segments. One step = gate, dispatch, experts, combine and their backward, composed
+    from the stage calls of the C ABI. Second workload of the library; the headline line is the noisy top-k one."""
+    from paper_1701_06538_b200 import binding as B
+    rank, local_rank, world = dist_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local_rank)
+    peaks, peak_kind = load_peaks()
+    cfg, S, D, host = build_device_state(w, keep_host_experts=False)
+    Sb = B.moe_query_balanced_sizes(cfg)
+    T, d, h, n, k, R = w.T, w.d, w.h, w.n, w.k, w.R
+    adt = D["x"].dtype
+    e = lambda *s_, dt=torch.float32: torch.empty(*s_, dtype=dt, device="cuda")
+    thr = torch.full((n,), 1.0 / n, device="cuda")
+    G = dict(logits=e(T, n), probs=e(T, n), mask_bits=e(T, Sb.mask_words, dt=torch.int32), tok_of_row=e(R, dt=torch.int32),
+             offsets=e(n + 1, dt=torch.int32), den=e(T), tok_ptr=e(T + 1, dt=torch.int32), tok_rows=e(R, dt=torch.int32),
+             loss=e(1), thr_counts=e(n, dt=torch.int32), ws=B.empty_bytes(Sb.ws_bytes))
+    xs, hid, ys, dys, dxs = e(R, d, dt=adt), e(R, h, dt=adt), e(R, d, dt=adt), e(R, d, dt=adt), e(R, d, dt=adt)
+    dG_row, dWg, dXg, dthr = e(R), e(d, n), e(T, d), e(n)
+    Wg = D["Wg"][:d * n]
+    calls = {
+        "gate_balanced": lambda: B.moe_gate_balanced(cfg, D["x"], Wg, thr, G["logits"], G["probs"], G["mask_bits"],
+                                                     G["tok_of_row"], G["offsets"], G["den"], G["tok_ptr"], G["tok_rows"],
+                                                     G["loss"], G["thr_counts"], G["ws"]),
+        "dispatch_balanced": lambda: B.moe_dispatch_balanced(cfg, D["x"], G["tok_of_row"], xs),
+        "expert_ffn": lambda: B.moe_expert_ffn(cfg, xs, G["offsets"], D["W1"], D["b1"], D["W2"], D["b2"], hid, ys, D["ws"]),
+        "combine_balanced": lambda: B.moe_combine_balanced(cfg, ys, G["probs"], G["den"], G["tok_ptr"], G["tok_rows"], D["y"]),
+        "combine_balanced_bwd": lambda: B.moe_combine_balanced_bwd(cfg, D["dY"], ys, G["probs"], G["den"], G["tok_of_row"],
+                                                                   dG_row, dys),
+        "expert_ffn_bwd": lambda: B.moe_expert_ffn_bwd(cfg, xs, hid, dys, G["offsets"], D["W1"], D["W2"], dxs, D["dW1"],
+                                                       D["db1"], D["dW2"], D["db2"], D["ws"]),
+        "gate_balanced_bwd": lambda: B.moe_gate_balanced_bwd(cfg, D["x"], Wg, G["probs"], G["mask_bits"], G["den"], thr,
+                                                             G["tok_ptr"], G["tok_rows"], dG_row, G["thr_counts"], 1.0, dWg,
+                                                             dXg, dthr, G["ws"]),
+        "dispatch_balanced_bwd": lambda: B.moe_dispatch_balanced_bwd(cfg, dxs, G["tok_ptr"], G["tok_rows"], dXg, D["dX"]),
+    }
+
+    def step():
+        for fn in calls.values():
+            fn()
+
+    small = "flushed" in workload_config(w)["l2"]
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if small else None
+
+    def timed(fn, K):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        torch.cuda.synchronize()
+        for a, b in ev:
+            if flush_buf is not None:
+                flush_buf.fill_(1)
+            a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in ev]
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert B.moe_check_status(D["ws"]) == 0
+    sampler = ClockSampler(local_rank)
+    l0 = B.moe_debug_launch_count()
+    ms = timed(step, args.steps)
+    launches = B.moe_debug_launch_count() - l0
+    hx, hdY = D["x"].cpu().pin_memory(), D["dY"].cpu().pin_memory()
+    hy, hdX = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+
+    def e2e_step():
+        D["x"].copy_(hx, non_blocking=True); D["dY"].copy_(hdY, non_blocking=True)
+        step()
+        hy.copy_(D["y"], non_blocking=True); hdX.copy_(D["dX"], non_blocking=True)
+
+    e2e_step()
+    ms_e2e = timed(e2e_step, args.steps)
+    clocks = sampler.stop()
+    stages = {name: {"ms": statistics.mean(timed(fn, max(3, min(args.steps, 10))))} for name, fn in calls.items()}
+    esz = 2 if w.act == "bf16" else 4
+    gemm_ms = stages["expert_ffn"]["ms"] + stages["expert_ffn_bwd"]["ms"]
+    achieved = 12.0 * R * d * h / (gemm_ms / 1e3) / 1e12
+    gemm_bytes = (6 * R * d + 5 * R * h) * esz + 6 * n * d * h * esz
+    achieved_gbs = gemm_bytes / (gemm_ms / 1e3) / 1e9
+    hbm_bound = achieved_gbs / peaks["hbm_gbs"] > achieved / peaks["bf16_tflops"]
+    roof = {"bound": "hbm" if hbm_bound else "tensor", "kernel": "expert grouped GEMMs on uniform segments (6 launches)",
+            "achieved": achieved_gbs if hbm_bound else achieved, "peak": peaks["hbm_gbs"] if hbm_bound else peaks["bf16_tflops"],
+            "unit": "GB/s" if hbm_bound else "TFLOP/s",
+            "frac": achieved_gbs / peaks["hbm_gbs"] if hbm_bound else achieved / peaks["bf16_tflops"], "traffic": None,
+            "peak_kind": f"{peak_kind} " + ("copy bandwidth" if hbm_bound else "burst bf16"), "tensor_tflops": achieved}
+    counts = torch.diff(G["offsets"]).cpu()
+    print(json.dumps({
+        "metric": METRIC, "value": T * args.steps / (sum(ms) / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.act == "bf16" else "f32", "data": "synthetic",
+        "config": dict(workload_config(w), gating="strictly balanced (Appendix F): every expert gets exactly k T / n rows",
+                       rows_per_expert=int(Sb.m), launch="stream"),
+        "clocks": clocks,
+        "e2e": {"value": T * args.steps / (sum(ms_e2e) / 1e3), "unit": UNIT, "h2d_bytes_per_step": 2 * hx.numel() * esz,
+                "d2h_bytes_per_step": 2 * hx.numel() * esz, "ms_per_step": sum(ms_e2e) / args.steps},
+        "gpu_launches": launches, "roofline": roof, "stages": stages,
+        "balance": {"rows_per_expert_min": int(counts.min()), "rows_per_expert_max": int(counts.max()),
+                    "examples_without_expert": int((torch.diff(G["tok_ptr"]) == 0).sum()),
+                    "loss_batchwise": float(G["loss"][0])}}))
+
+
 def balance_metrics(D):
     """The balance metrics of the paper's loss-ablation table, for the realised routing."""
     imp, load, counts = D["importance"].double(), D["load"][:D["importance"].numel()].double(), D["counts"].double()
@@ -515,11 +616,15 @@ def main():
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="replay the step from a CUDA graph (auto: for the small, launch-bound workloads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gating", default="noisy-topk", choices=["noisy-topk", "balanced"],
+                    help="balanced: the strictly balanced gating of Appendix F (flat configs whose k T is a multiple of n)")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]
     if args.tokens:
         w = w.scaled(args.tokens)
-    if args.impl == "reference":
+    if args.gating == "balanced" and args.impl == "ours":
+        run_balanced(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

@@ -297,6 +297,57 @@ int32_t moe_backward(const moe_config *cfg, const void *dY, const void *x, const
                      void *db2, void *ws, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Strictly balanced gating (Appendix F, Eq. 15-20), flat layers, training time: every expert receives exactly
+ * m = k*T/n examples (k*T must be a multiple of n).
+ *   probs  = Softmax(x.W_g)                                        (Eq. 15; logits by the fixed fma chain of moe_gate)
+ *   mask   = for every expert the m largest probs of its column over the batch, equal values to the
+ *            lower token                                           (Eq. 18, batchwise mask)
+ *   G      = probs * mask / sum_j probs_j * mask_j                 (Eq. 16; an example nobody keeps gets G = 0, y = 0)
+ *   loss   = sum (M_threshold - M_batchwise) * (probs - thresholds) with M_threshold = [probs > thresholds] (Eq. 19-20)
+ * An example is kept by a variable number of experts, so the routing tables are by sorted row: rows are
+ * expert-major (expert e owns rows e*m .. e*m+m-1, in token order), tok_of_row [R] is each row's token,
+ * offsets [n+1] = e*m (for moe_expert_ffn / moe_expert_ffn_bwd, which run unchanged on these uniform segments),
+ * and tok_ptr [T+1] / tok_rows [R] list every token's rows in ascending expert order. The gate of a row is
+ * probs[token, expert] / den[token]. mask_bits [T, mask_words] uint32 holds the mask (bit e%32 of word e/32).
+ * Routing by the threshold mask alone (inference without a batch) is not built; the mask enters the loss, and
+ * thr_counts [n] = how many examples each expert's threshold would keep.
+ * Sizes: moe_query_balanced_sizes. The backward treats the mask as a constant; L_batchwise enters scaled by
+ * w_batchwise and reaches probs and the thresholds.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct moe_balanced_sizes {
+    int64_t m;          /* examples per expert: k*T/n                              */
+    int64_t R;          /* sorted rows: n*m = k*T                                  */
+    int64_t mask_words; /* uint32 words per token of mask_bits: ceil(n/32)         */
+    int64_t ws_bytes;   /* workspace of moe_gate_balanced / moe_gate_balanced_bwd  */
+} moe_balanced_sizes;
+int32_t moe_query_balanced_sizes(const moe_config *cfg, moe_balanced_sizes *host_out);
+
+/* in : x [T,d] act, Wg [d,n], thresholds [n]
+ * out: logits, probs [T,n]; mask_bits [T,mask_words]; tok_of_row [R]; offsets [n+1]; den [T]; tok_ptr [T+1];
+ *      tok_rows [R]; loss_batchwise [1]; thr_counts [n] */
+int32_t moe_gate_balanced(const moe_config *cfg, const void *x, const float *Wg, const float *thresholds, float *logits,
+                          float *probs, uint32_t *mask_bits, int32_t *tok_of_row, int32_t *offsets, float *den,
+                          int32_t *tok_ptr, int32_t *tok_rows, float *loss_batchwise, int32_t *thr_counts, void *ws,
+                          void *stream);
+/* xs [R,d] act: xs[r] = x[tok_of_row[r]] */
+int32_t moe_dispatch_balanced(const moe_config *cfg, const void *x, const int32_t *tok_of_row, void *xs, void *stream);
+/* y[t] = sum over the rows of token t of G * ys[row], ascending expert (Eq. 1)   out: y [T,d] act */
+int32_t moe_combine_balanced(const moe_config *cfg, const void *ys, const float *probs, const float *den,
+                             const int32_t *tok_ptr, const int32_t *tok_rows, void *y, void *stream);
+/* out: dG_row [R] = <dY[token], ys[row]>, dys [R,d] act = G * dY[token] */
+int32_t moe_combine_balanced_bwd(const moe_config *cfg, const void *dY, const void *ys, const float *probs,
+                                 const float *den, const int32_t *tok_of_row, float *dG_row, void *dys, void *stream);
+/* out: dWg [d,n], dX_gate [T,d] float, dthresholds [n] */
+int32_t moe_gate_balanced_bwd(const moe_config *cfg, const void *x, const float *Wg, const float *probs,
+                              const uint32_t *mask_bits, const float *den, const float *thresholds,
+                              const int32_t *tok_ptr, const int32_t *tok_rows, const float *dG_row,
+                              const int32_t *thr_counts, float w_batchwise, float *dWg, float *dX_gate,
+                              float *dthresholds, void *ws, void *stream);
+/* dX [T,d] act = sum over the rows of token t of dxs[row] + dX_gate[t] */
+int32_t moe_dispatch_balanced_bwd(const moe_config *cfg, const void *dxs, const int32_t *tok_ptr,
+                                  const int32_t *tok_rows, const float *dX_gate, void *dX, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * Optimiser step on the expert parameters (Appendix D, "Training": the memory optimisations): Adam with
  * beta1 = 0 (no first-moment estimate) and a factored second-moment estimate. For each expert weight matrix
  * only the running averages (decay beta2) of the row-wise and of the column-wise means of the squared

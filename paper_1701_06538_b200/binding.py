@@ -24,7 +24,9 @@ EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_wor
            "moe_gate", "moe_dispatch", "moe_dispatch_noalloc", "moe_expert_ffn", "moe_combine", "moe_losses", "moe_combine_bwd",
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward",
-           "moe_expert_adam_factored", "moe_check_buffer_sizes", "moe_debug_wait_timeout", "moe_debug_bounds_violations"]
+           "moe_expert_adam_factored", "moe_check_buffer_sizes", "moe_debug_wait_timeout", "moe_debug_bounds_violations",
+           "moe_query_balanced_sizes", "moe_gate_balanced", "moe_dispatch_balanced", "moe_combine_balanced",
+           "moe_combine_balanced_bwd", "moe_gate_balanced_bwd", "moe_dispatch_balanced_bwd"]
 
 
 class MoeError(RuntimeError):
@@ -49,6 +51,10 @@ class moe_ctx_layout(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int64) for name in
                 ("topk_idx", "gates", "clean", "raw_noise", "kth_vals", "kth_idx", "xs", "perm", "inv_perm",
                  "counts", "offsets", "hid", "ys", "importance", "load", "losses")]
+
+
+class moe_balanced_sizes(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int64) for name in ("m", "R", "mask_words", "ws_bytes")]
 
 
 _lib = None
@@ -209,6 +215,42 @@ def moe_forward(cfg, x, Wg, Wnoise, noise, W1, b1, W2, b2, y, losses, importance
 def moe_backward(cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2, ws):
     _call("moe_backward", cfg, dY, x, Wg, Wnoise, noise, W1, b1, W2, b2, ctx, dX, dWg, dWnoise, dW1, db1, dW2, db2,
           ws)
+
+
+def moe_query_balanced_sizes(cfg) -> moe_balanced_sizes:
+    out = moe_balanced_sizes()
+    status = lib().moe_query_balanced_sizes(ctypes.byref(cfg), ctypes.byref(out))
+    if status != 0:
+        raise MoeError("moe_query_balanced_sizes", status)
+    return out
+
+
+def moe_gate_balanced(cfg, x, Wg, thresholds, logits, probs, mask_bits, tok_of_row, offsets, den, tok_ptr, tok_rows,
+                      loss_batchwise, thr_counts, ws):
+    _call("moe_gate_balanced", cfg, x, Wg, thresholds, logits, probs, mask_bits, tok_of_row, offsets, den, tok_ptr,
+          tok_rows, loss_batchwise, thr_counts, ws)
+
+
+def moe_dispatch_balanced(cfg, x, tok_of_row, xs):
+    _call("moe_dispatch_balanced", cfg, x, tok_of_row, xs)
+
+
+def moe_combine_balanced(cfg, ys, probs, den, tok_ptr, tok_rows, y):
+    _call("moe_combine_balanced", cfg, ys, probs, den, tok_ptr, tok_rows, y)
+
+
+def moe_combine_balanced_bwd(cfg, dY, ys, probs, den, tok_of_row, dG_row, dys):
+    _call("moe_combine_balanced_bwd", cfg, dY, ys, probs, den, tok_of_row, dG_row, dys)
+
+
+def moe_gate_balanced_bwd(cfg, x, Wg, probs, mask_bits, den, thresholds, tok_ptr, tok_rows, dG_row, thr_counts, w_batchwise,
+                          dWg, dX_gate, dthresholds, ws):
+    _call("moe_gate_balanced_bwd", cfg, x, Wg, probs, mask_bits, den, thresholds, tok_ptr, tok_rows, dG_row, thr_counts,
+          float(w_batchwise), dWg, dX_gate, dthresholds, ws)
+
+
+def moe_dispatch_balanced_bwd(cfg, dxs, tok_ptr, tok_rows, dX_gate, dX):
+    _call("moe_dispatch_balanced_bwd", cfg, dxs, tok_ptr, tok_rows, dX_gate, dX)
 
 
 def moe_expert_adam_factored(cfg, W1, b1, W2, b2, dW1, db1, dW2, db2, state, lr, beta2, eps, step, ws):

@@ -920,6 +920,111 @@ int32_t moe_expert_adam_factored(const moe_config *cfg, void *W1, void *b1, void
                               step, reinterpret_cast<float *>(static_cast<char *>(ws) + kWsHeader), as_stream(stream));
 }
 
+// ---------------------------------------------------------------------------- strictly balanced gating (Appendix F)
+static int32_t check_balanced(const moe_config *c) {
+    MOE_TRY(check_config(c));
+    if (c->a > 0) return MOE_ERR_UNSUPPORTED;                       // flat layers only
+    if (c->T > 0 && ((int64_t)c->T * c->k) % c->n != 0) return MOE_ERR_INVALID_ARG;  // m = k T / n must be whole
+    return MOE_OK;
+}
+
+int32_t moe_query_balanced_sizes(const moe_config *cfg, moe_balanced_sizes *out) {
+    MOE_TRY(check_balanced(cfg));
+    if (!out) return MOE_ERR_INVALID_ARG;
+    out->m = (int64_t)cfg->T * cfg->k / cfg->n;
+    out->R = (int64_t)cfg->T * cfg->k;
+    out->mask_words = (cfg->n + 31) / 32;
+    const int64_t fwd = balanced_ws_bytes(cfg->T, cfg->n);
+    const int64_t bwd = measure([&](Carver &cv) {   // the larger of the two ways moe_gate_balanced_bwd carves
+        cv.take<bf16>((int64_t)cfg->T * 3 * cfg->n); cv.take<bf16>((int64_t)cfg->d * 3 * cfg->n);
+        cv.take<float>(tc_gate_bwd_partials(cfg->T, cfg->d, cfg->n / 2 > 0 ? cfg->n / 2 : 1));
+        cv.take<float>((int64_t)cfg->T * cfg->n);
+    });
+    out->ws_bytes = kWsHeader + (fwd > bwd ? fwd : bwd);
+    return MOE_OK;
+}
+
+int32_t moe_gate_balanced(const moe_config *cfg, const void *x, const float *Wg, const float *thresholds, float *logits,
+                          float *probs, uint32_t *mask_bits, int32_t *tok_of_row, int32_t *offsets, float *den,
+                          int32_t *tok_ptr, int32_t *tok_rows, float *loss_batchwise, int32_t *thr_counts, void *ws,
+                          void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(x, Wg, thresholds, logits, probs, mask_bits, tok_of_row, offsets, den, tok_ptr, tok_rows, loss_batchwise,
+                 thr_counts, ws);
+    return launch_balanced_gate(x, cfg->act, cfg->T, cfg->d, cfg->n, cfg->k, Wg, thresholds, logits, probs, mask_bits,
+                                tok_of_row, offsets, den, tok_ptr, tok_rows, loss_batchwise, thr_counts,
+                                static_cast<char *>(ws) + kWsHeader, as_stream(stream));
+}
+
+int32_t moe_dispatch_balanced(const moe_config *cfg, const void *x, const int32_t *tok_of_row, void *xs, void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(x, tok_of_row, xs);
+    return launch_balanced_gather(x, cfg->act, tok_of_row, (int64_t)cfg->T * cfg->k, cfg->T, cfg->d, xs, as_stream(stream));
+}
+
+int32_t moe_combine_balanced(const moe_config *cfg, const void *ys, const float *probs, const float *den,
+                             const int32_t *tok_ptr, const int32_t *tok_rows, void *y, void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(ys, probs, den, tok_ptr, tok_rows, y);
+    const int64_t R = (int64_t)cfg->T * cfg->k;
+    return launch_balanced_combine(ys, cfg->act, probs, den, tok_ptr, tok_rows, cfg->T, R, cfg->n, (int32_t)(R / cfg->n),
+                                   cfg->d, y, as_stream(stream));
+}
+
+int32_t moe_combine_balanced_bwd(const moe_config *cfg, const void *dY, const void *ys, const float *probs,
+                                 const float *den, const int32_t *tok_of_row, float *dG_row, void *dys, void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(dY, ys, probs, den, tok_of_row, dG_row, dys);
+    const int64_t R = (int64_t)cfg->T * cfg->k;
+    return launch_balanced_combine_bwd(dY, ys, cfg->act, probs, den, tok_of_row, R, cfg->T, cfg->n, (int32_t)(R / cfg->n),
+                                       cfg->d, dG_row, dys, as_stream(stream));
+}
+
+int32_t moe_gate_balanced_bwd(const moe_config *cfg, const void *x, const float *Wg, const float *probs,
+                              const uint32_t *mask_bits, const float *den, const float *thresholds,
+                              const int32_t *tok_ptr, const int32_t *tok_rows, const float *dG_row,
+                              const int32_t *thr_counts, float w_batchwise, float *dWg, float *dX_gate,
+                              float *dthresholds, void *ws, void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(x, Wg, probs, mask_bits, den, thresholds, tok_ptr, tok_rows, dG_row, thr_counts, dWg, dX_gate, dthresholds,
+                 ws);
+    const Dims D = dims_of(cfg);
+    cudaStream_t st = as_stream(stream);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    // the two contractions on the tensor cores (three-term bf16 splits, as in moe_gate_bwd) when the shapes allow: the
+    // n logit columns are handled as the two column halves of one [d, n] matrix
+    const int32_t half = (int32_t)(D.n / 2);
+    const bool tc = D.n % 2 == 0 && D.T > 0 && tc_gate_bwd_supported(D.act, (int32_t)D.d, half);
+    if (tc) {
+        void *dsplit = cv.take<bf16>(D.T * 3 * D.n);
+        void *wsplit = cv.take<bf16>(D.d * 3 * D.n);
+        float *partials = cv.take<float>(tc_gate_bwd_partials(D.T, (int32_t)D.d, half));
+        MOE_TRY(reset_status(ws, st));
+        MOE_TRY(launch_balanced_gate_bwd(probs, mask_bits, den, thresholds, tok_ptr, tok_rows, dG_row, thr_counts,
+                                         w_batchwise, D.T, (int32_t)D.n, (int32_t)(D.R / D.n), nullptr, dsplit, dthresholds,
+                                         st));
+        return launch_tc_gate_bwd(x, D.T, (int32_t)D.d, half, Wg, Wg + half, dsplit, wsplit, partials, dWg, dWg + half, dX_gate,
+                                  status_word(ws), st, D.flags, (int32_t)D.n);
+    }
+    float *dc = cv.take<float>(D.T * D.n);
+    MOE_TRY(launch_balanced_gate_bwd(probs, mask_bits, den, thresholds, tok_ptr, tok_rows, dG_row, thr_counts, w_batchwise,
+                                     D.T, (int32_t)D.n, (int32_t)(D.R / D.n), dc, nullptr, dthresholds, st));
+    if (D.T == 0) {
+        MOE_CUDA(cudaMemsetAsync(dWg, 0, sizeof(float) * D.d * D.n, st));
+        return MOE_OK;
+    }
+    return gate_weight_grads(D, x, dc, Wg, D.n, dWg, dX_gate, false, st);
+}
+
+int32_t moe_dispatch_balanced_bwd(const moe_config *cfg, const void *dxs, const int32_t *tok_ptr,
+                                  const int32_t *tok_rows, const float *dX_gate, void *dX, void *stream) {
+    MOE_TRY(check_balanced(cfg));
+    REQUIRE_PTRS(dxs, tok_ptr, tok_rows, dX_gate, dX);
+    return launch_balanced_dispatch_bwd(dxs, cfg->act, tok_ptr, tok_rows, dX_gate, cfg->T, (int64_t)cfg->T * cfg->k, cfg->d,
+                                        dX, as_stream(stream));
+}
+
 int32_t moe_combine_layer(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm,
                           const void *x, const uint8_t *keep_bits, float drop_prob, void *out, void *stream) {
     MOE_TRY(check_config(cfg));

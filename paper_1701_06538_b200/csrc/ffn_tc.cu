@@ -1672,14 +1672,16 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
 // bf16 already. dsplit is [T, 3 * n2] = (hi | mid | lo) of the [T, n2] logit gradients (n2 = 2n: clean
 // columns then raw-noise columns), wsplit is [d, 3 * n2] likewise for [W_g | W_noise].
 // ------------------------------------------------------------------------------------------
+// ldw: row stride of Wg and Wn in floats (n for two separate [d, n] matrices; 2n when they are the two halves of the
+// columns of one [d, 2n] matrix)
 __global__ void __launch_bounds__(256) split_weights_kernel(const float *__restrict__ Wg,
                                                             const float *__restrict__ Wn, int32_t d, int32_t n,
-                                                            bf16 *__restrict__ wsplit) {
+                                                            bf16 *__restrict__ wsplit, int32_t ldw) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int32_t n2 = 2 * n;
     if (i >= (int64_t)d * n2) return;
     const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
-    const float v = j < n ? Wg[(int64_t)q * n + j] : Wn[(int64_t)q * n + (j - n)];
+    const float v = j < n ? Wg[(int64_t)q * ldw + j] : Wn[(int64_t)q * ldw + (j - n)];
     const bf16 hi = __float2bfloat16_rn(v);
     const float r1 = v - __bfloat162float(hi);
     const bf16 mid = __float2bfloat16_rn(r1);
@@ -1691,7 +1693,8 @@ __global__ void __launch_bounds__(256) split_weights_kernel(const float *__restr
 // out (group g = blockIdx.y) = sum_c part[c * part_stride + g * d * 2n + .], split into the W_g and W_noise halves
 __global__ void __launch_bounds__(256) reduce_partials_kernel(const float *__restrict__ part, int32_t nparts,
                                                               int64_t part_stride, int32_t d, int32_t n,
-                                                              float *__restrict__ dWg, float *__restrict__ dWn) {
+                                                              float *__restrict__ dWg, float *__restrict__ dWn,
+                                                              int32_t ldw) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int32_t n2 = 2 * n;
     const int64_t total = (int64_t)d * n2;
@@ -1700,8 +1703,8 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float *__res
     double s = 0.0;
     for (int32_t c = 0; c < nparts; ++c) s += (double)part[(int64_t)c * part_stride + g * total + i];
     const int32_t q = (int32_t)(i / n2), j = (int32_t)(i % n2);
-    if (j < n) dWg[(g * d + q) * n + j] = (float)s;
-    else dWn[(g * d + q) * n + (j - n)] = (float)s;
+    if (j < n) dWg[(g * d + q) * ldw + j] = (float)s;
+    else dWn[(g * d + q) * ldw + (j - n)] = (float)s;
 }
 
 bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n) {
@@ -1737,14 +1740,18 @@ int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n) {
 
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
-                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags) {
+                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags, int32_t ldw) {
     const int32_t n2 = 2 * n;
+    if (T == 0 && ldw > 0) {
+        for (int32_t q = 0; q < d; ++q) MOE_CUDA(cudaMemsetAsync(dWg + (int64_t)q * ldw, 0, sizeof(float) * n2, st));
+        return MOE_OK;
+    }
     if (T == 0) {
         MOE_CUDA(cudaMemsetAsync(dWg, 0, sizeof(float) * d * n, st));
         MOE_CUDA(cudaMemsetAsync(dWn, 0, sizeof(float) * d * n, st));
         return MOE_OK;
     }
-    split_weights_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit);
+    split_weights_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(Wg, Wn, d, n, (bf16 *)wsplit, ldw > 0 ? ldw : n);
     MOE_LAUNCHED();
     int32_t nr, rows;
     gate_bwd_split(T, d, n, &nr, &rows);
@@ -1758,7 +1765,8 @@ int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const
         p.rows_per_seg = rows; p.segs_per_term = nr; p.b_term_chunks = n2 / 64;
         p.sub_kb0 = GB_ROWS_HI / BK; p.sub_kb = GB_ROWS_LO / BK; p.interleave = 3;
         MOE_TRY(launch_acc_wgrad(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
-        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, 3 * nr, (int64_t)d * n2, d, n, dWg, dWn);
+        reduce_partials_kernel<<<(unsigned)cdiv((int64_t)d * n2, 256), 256, 0, st>>>(partials, 3 * nr, (int64_t)d * n2, d, n, dWg, dWn,
+                                                                                     ldw > 0 ? ldw : n);
         MOE_LAUNCHED();
     }
     {   // dX_gate: six cross terms of the two split operands, concatenated along the contraction
@@ -1840,7 +1848,7 @@ int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, voi
                                      int64_t P1, int32_t d, int32_t b, float *partials, float *dWg_s, float *dWn_s,
                                      float *dX_sec, int32_t *status, cudaStream_t st) {
     const int32_t n2 = 2 * b;
-    split_weights_kernel<<<(unsigned)cdiv((int64_t)a * d * n2, 256), 256, 0, st>>>(Wg_s, Wn_s, a * d, b, (bf16 *)wsplit_s);
+    split_weights_kernel<<<(unsigned)cdiv((int64_t)a * d * n2, 256), 256, 0, st>>>(Wg_s, Wn_s, a * d, b, (bf16 *)wsplit_s, b);
     MOE_LAUNCHED();
     {   // dW_s[i] = sum over the slots of group i of x[token]^T . dlogit[slot], one partial per precision term
         CUtensorMap tmA, tmB;
@@ -1851,7 +1859,7 @@ int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, voi
         p.M = d; p.N = n2; p.R = P1; p.out_f32 = partials; p.status = status;
         MOE_TRY(launch<WGRAD>(tmA, tmB, p, (int64_t)p.nseg * cdiv(d, BM) * cdiv(n2, BN), st));
         reduce_partials_kernel<<<dim3((unsigned)cdiv((int64_t)d * n2, 256), (unsigned)a), 256, 0, st>>>(
-            partials, 3, (int64_t)a * d * n2, d, b, dWg_s, dWn_s);
+            partials, 3, (int64_t)a * d * n2, d, b, dWg_s, dWn_s, b);
         MOE_LAUNCHED();
     }
     if (P1 > 0) {   // dX_sec[row] = dlogit[row] . [W_g | W_noise][group]^T, six cross terms

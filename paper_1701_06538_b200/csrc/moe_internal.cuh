@@ -227,6 +227,29 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
                       cudaStream_t st, bool first_only = false);
 
+// ----------------------------------------------------------------------------- strictly balanced gating (balanced.cu)
+int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st);  // route.cu
+int64_t balanced_ws_bytes(int64_t T, int32_t n);
+int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, int32_t k, const float *Wg,
+                             const float *thr, float *logits, float *probs, uint32_t *mask_bits, int32_t *tok_of_row,
+                             int32_t *offsets, float *den, int32_t *tok_ptr, int32_t *tok_rows, float *loss,
+                             int32_t *thr_counts, void *ws, cudaStream_t st);
+int32_t launch_balanced_gather(const void *x, int32_t act, const int32_t *tok_of_row, int64_t R, int64_t T, int32_t d,
+                               void *xs, cudaStream_t st);
+int32_t launch_balanced_combine(const void *ys, int32_t act, const float *p, const float *den, const int32_t *tok_ptr,
+                                const int32_t *tok_rows, int64_t T, int64_t R, int32_t n, int32_t m, int32_t d, void *y,
+                                cudaStream_t st);
+int32_t launch_balanced_combine_bwd(const void *dY, const void *ys, int32_t act, const float *p, const float *den,
+                                    const int32_t *tok_of_row, int64_t R, int64_t T, int32_t n, int32_t m, int32_t d,
+                                    float *dG_row, void *dys, cudaStream_t st);
+// dc [T, n] float, or (dsplit given) its three-term bf16 split [T, 3n] = (hi | mid | lo) for the tensor-core contractions
+int32_t launch_balanced_gate_bwd(const float *p, const uint32_t *mask_bits, const float *den, const float *thr,
+                                 const int32_t *tok_ptr, const int32_t *tok_rows, const float *dG_row,
+                                 const int32_t *thr_counts, float w, int64_t T, int32_t n, int32_t m, float *dc,
+                                 void *dsplit, float *dthr, cudaStream_t st);
+int32_t launch_balanced_dispatch_bwd(const void *dxs, int32_t act, const int32_t *tok_ptr, const int32_t *tok_rows,
+                                     const float *dX_gate, int64_t T, int64_t R, int32_t d, void *dX, cudaStream_t st);
+
 int32_t launch_debug_wait(int32_t *status, unsigned long long limit_ns, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- optimiser step (optim.cu)
@@ -239,7 +262,8 @@ bool tc_gate_bwd_supported(int32_t act, int32_t d, int32_t n);
 int64_t tc_gate_bwd_partials(int64_t T, int32_t d, int32_t n);  // floats of partial-sum scratch
 int32_t launch_tc_gate_bwd(const void *x, int64_t T, int32_t d, int32_t n, const float *Wg, const float *Wn,
                            const void *dsplit, void *wsplit, float *partials, float *dWg, float *dWn,
-                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags);
+                           float *dX_gate, int32_t *status, cudaStream_t st, int32_t flags, int32_t ldw = 0);
+// (ldw > 0: Wg / Wn, dWg / dWn are the left and right column halves of one [d, 2n] matrix with row stride ldw)
 int32_t launch_tc_gate_fwd_grouped(const void *xs_p, int64_t P1, int32_t d, int32_t a, int32_t b, const void *wsplit_s,
                                    const int32_t *offsets_p, int32_t *tile_prefix, float *cr_s, int32_t *status,
                                    cudaStream_t st, int32_t flags);

@@ -164,6 +164,13 @@ int32_t launch_dispatch_index(const int32_t *topk_idx, int64_t R, int32_t n, int
     return MOE_OK;
 }
 
+// out[0..n] = exclusive prefix sums of counts[0..n-1] (one block; any n)
+int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st) {
+    dispatch_scan_experts_kernel<<<1, 1024, 0, st>>>(counts, n, out);
+    MOE_LAUNCHED();
+    return MOE_OK;
+}
+
 // tile_prefix[e] = number of bm-row tiles of the segments before e (tile_prefix[n] = total)
 __global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t *__restrict__ offsets, int32_t n,
                                                            int32_t bm, int32_t *__restrict__ tile_prefix) {
