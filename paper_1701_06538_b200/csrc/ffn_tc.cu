@@ -294,6 +294,24 @@ __device__ __forceinline__ void pack32(int mode, const uint32_t (&v)[32], const 
     }
 }
 
+// The bias values of one warp's 128 output columns are fetched before the warp waits for its accumulator (the load
+// latency used to sit between the tensor-memory load and the arithmetic of every 32-column piece): lane l < 16 holds
+// the 16-byte piece l; piece 4 * ci + q, q = 0..3, of the ci-th 32-column piece is handed to every lane by shuffles.
+__device__ __forceinline__ uint4 bias_slice_load(const bf16 *bias, int64_t row_off, int32_t col_first, int32_t N, int lane) {
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (bias && lane < 16 && col_first + lane * 8 < N) v = *reinterpret_cast<const uint4 *>(bias + row_off + col_first + lane * 8);
+    return v;
+}
+__device__ __forceinline__ void bias_slice_piece(const uint4 &mine, int ci, uint4 (&out)[4]) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        out[q].x = __shfl_sync(0xffffffffu, mine.x, 4 * ci + q);
+        out[q].y = __shfl_sync(0xffffffffu, mine.y, 4 * ci + q);
+        out[q].z = __shfl_sync(0xffffffffu, mine.z, 4 * ci + q);
+        out[q].w = __shfl_sync(0xffffffffu, mine.w, 4 * ci + q);
+    }
+}
+
 struct Tile {
     int32_t e;        // expert / segment
     int32_t row0;     // ROW_*: first sorted row; WGRAD: first row of the segment
@@ -497,26 +515,32 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + A_BYTES;
+                int ksteps = BK / 16;  // K steps of 16 rows to issue for this block
                 if (KIND == WGRAD && kb == t.kblocks - 1) {
                     const int valid = t.row_end - (t.row0 + kb * BK);  // rows of this block inside the segment
                     if (valid < BK) {
-                        // zero K rows [valid, BK) of A and of B (they belong to the next segment: a non-finite value
-                        // there must not reach this segment's sums): 128-B lines in all 64-column chunks; the A tile's
-                        // two chunks are directly followed by the B tile's four
-                        const int lines = (BK - valid) * ((BM + BN) / 64);
+                        // The rows behind the segment's end belong to the next segment. Whole K steps behind it are not
+                        // issued at all; in the step that holds the end, K rows [valid, end of the step) are zeroed in A
+                        // AND in B (0 x finite = 0 would do for finite data; both keep a non-finite value of the next
+                        // segment out of this segment's sums): 128-B lines in all 64-column chunks, the A tile's two
+                        // chunks directly followed by the B tile's four.
+                        ksteps = (valid + 15) / 16;
+                        const int nz = ksteps * 16 - valid;
+                        const int lines = nz * ((BM + BN) / 64);
                         for (int u = lane; u < lines * 8; u += 32) {
                             const int line = u >> 3, part = u & 7;
-                            const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
+                            const int chunk = line / nz, krow = valid + line % nz;
                             *reinterpret_cast<uint4 *>(smem + s * STAGE_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
                                 make_uint4(0, 0, 0, 0);
                         }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        if (nz > 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                     }
                 }
                 if (lane == 0) {
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) {
+                        if (k >= ksteps) break;
                         uint64_t ad, bd;
                         if (KIND == WGRAD) ad = desc_mnmajor(a_src + k * 16 * 128);
                         else ad = desc_kmajor(a_src + k * 32);
@@ -597,6 +621,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 __syncwarp();  // the sums are read before the next tile overwrites them
                 continue;
             }
+            const int half_w = (warp - 2) >> 2;
+            const uint4 bias_mine = bias_slice_load(p.bias, (int64_t)t.e * p.N, t.n0 + half_w * (BN / 2), p.N, lane);
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
                 if (!ok) break;
@@ -633,6 +659,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
+                uint4 bias_raw[4];
+                if (p.bias) bias_slice_piece(bias_mine, c - half * (BN / 64), bias_raw);  // whole warp: shuffles
                 if (p.out_f32) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
@@ -649,12 +677,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     __syncwarp();
                 } else if (row_ok || p.colsum_part) {  // with column sums the whole warp takes part (shuffles)
                     uint4 packed[4];
-                    uint4 bias_raw[4], mask_raw[4];
-                    if (p.bias) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
-                    }
+                    uint4 mask_raw[4];
                     if (p.mask && row_ok) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
@@ -901,14 +924,16 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // rows [valid, 64) of stage s's A and B tiles (K rows past the segment end; two 64-column chunks each, the B tile
-    // directly behind the A tile) := 0. Zeroing A alone would do for finite data (0 x finite = 0); B as well keeps a
-    // non-finite value of the next segment out of this segment's sums.
+    // K rows past the segment end in stage s's A and B tiles (two 64-column chunks each, the B tile directly behind the
+    // A tile) := 0. Zeroing A alone would do for finite data (0 x finite = 0); B as well keeps a non-finite value of the
+    // next segment out of this segment's sums.
     auto zero_tail = [&](int s, int valid) {
-        const int lines = (BK - valid) * 4;
+        const int nz = ((valid + 15) / 16) * 16 - valid;  // up to the end of the K step of 16 that holds the segment's end:
+                                                           // the K steps behind it are not issued at all
+        const int lines = nz * 4;
         for (int u = lane; u < lines * 8; u += 32) {
             const int line = u >> 3, part = u & 7;
-            const int chunk = line / (BK - valid), krow = valid + line % (BK - valid);
+            const int chunk = line / nz, krow = valid + line % nz;
             *reinterpret_cast<uint4 *>(smem + s * STAGE2_BYTES + chunk * (BK * 128) + krow * 128 + part * 16) =
                 make_uint4(0, 0, 0, 0);
         }
@@ -1033,9 +1058,10 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     // K-major tile and by 16 rows of 128 bytes in an MN-major one; the sum never leaves the address field
                     constexpr uint64_t a_step = KIND == WGRAD ? (16 * 128) >> 4 : 32 >> 4;
                     constexpr uint64_t b_step = KIND == ROW_BK ? 32 >> 4 : (16 * 128) >> 4;
+                    const int ksteps = (KIND == WGRAD && kb == t.kblocks - 1) ? (tail_valid + 15) / 16 : BK / 16;
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
-                        tc_mma2_bf16(d_tmem, ad0 + k * a_step, bd0 + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                        if (k < ksteps) tc_mma2_bf16(d_tmem, ad0 + k * a_step, bd0 + k * b_step, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit2(empty_bar(s));
                     tr_issue += TILE_CLOCK() - ti0;
                     if (++s == NST) { s = 0; ph ^= 1u; }
@@ -1112,6 +1138,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const bool have_acc = t.kblocks > 0;
             ++trace_tile;
             if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 0, TILE_CLOCK());
+            const uint4 bias_mine = bias_slice_load(p.bias, (int64_t)t.e * p.N, t.n0 + half * (BN / 2), p.N, lane);
             if (have_acc) {
                 ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
                 if (!ok) break;
@@ -1159,6 +1186,8 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
+                uint4 bias_raw[4];
+                if (p.bias) bias_slice_piece(bias_mine, c - half * (BN / 64), bias_raw);  // whole warp: shuffles
                 if (p.out_f32) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q)
@@ -1175,12 +1204,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     __syncwarp();
                 } else if (row_ok || p.colsum_part) {  // with column sums the whole warp takes part (shuffles)
                     uint4 packed[4];
-                    uint4 bias_raw[4], mask_raw[4];
-                    if (p.bias) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            bias_raw[q] = reinterpret_cast<const uint4 *>(p.bias + (int64_t)t.e * p.N + col0)[q];
-                    }
+                    uint4 mask_raw[4];
                     if (MASKT) {  // from the tile in shared memory: row = this thread's row, 16-B pieces swizzled by row
                         const uint8_t *mrow_p = smem + NST * STAGE2_BYTES + (c >> 1) * 16384 + mrow * 128;
 #pragma unroll

