@@ -374,7 +374,8 @@ def run_ours(args, w):
     value = replicas.job_throughput(w.T, args.steps, total_ms, world)
     value_e2e = replicas.job_throughput(w.T, args.steps, total_e2e, world)
 
-    stages = stage_timings(B, cfg, S, D, w, timed, max(3, min(args.steps, 10)), peaks)
+    stages = stage_timings(B, cfg, S, D, w, (lambda: flush_buf.fill_(1)) if flush_buf is not None else (lambda: None),
+                           max(3, min(args.steps, 10)), peaks)
     # Roofline of the dominant kernel family, the expert grouped GEMMs (six launches per step). They are bound by the
     # tensor cores when the segments are long and by HBM when there are so many experts that every weight is read
     # for a handful of rows (c4): both fractions are computed from the algorithmic flop / bytes, the larger one binds.
@@ -540,7 +541,7 @@ def balance_metrics(D):
             "max_over_mean_count": float(counts.max() / counts.mean())}
 
 
-def stage_timings(B, cfg, S, D, w, timed, K, peaks):
+def stage_timings(B, cfg, S, D, w, flush, K, peaks):
     """Each stage call alone, K launches between events, on the tensors the fused forward saved."""
     V = B.ctx_views(cfg, D["ctx"])
     T, d, h, n, k, R = w.T, w.d, w.h, w.n, w.k, w.R
@@ -557,8 +558,10 @@ def stage_timings(B, cfg, S, D, w, timed, K, peaks):
                  4.0 * T * d * gate_cols, T * d * esz + 3 * 4 * T * gate_cols + 8 * R + 16 * T),
         "dispatch": (lambda: B.moe_dispatch(cfg, D["x"], V["topk_idx"], V["xs"], V["perm"], V["inv_perm"],
                                             V["counts"], V["offsets"], ws), 0.0, (1 + k) * T * d * esz + 12 * R),
-        "expert_ffn": (lambda: B.moe_expert_ffn(cfg, V["xs"], V["offsets"], D["W1"], D["b1"], D["W2"], D["b2"],
-                                                V["hid"], V["ys"], ws),
+        "expert_ffn": ((lambda: B.moe_expert_ffn_bits(cfg, V["xs"], V["offsets"], D["W1"], D["b1"], D["W2"], D["b2"],
+                                                      V["hid"], V["ys"], V["relu_bits"], ws)) if "relu_bits" in V else
+                       (lambda: B.moe_expert_ffn(cfg, V["xs"], V["offsets"], D["W1"], D["b1"], D["W2"], D["b2"],
+                                                 V["hid"], V["ys"], ws)),
                        4.0 * R * d * h, (2 * R * d + 2 * R * h) * esz + 2 * n * d * h * esz),
         "combine": (lambda: B.moe_combine(cfg, V["ys"], V["gates"], V["inv_perm"], D["y"]), 0.0,
                     (k + 1) * T * d * esz + 8 * R),
@@ -566,8 +569,12 @@ def stage_timings(B, cfg, S, D, w, timed, K, peaks):
                                         D["importance"], D["load"], D["losses"], ws), 0.0, 2 * 4 * T * gate_cols + 16 * R),
         "combine_bwd": (lambda: B.moe_combine_bwd(cfg, D["dY"], V["ys"], V["gates"], V["inv_perm"], dgates, dys), 0.0,
                         (1 + 2 * k) * T * d * esz + 12 * R),
-        "expert_ffn_bwd": (lambda: B.moe_expert_ffn_bwd(cfg, V["xs"], V["hid"], dys, V["offsets"], D["W1"], D["W2"],
-                                                        dxs, D["dW1"], D["db1"], D["dW2"], D["db2"], ws),
+        # the calls the fused path makes: with the ReLU mask as bits where the layer runs on the tensor cores
+        "expert_ffn_bwd": ((lambda: B.moe_expert_ffn_bwd_bits(cfg, V["xs"], V["hid"], V["relu_bits"], dys, V["offsets"],
+                                                              D["W1"], D["W2"], dxs, D["dW1"], D["db1"], D["dW2"],
+                                                              D["db2"], ws)) if "relu_bits" in V else
+                           (lambda: B.moe_expert_ffn_bwd(cfg, V["xs"], V["hid"], dys, V["offsets"], D["W1"], D["W2"],
+                                                         dxs, D["dW1"], D["db1"], D["dW2"], D["db2"], ws)),
                            8.0 * R * d * h, (4 * R * d + 3 * R * h) * esz + 4 * n * d * h * esz),
         "losses_bwd": (lambda: B.moe_losses_bwd(cfg, D["importance"], D["load"], V["topk_idx"], dgates, dload, ws),
                        0.0, 12 * R),
@@ -594,10 +601,25 @@ def stage_timings(B, cfg, S, D, w, timed, K, peaks):
     calls["adam_factored"] = (lambda: B.moe_expert_adam_factored(cfg, D["W1"], D["b1"], D["W2"], D["b2"], D["dW1"], D["db1"],
                                                                  D["dW2"], D["db2"], adam_state, 0.0, 0.999, 1e-8, 1, adam_ws),
                               0.0, 4 * 2 * n * d * h * esz)
+    # Every stage between its own pair of events, the stages taken in turn K times over (not K launches of one stage
+    # back to back): the chip then sits in the power and clock state of a real step, where tensor-core and streaming
+    # kernels alternate, instead of the state ten identical GEMM launches in a row drive it into.
+    for fn, _, _ in calls.values():
+        fn()
+    torch.cuda.synchronize()
+    ev = {name: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+          for name in calls}
+    for i in range(K):
+        for name, (fn, _, _) in calls.items():
+            a, b = ev[name][i]
+            flush()  # small workloads: L2 written over before every timed call
+            a.record()
+            fn()
+            b.record()
+    torch.cuda.synchronize()
     out = {}
     for name, (fn, flop, byts) in calls.items():
-        fn()
-        ms = statistics.mean(timed(fn, K))
+        ms = statistics.mean(a.elapsed_time(b) for a, b in ev[name])
         rec = {"ms": ms, "GB/s": byts / ms / 1e6, "hbm_frac": byts / ms / 1e6 / peaks["hbm_gbs"]}
         if flop:
             rec["TFLOP/s"] = flop / ms / 1e9

@@ -115,6 +115,8 @@ typedef struct moe_ctx_layout {
     int64_t xs, perm, inv_perm, counts, offsets;                  /* moe_dispatch outputs */
     int64_t hid, ys;                                              /* moe_expert_ffn outputs */
     int64_t importance, load, losses;                             /* moe_losses outputs   */
+    int64_t relu_bits; /* bf16 layers on the tensor cores that keep hid: [R, h/32] uint32, bit set where hid > 0 (the
+                          backward's ReLU mask, read instead of hid); absent otherwise */
 } moe_ctx_layout;
 
 /* Checks a configuration: positive sizes, 1 <= k <= min(n, MOE_MAX_K), n <= MOE_MAX_EXPERTS,
@@ -224,6 +226,17 @@ int32_t moe_dispatch_noalloc(const moe_config *cfg, const void *x, const int32_t
 int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
                        const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws,
                        void *stream);
+
+/* The same two calls with the ReLU mask as bits (bf16 layers whose widths are multiples of 64; MOE_ERR_UNSUPPORTED
+ * otherwise): moe_expert_ffn_bits also writes relu_bits [R, h/32] uint32 (bit j of word c of a row: hid[row, 32c+j] > 0),
+ * and moe_expert_ffn_bwd_bits masks dz with those bits instead of reading hid a second time as a mask (R*h/8 bytes
+ * instead of 2*R*h). Same results bit for bit. This is the path the fused calls take (moe_ctx_layout.relu_bits). */
+int32_t moe_expert_ffn_bits(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
+                            const void *b1, const void *W2, const void *b2, void *hid, void *ys, uint32_t *relu_bits,
+                            void *ws, void *stream);
+int32_t moe_expert_ffn_bwd_bits(const moe_config *cfg, const void *xs, const void *hid, const uint32_t *relu_bits,
+                                const void *dys, const int32_t *offsets, const void *W1, const void *W2, void *dxs,
+                                void *dW1, void *db1, void *dW2, void *db2, void *ws, void *stream);
 
 /* Combine (Eq. 1): y[t] = sum_s gates[t,s] * ys[inv_perm[t*k+s]], float sum in slot order.
  * `gates` is the [T,k] (product) gate tensor.   out: y [T,d] act */

@@ -25,7 +25,7 @@ EXPORTS = ["moe_debug_launch_count", "moe_validate", "moe_query_sizes", "moe_wor
            "moe_expert_ffn_bwd", "moe_dispatch_bwd", "moe_losses_bwd", "moe_gate_bwd", "moe_forward",
            "moe_backward", "moe_combine_layer", "moe_combine_layer_bwd", "moe_layer_forward", "moe_layer_backward",
            "moe_expert_adam_factored", "moe_check_buffer_sizes", "moe_debug_wait_timeout", "moe_debug_bounds_violations",
-           "moe_query_balanced_sizes", "moe_gate_balanced", "moe_dispatch_balanced", "moe_combine_balanced",
+           "moe_expert_ffn_bits", "moe_expert_ffn_bwd_bits", "moe_query_balanced_sizes", "moe_gate_balanced", "moe_dispatch_balanced", "moe_combine_balanced",
            "moe_combine_balanced_bwd", "moe_gate_balanced_bwd", "moe_dispatch_balanced_bwd"]
 
 
@@ -50,7 +50,7 @@ class moe_sizes(ctypes.Structure):
 class moe_ctx_layout(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int64) for name in
                 ("topk_idx", "gates", "clean", "raw_noise", "kth_vals", "kth_idx", "xs", "perm", "inv_perm",
-                 "counts", "offsets", "hid", "ys", "importance", "load", "losses")]
+                 "counts", "offsets", "hid", "ys", "importance", "load", "losses", "relu_bits")]
 
 
 class moe_balanced_sizes(ctypes.Structure):
@@ -176,6 +176,14 @@ def moe_dispatch_noalloc(cfg, x, topk_idx, xs, perm, inv_perm, counts, offsets):
 
 def moe_expert_ffn(cfg, xs, offsets, W1, b1, W2, b2, hid, ys, ws):
     _call("moe_expert_ffn", cfg, xs, offsets, W1, b1, W2, b2, hid, ys, ws)
+
+
+def moe_expert_ffn_bits(cfg, xs, offsets, W1, b1, W2, b2, hid, ys, relu_bits, ws):
+    _call("moe_expert_ffn_bits", cfg, xs, offsets, W1, b1, W2, b2, hid, ys, relu_bits, ws)
+
+
+def moe_expert_ffn_bwd_bits(cfg, xs, hid, relu_bits, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws):
+    _call("moe_expert_ffn_bwd_bits", cfg, xs, hid, relu_bits, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws)
 
 
 def moe_combine(cfg, ys, gates, inv_perm, y):
@@ -309,4 +317,6 @@ def ctx_views(cfg, ctx):
                 load=view(L.load, S.load_elems, torch.float32, (-1,)), losses=view(L.losses, 2, torch.float32, (2,)))
     if not cfg.flags & MOE_FLAG_RECOMPUTE_HID:  # with the flag the context keeps no hidden activations
         views["hid"] = view(L.hid, R * h, adt, (R, h))
+        if L.relu_bits + R * (h // 32) * 4 <= S.ctx_bytes and h % 32 == 0 and L.relu_bits > L.losses:
+            views["relu_bits"] = view(L.relu_bits, R * (h // 32), torch.int32, (R, h // 32))
     return views

@@ -278,8 +278,9 @@ struct Ctx {
     int32_t *topk_idx, *kth_idx, *perm, *inv_perm, *counts, *offsets;
     float *gates, *clean, *raw_noise, *kth_vals, *importance, *load, *losses;
     void *xs, *hid, *ys;
+    uint32_t *relu_bits;  // tensor-core layers that keep hid: one bit per hidden activation for the backward's ReLU mask
     moe_ctx_layout off;
-    Ctx(void *base, const Dims &D) {
+    Ctx(void *base, const Dims &D, bool has_bits) {
         Carver cv(base);
         auto at = [&]() { return (int64_t)cv.off; };
         off.topk_idx = at(); topk_idx = cv.take<int32_t>(D.R);
@@ -298,6 +299,8 @@ struct Ctx {
         off.importance = at(); importance = cv.take<float>(D.n);
         off.load = at(); load = cv.take<float>(D.load);
         off.losses = at(); losses = cv.take<float>(2);
+        off.relu_bits = at();
+        relu_bits = (has_bits && !(D.flags & MOE_FLAG_RECOMPUTE_HID)) ? cv.take<uint32_t>(D.R * (D.h / 32)) : nullptr;
         bytes = (int64_t)cv.off;
     }
     int64_t bytes;
@@ -399,12 +402,14 @@ SimtGemm base_gemm(const Dims &D) {
 // first_only: only hid = relu(xs.W1 + b1) is computed (ys is not touched).
 int32_t do_expert_ffn(const moe_config *c, const Dims &D, const void *xs, const int32_t *offsets, const void *W1,
                       const void *b1, const void *W2, const void *b2, void *hid, void *ys, void *ws_base,
-                      Carver &cv, cudaStream_t st, bool first_only = false, void **hid_used = nullptr) {
+                      Carver &cv, cudaStream_t st, bool first_only = false, void **hid_used = nullptr,
+                      uint32_t *relu_bits = nullptr) {
     FfnWs w(cv, D, c);
     if (!hid) hid = w.hid;
     if (!hid) return MOE_ERR_INVALID_ARG;
     if (hid_used) *hid_used = hid;
-    if (w.tc) return launch_tc_ffn(*c, xs, offsets, W1, b1, W2, b2, hid, ys, w.tc, status_word(ws_base), st, first_only);
+    if (w.tc)
+        return launch_tc_ffn(*c, xs, offsets, W1, b1, W2, b2, hid, ys, w.tc, status_word(ws_base), st, first_only, relu_bits);
     SimtGemm g = base_gemm(D);  // hid = relu(xs.W1 + b1)
     g.A = xs; g.B = W1; g.C = hid; g.bias = b1; g.relu = 1;
     g.sa_i = D.d; g.sa_k = 1; g.sb_k = D.h; g.sb_j = 1; g.sc_i = D.h; g.sc_j = 1;
@@ -450,12 +455,13 @@ int32_t do_losses(const moe_config *c, const Dims &D, const int32_t *topk_idx, c
 
 int32_t do_expert_ffn_bwd(const moe_config *c, const Dims &D, const void *xs, const void *hid, const void *dys,
                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
-                          void *dW2, void *db2, void *ws_base, Carver &cv, cudaStream_t st) {
+                          void *dW2, void *db2, void *ws_base, Carver &cv, cudaStream_t st,
+                          const uint32_t *relu_bits = nullptr) {
     FfnBwdWs w(cv, D);
     const int32_t n = (int32_t)D.n;
     if (tc_ffn_supported(*c))
         return launch_tc_ffn_bwd(*c, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, w.dz, w.colsum,
-                                 w.tile_prefix, status_word(ws_base), st);
+                                 w.tile_prefix, status_word(ws_base), st, relu_bits);
     MOE_TRY(launch_segment_colsum(dys, D.act, offsets, n, D.R, (int32_t)D.d, db2, w.colsum, w.tile_prefix, st));
     SimtGemm g = base_gemm(D);  // dW2[e] = hid_e^T . dys_e
     g.A = hid; g.B = dys; g.C = dW2;
@@ -642,7 +648,7 @@ int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *out) {
     out->ws_bytes = fwd > stage_bwd ? fwd : stage_bwd;
     out->ws_fwd_bytes = fwd;
     out->ws_bwd_bytes = measure([&](Carver &cv) { BwdWs w(cv, D); (void)w; }) + stage_bwd;
-    Ctx ctx(nullptr, D);
+    Ctx ctx(nullptr, D, tc_ffn_supported(*cfg));
     out->ctx_bytes = ctx.bytes;
     return MOE_OK;
 }
@@ -650,7 +656,7 @@ int32_t moe_query_sizes(const moe_config *cfg, moe_sizes *out) {
 int32_t moe_query_ctx_layout(const moe_config *cfg, moe_ctx_layout *out) {
     MOE_TRY(check_config(cfg));
     if (!out) return MOE_ERR_INVALID_ARG;
-    Ctx ctx(nullptr, dims_of(cfg));
+    Ctx ctx(nullptr, dims_of(cfg), tc_ffn_supported(*cfg));
     *out = ctx.off;
     return MOE_OK;
 }
@@ -729,6 +735,33 @@ int32_t moe_expert_ffn(const moe_config *cfg, const void *xs, const int32_t *off
     cv.take_bytes(kWsHeader);
     MOE_TRY(reset_status(ws, as_stream(stream)));
     return do_expert_ffn(cfg, D, xs, offsets, W1, b1, W2, b2, hid, ys, ws, cv, as_stream(stream));
+}
+
+int32_t moe_expert_ffn_bits(const moe_config *cfg, const void *xs, const int32_t *offsets, const void *W1,
+                            const void *b1, const void *W2, const void *b2, void *hid, void *ys, uint32_t *relu_bits,
+                            void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(xs, offsets, W1, b1, W2, b2, hid, ys, relu_bits, ws);
+    if (!tc_ffn_supported(*cfg)) return MOE_ERR_UNSUPPORTED;
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return do_expert_ffn(cfg, D, xs, offsets, W1, b1, W2, b2, hid, ys, ws, cv, as_stream(stream), false, nullptr, relu_bits);
+}
+
+int32_t moe_expert_ffn_bwd_bits(const moe_config *cfg, const void *xs, const void *hid, const uint32_t *relu_bits,
+                                const void *dys, const int32_t *offsets, const void *W1, const void *W2, void *dxs,
+                                void *dW1, void *db1, void *dW2, void *db2, void *ws, void *stream) {
+    MOE_TRY(check_config(cfg));
+    REQUIRE_PTRS(xs, hid, relu_bits, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws);
+    if (!tc_ffn_supported(*cfg)) return MOE_ERR_UNSUPPORTED;
+    const Dims D = dims_of(cfg);
+    Carver cv(ws);
+    cv.take_bytes(kWsHeader);
+    MOE_TRY(reset_status(ws, as_stream(stream)));
+    return do_expert_ffn_bwd(cfg, D, xs, hid, dys, offsets, W1, W2, dxs, dW1, db1, dW2, db2, ws, cv, as_stream(stream),
+                             relu_bits);
 }
 
 int32_t moe_combine(const moe_config *cfg, const void *ys, const float *gates, const int32_t *inv_perm, void *y,
@@ -814,7 +847,7 @@ static int32_t forward_impl(const moe_config *cfg, const void *x, const float *W
     if (keep_bits) MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
     const Dims D = dims_of(cfg);
     cudaStream_t st = as_stream(stream);
-    Ctx C(ctx, D);
+    Ctx C(ctx, D, tc_ffn_supported(*cfg));
     MOE_TRY(reset_status(ws, st));
     auto fresh = [&]() { Carver cv(ws); cv.take_bytes(kWsHeader); return cv; };
     { Carver cv = fresh();
@@ -823,7 +856,8 @@ static int32_t forward_impl(const moe_config *cfg, const void *x, const float *W
     { Carver cv = fresh();
       MOE_TRY(do_dispatch(D, x, C.topk_idx, C.xs, C.perm, C.inv_perm, C.counts, C.offsets, cv, st)); }
     { Carver cv = fresh();
-      MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st)); }  // C.hid null: stays in ws
+      MOE_TRY(do_expert_ffn(cfg, D, C.xs, C.offsets, W1, b1, W2, b2, C.hid, C.ys, ws, cv, st, false, nullptr,
+                            C.relu_bits)); }  // C.hid null: stays in ws
     MOE_TRY(launch_combine(C.ys, D.act, C.gates, C.inv_perm, D.T, (int32_t)D.k, (int32_t)D.d, y, st,
                            keep_bits ? x : nullptr, keep_bits, keep_bits ? 1.0f / (1.0f - drop_prob) : 1.0f));
     { Carver cv = fresh();
@@ -862,7 +896,7 @@ static int32_t backward_impl(const moe_config *cfg, const void *dY, const void *
     if (keep_bits) MOE_TRY(check_layer(cfg, keep_bits, drop_prob));
     const Dims D = dims_of(cfg);
     cudaStream_t st = as_stream(stream);
-    Ctx C(const_cast<void *>(ctx), D);
+    Ctx C(const_cast<void *>(ctx), D, tc_ffn_supported(*cfg));
     MOE_TRY(reset_status(ws, st));
     Carver base(ws);
     base.take_bytes(kWsHeader);
@@ -881,7 +915,7 @@ static int32_t backward_impl(const moe_config *cfg, const void *dY, const void *
           cv = fresh();
       }
       MOE_TRY(do_expert_ffn_bwd(cfg, D, C.xs, hid, B.dys, C.offsets, W1, W2, B.dxs, dW1, db1, dW2, db2, ws, cv,
-                                st)); }
+                                st, C.relu_bits)); }
     { Carver cv = fresh();
       MOE_TRY(do_losses_bwd(cfg, D, C.importance, C.load, C.topk_idx, B.dgates, B.dload, cv, st)); }
     { Carver cv = fresh();

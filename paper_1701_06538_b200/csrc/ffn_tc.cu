@@ -62,6 +62,10 @@ struct GemmParams {
     float *out_f32;    // if set, results are written here as float instead of `out`
     const bf16 *bias;  // [nseg, N] or nullptr
     const bf16 *mask;  // [R, N] or nullptr: result kept where mask > 0
+    // the same mask as one bit per element, [R, N / 32] words (bit j of word c: column 32 c + j): bits_out is written by
+    // the GEMM whose output the mask is taken of (bit = stored value > 0), bits_in is applied like `mask`
+    uint32_t *bits_out;
+    const uint32_t *bits_in;
     // ROW_* with bf16 output: if set, column sums of the stored values over each epilogue warp's 32 rows,
     // [32-row block][N] floats; block = (global M tile * CTAs per tile + CTA rank) * 4 + row quarter
     float *colsum_part;
@@ -260,9 +264,9 @@ __device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
 // Epilogue arithmetic of one thread's 32 accumulator columns: bias, ReLU, ReLU mask, rounding to bf16. The three
 // options are template parameters so that the loop body has no branches (with run-time flags every element pair became
 // its own basic block and the chain add -> max -> convert ran serially, 16 times).
-template <bool BIAS, bool RELU, bool MASK>
+template <bool BIAS, bool RELU, bool MASK, bool BITS = false>
 __device__ __forceinline__ void pack32_mode(const uint32_t (&v)[32], const uint4 (&bias_raw)[4], const uint4 (&mask_raw)[4],
-                                            uint4 (&packed)[4]) {
+                                            uint4 (&packed)[4], uint32_t keep_word = 0u) {
     const uint32_t *bw = reinterpret_cast<const uint32_t *>(bias_raw);
     const uint32_t *mw = reinterpret_cast<const uint32_t *>(mask_raw);
     uint32_t *out = reinterpret_cast<uint32_t *>(packed);
@@ -275,13 +279,33 @@ __device__ __forceinline__ void pack32_mode(const uint32_t (&v)[32], const uint4
             if (!(__uint_as_float(mw[j] << 16) > 0.0f)) x0 = 0.0f;
             if (!(__uint_as_float(mw[j] & 0xffff0000u) > 0.0f)) x1 = 0.0f;
         }
+        if (BITS) {
+            if (!((keep_word >> (2 * j)) & 1u)) x0 = 0.0f;
+            if (!((keep_word >> (2 * j + 1)) & 1u)) x1 = 0.0f;
+        }
         const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
         out[j] = *reinterpret_cast<const uint32_t *>(&h);
     }
 }
-// mode: bit 0 bias, bit 1 ReLU, bit 2 mask (the combinations the layer uses are specialised)
+// one bit per packed value: set where the stored bf16 value is greater than zero
+__device__ __forceinline__ uint32_t positive_bits(const uint4 (&packed)[4]) {
+    const uint32_t *pw = reinterpret_cast<const uint32_t *>(packed);
+    uint32_t word = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const uint32_t lo = pw[j] & 0xffffu, hi = pw[j] >> 16;
+        word |= (uint32_t)(lo != 0u && !(lo & 0x8000u)) << (2 * j);
+        word |= (uint32_t)(hi != 0u && !(hi & 0x8000u)) << (2 * j + 1);
+    }
+    return word;
+}
+// mode: bit 0 bias, bit 1 ReLU, bit 2 mask, bit 3 mask as bits (the combinations the layer uses are specialised)
 __device__ __forceinline__ void pack32(int mode, const uint32_t (&v)[32], const uint4 (&bias_raw)[4],
-                                       const uint4 (&mask_raw)[4], uint4 (&packed)[4]) {
+                                       const uint4 (&mask_raw)[4], uint4 (&packed)[4], uint32_t keep_word = 0u) {
+    if (mode & 8) {
+        pack32_mode<false, false, false, true>(v, bias_raw, mask_raw, packed, keep_word);
+        return;
+    }
     switch (mode) {
         case 0: pack32_mode<false, false, false>(v, bias_raw, mask_raw, packed); break;
         case 1: pack32_mode<true, false, false>(v, bias_raw, mask_raw, packed); break;
@@ -567,7 +591,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter + 31 belong to this warp
-        const int pack_mode = (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
+        const int pack_mode = p.bits_in ? 8 : (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
@@ -683,7 +707,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int q = 0; q < 4; ++q)
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
                     }
-                    pack32(pack_mode, v, bias_raw, mask_raw, packed);
+                    uint32_t keep_word = 0u;
+                    if (p.bits_in && row_ok) keep_word = p.bits_in[out_row * (p.N >> 5) + (col0 >> 5)];
+                    pack32(pack_mode, v, bias_raw, mask_raw, packed, keep_word);
+                    if (p.bits_out && row_ok) p.bits_out[out_row * (p.N >> 5) + (col0 >> 5)] = positive_bits(packed);
                     if (row_ok) {
                         uint4 *dst = reinterpret_cast<uint4 *>(p.out + out_off + out_row * p.N + col0);
                         st_global_32B(dst, packed[0], packed[1]);  // two full 32-byte sectors per row piece
@@ -1125,7 +1152,7 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         const int quarter = warp & 3, half = (warp - 2) >> 2;
-        const int pack_mode = (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
+        const int pack_mode = p.bits_in ? 8 : (p.bias ? 1 : 0) | (p.relu ? 2 : 0) | (p.mask ? 4 : 0);
         uint8_t *stage_o = smem + NST * STAGE2_BYTES + (warp - 2) * 4096;
         uint32_t mask_ph = 0;
         int acc = 0;
@@ -1139,12 +1166,6 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ++trace_tile;
             if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 0, TILE_CLOCK());
             const uint4 bias_mine = bias_slice_load(p.bias, (int64_t)t.e * p.N, t.n0 + half * (BN / 2), p.N, lane);
-            if (have_acc) {
-                ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
-                if (!ok) break;
-                tc_fence_after();
-            }
-            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 1, TILE_CLOCK());
             long long tr_ld = 0, tr_st = 0, tr_pack = 0;
             int64_t tile_row0, out_off = 0;
             int32_t rows_valid;
@@ -1159,6 +1180,21 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const int my_piece = lane & 7, my_sub = lane >> 3;
             const bool row_ok = lane < rows_valid;
             const int64_t out_row = tile_row0 + lane;
+            uint4 keep4 = make_uint4(0, 0, 0, 0);  // the mask bits of this thread's row for the warp's four 32-column pieces
+            if (p.bits_in && row_ok) {
+                const uint32_t *kw = p.bits_in + out_row * (p.N >> 5) + ((t.n0 + half * (BN / 2)) >> 5);
+                const int left = (p.N - (t.n0 + half * (BN / 2))) >> 5;  // words that exist in this row from here on
+                if (left > 0) keep4.x = kw[0];
+                if (left > 1) keep4.y = kw[1];
+                if (left > 2) keep4.z = kw[2];
+                if (left > 3) keep4.w = kw[3];
+            }
+            if (have_acc) {  // (the loads above are in flight while the warp waits for its accumulator)
+                ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            if (warp == 2 && lane == 0) TILE_TRACE_SET(2, trace_tile, 1, TILE_CLOCK());
             if (MASKT) {
                 ok = mbar_wait(mfull_bar, mask_ph, abort_flag, p.status);
                 if (!ok) break;
@@ -1216,7 +1252,9 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             mask_raw[q] = reinterpret_cast<const uint4 *>(p.mask + out_row * p.N + col0)[q];
                     }
                     const long long tp0 = TILE_CLOCK();
-                    pack32(pack_mode, v, bias_raw, mask_raw, packed);
+                    const int ci = c - half * (BN / 64);
+                    pack32(pack_mode, v, bias_raw, mask_raw, packed, ci == 0 ? keep4.x : ci == 1 ? keep4.y : ci == 2 ? keep4.z : keep4.w);
+                    if (p.bits_out && row_ok) p.bits_out[out_row * (p.N >> 5) + (col0 >> 5)] = positive_bits(packed);
                     tr_pack += TILE_CLOCK() - tp0;
                     if (staged) {
                         uint8_t *blk = smem + NST * STAGE2_BYTES + (c >> 1) * 16384;
@@ -1587,7 +1625,8 @@ int64_t tc_colsum_part_floats(int64_t R, int32_t nseg, int32_t N) { return (cdiv
 int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t *offsets, int32_t nseg, int64_t R,
                     int32_t N, int32_t K, void *out, const void *bias, const void *mask, int relu,
                     int32_t *tile_prefix, int32_t *status, cudaStream_t st, int32_t flags,
-                    float *colsum_part = nullptr, void *colsum_out = nullptr) {
+                    float *colsum_part = nullptr, void *colsum_out = nullptr, uint32_t *bits_out = nullptr,
+                    const uint32_t *bits_in = nullptr) {
     if (R == 0) {
         if (colsum_out) MOE_CUDA(cudaMemsetAsync(colsum_out, 0, sizeof(bf16) * (size_t)nseg * N, st));
         return MOE_OK;
@@ -1605,6 +1644,8 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     p.offsets = offsets; p.tile_prefix = tile_prefix; p.tile_info = tile_info_of(tile_prefix, nseg);
     p.nseg = nseg; p.M = 0; p.N = N; p.K = K; p.R = R;
     p.out = (bf16 *)out; p.bias = (const bf16 *)bias; p.mask = (const bf16 *)mask; p.relu = relu; p.status = status;
+    p.bits_out = bits_out; p.bits_in = bits_in;
+    if (bits_in) p.mask = nullptr;  // the bits replace the element-wise mask tensor
     p.colsum_part = colsum_out ? colsum_part : nullptr;
     if (use_two_cta(R, nseg, flags)) {  // segments long enough to fill 256-row tiles: SM pairs
         if (transposed) MOE_TRY(map_weight_kmajor_half(&tmB, W, nseg, N, K));
@@ -1621,7 +1662,7 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
             const uint32_t box[2] = {64, 32};
             MOE_TRY(make_map(&tmO, out, 2, dims, str, box));
         }
-        if (transposed && mask) {  // the ReLU-mask rows come in as TMA tiles
+        if (transposed && mask && !bits_in) {  // the ReLU-mask rows come in as TMA tiles
             CUtensorMap tmM;
             MOE_TRY(map_rows_kmajor(&tmM, mask, R, N));
             return finish(launch2<ROW_BK, true>(tmA, tmB, p, max_tiles2, st, &tmM, &tmO), 8);
@@ -1681,10 +1722,11 @@ int32_t tc_wgrad_gemm(const void *A, const void *B, const int32_t *offsets, int3
 
 int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offsets, const void *W1, const void *b1,
                       const void *W2, const void *b2, void *hid, void *ys, void *ws, int32_t *status_word,
-                      cudaStream_t st, bool first_only) {
+                      cudaStream_t st, bool first_only, uint32_t *relu_bits) {
     const int64_t R = (int64_t)c.T * c.k;
     int32_t *tile_prefix = static_cast<int32_t *>(ws);
-    MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st, c.flags));
+    MOE_TRY(tc_row_gemm(xs, W1, false, offsets, c.n, R, c.h, c.d, hid, b1, nullptr, 1, tile_prefix, status_word, st, c.flags,
+                        nullptr, nullptr, relu_bits));
     if (first_only) return MOE_OK;
     return tc_row_gemm(hid, W2, false, offsets, c.n, R, c.d, c.h, ys, b2, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }
@@ -1906,12 +1948,13 @@ int32_t launch_tc_hier_secondary_bwd(const void *xs_p, const void *dsplit_s, voi
 int32_t launch_tc_ffn_bwd(const moe_config &c, const void *xs, const void *hid, const void *dys,
                           const int32_t *offsets, const void *W1, const void *W2, void *dxs, void *dW1, void *db1,
                           void *dW2, void *db2, void *dz, float *colsum, int32_t *tile_prefix, int32_t *status_word,
-                          cudaStream_t st) {
+                          cudaStream_t st, const uint32_t *relu_bits) {
     const int64_t R = (int64_t)c.T * c.k;
     MOE_TRY(launch_segment_colsum(dys, c.act, offsets, c.n, R, c.d, db2, colsum, tile_prefix, st));
     MOE_TRY(tc_wgrad_gemm(hid, dys, offsets, c.n, R, c.h, c.d, dW2, status_word, st, c.flags, tile_prefix));
     // db1 = column sums of dz, formed in the epilogue of the GEMM that produces dz
-    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, c.flags, colsum, db1));
+    MOE_TRY(tc_row_gemm(dys, W2, true, offsets, c.n, R, c.h, c.d, dz, nullptr, hid, 0, tile_prefix, status_word, st, c.flags, colsum, db1,
+                        nullptr, relu_bits));
     MOE_TRY(tc_wgrad_gemm(xs, dz, offsets, c.n, R, c.d, c.h, dW1, status_word, st, c.flags, tile_prefix));
     return tc_row_gemm(dz, W1, true, offsets, c.n, R, c.d, c.h, dxs, nullptr, nullptr, 0, tile_prefix, status_word, st, c.flags);
 }

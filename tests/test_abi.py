@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.moe_config) == 52
     assert ctypes.sizeof(B.moe_sizes) == 14 * 8
-    assert ctypes.sizeof(B.moe_ctx_layout) == 16 * 8
+    assert ctypes.sizeof(B.moe_ctx_layout) == 17 * 8
 
 
 def test_validate_accepts_the_five_workloads_and_rejects_bad_ones(lib):

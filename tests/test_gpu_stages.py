@@ -391,3 +391,30 @@ def test_non_finite_rows_of_one_expert_do_not_reach_the_others_weight_gradients(
         others = [e for e in range(w.n) if e != bad]
         for name, got, want in (("dW1", dW1, Bk.dW1), ("dW2", dW2, Bk.dW2), ("db1", db1, Bk.db1), ("db2", db2, Bk.db2)):
             assert_close(host(got)[others], np.asarray(want)[others], tol_act(w), name)
+
+
+def test_expert_stages_with_the_relu_mask_as_bits(case):
+    """moe_expert_ffn_bits / moe_expert_ffn_bwd_bits: the mask bits are exactly [hid > 0], and the backward that reads
+    them gives bit for bit what the backward that reads hid gives."""
+    w, I, F, Bk, D, cfg = case
+    if not (w.act == "bf16" and w.d % 64 == 0 and w.h % 64 == 0):
+        with pytest.raises(B.MoeError):
+            B.moe_expert_ffn_bits(cfg, dev_act(F.D.xs, w), dev(F.D.offsets), D["W1"], D["b1"], D["W2"], D["b2"],
+                                  act_empty(w, 1, 1), act_empty(w, 1, 1), i32(8), B.empty_bytes(1024))
+        return
+    ws, S = ws_for(cfg)
+    hid, ys = act_empty(w, S.R, w.h), act_empty(w, S.R, w.d)
+    bits = torch.full((S.R, w.h // 32), -1, dtype=torch.int32, device="cuda")
+    xs, offs = dev_act(F.D.xs, w), dev(F.D.offsets)
+    B.moe_expert_ffn_bits(cfg, xs, offs, D["W1"], D["b1"], D["W2"], D["b2"], hid, ys, bits, ws)
+    assert B.moe_check_status(ws) == 0
+    want = np.packbits(host(hid) > 0, axis=1, bitorder="little").view(np.uint32)
+    assert (host(bits).view(np.uint32) == want).all()
+    dys = dev_act(Bk.dys, w)
+    a = [act_empty(w, S.R, w.d), act_empty(w, w.n, w.d, w.h), act_empty(w, w.n, w.h), act_empty(w, w.n, w.h, w.d), act_empty(w, w.n, w.d)]
+    b = [torch.empty_like(t) for t in a]
+    B.moe_expert_ffn_bwd(cfg, xs, hid, dys, offs, D["W1"], D["W2"], *a, ws)
+    B.moe_expert_ffn_bwd_bits(cfg, xs, hid, bits, dys, offs, D["W1"], D["W2"], *b, ws)
+    assert B.moe_check_status(ws) == 0
+    for name, p, q in zip(("dxs", "dW1", "db1", "dW2", "db2"), a, b):
+        assert torch.equal(p, q), name
