@@ -108,6 +108,8 @@ struct GateWs {
     float *cr, *wnorm, *xnorm, *wt;
     void *wsplit;
     int32_t *unsafe_list, *unsafe_count, *full_list;
+    float *unsafe_low, *unsafe_low_s;
+    void *unsafe_span, *unsafe_span_s;  // int2 per listed row
     void *chain_list;
     // the same for the secondary gates of the hierarchical layer (rows = slots sorted by primary group)
     bool screen2;
@@ -116,7 +118,7 @@ struct GateWs {
     int32_t *unsafe_list_s, *unsafe_count_s;
     GateWs(Carver &cv, const Dims &D) {
         screen2 = false;
-        xs_p = wsplit_s = chain_list_s = nullptr; cr_s = wnorm_s = wt_s = nullptr; unsafe_list_s = unsafe_count_s = nullptr;
+        xs_p = wsplit_s = chain_list_s = nullptr; cr_s = wnorm_s = wt_s = nullptr; unsafe_list_s = unsafe_count_s = nullptr; unsafe_low = unsafe_low_s = nullptr; unsafe_span = unsafe_span_s = nullptr;
         idx_p = idx_s = perm_p = inv_perm_p = counts_p = offsets_p = scratch = tile_prefix = nullptr;
         cr = wnorm = xnorm = wt = nullptr; wsplit = nullptr; unsafe_list = unsafe_count = full_list = nullptr; chain_list = nullptr;
         const int64_t n1 = D.hier ? D.a : D.n;  // width of the (first) gate
@@ -128,6 +130,8 @@ struct GateWs {
             wt = cv.take<float>(2 * n1 * D.d);
             xnorm = cv.take<float>(D.T);
             unsafe_list = cv.take<int32_t>(D.T);
+            unsafe_low = cv.take<float>(D.T);
+            unsafe_span = cv.take_bytes(D.T * 8);
             unsafe_count = cv.take<int32_t>(64);
             full_list = cv.take<int32_t>(D.T);
             chain_list = cv.take_bytes(D.T * 2 * SCREEN_MAX_CAND * 8);
@@ -151,6 +155,8 @@ struct GateWs {
             wnorm_s = cv.take<float>(D.a * 2 * D.b);
             wt_s = cv.take<float>(D.a * 2 * D.b * D.d);
             unsafe_list_s = cv.take<int32_t>(P1);
+            unsafe_low_s = cv.take<float>(P1);
+            unsafe_span_s = cv.take_bytes(P1 * 8);
             unsafe_count_s = cv.take<int32_t>(64);
             chain_list_s = cv.take_bytes(P1 * 2 * D.b * 8);  // worst case: every column of every slot
         }
@@ -331,18 +337,18 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
     auto first_gate = [&](int32_t n1, int32_t k1, int32_t *idx_out, float *gates_out) -> int32_t {
         if (w.screen) {
             MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, w.wsplit, w.wnorm, w.xnorm,
-                                               w.unsafe_count, w.wt, st));
+                                               w.unsafe_count, w.wt, st, 1, false));  // the screen forms the row norms
             MOE_TRY(launch_tc_gate_fwd(x, D.T, (int32_t)D.d, n1, w.wsplit, w.cr, status_word(ws_base), st));
             MOE_TRY(launch_gate_screen(w.cr, noise, w.xnorm, w.wnorm, (int32_t)D.d, D.T, n1, k1, idx_out, gates_out,
-                                       clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_count, w.chain_list,
-                                       w.full_list, st));
+                                       clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_low, w.unsafe_count,
+                                       w.chain_list, w.full_list, st, nullptr, 1, nullptr, w.unsafe_span, x));
             // exact chains for the few columns that decide an uncertain row; whole rows only where there are many
             MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, n1, w.wt, w.chain_list, w.unsafe_count + 1, clean, raw_noise,
                                        st));
             MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, clean, raw_noise, nullptr, 0,
                                       w.full_list, 1, nullptr, st, w.unsafe_count + 2));
             return launch_gate_select(clean, raw_noise, noise, D.T, n1, k1, idx_out, gates_out, kth_vals, kth_idx, st,
-                                      w.unsafe_list, w.unsafe_count);
+                                      w.unsafe_list, w.unsafe_count, w.unsafe_span, w.chain_list);
         }
         MOE_TRY(launch_projection(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, clean, raw_noise, nullptr, 0, nullptr, 1,
                                   nullptr, st));
@@ -367,12 +373,13 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
                                            w.tile_prefix, w.cr_s, status_word(ws_base), st, D.flags));
         MOE_TRY(launch_gate_screen(w.cr_s, noise + lp, w.xnorm, w.wnorm_s, (int32_t)D.d, P1, (int32_t)D.b, (int32_t)D.k2,
                                    w.idx_s, g_s, clean + lp, raw_noise + lp, kth_vals + 2 * D.T, kth_idx + 2 * D.T,
-                                   w.unsafe_list_s, w.unsafe_count_s, w.chain_list_s, nullptr, st, w.perm_p,
-                                   (int32_t)D.k1, w.idx_p));
+                                   w.unsafe_list_s, w.unsafe_low_s, w.unsafe_count_s, w.chain_list_s, nullptr, st, w.perm_p,
+                                   (int32_t)D.k1, w.idx_p, w.unsafe_span_s, nullptr));
         MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, (int32_t)D.b, w.wt_s, w.chain_list_s, w.unsafe_count_s + 1,
                                    clean + lp, raw_noise + lp, st, (int32_t)D.k1));
         MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s, g_s,
-                                   kth_vals + 2 * D.T, kth_idx + 2 * D.T, st, w.unsafe_list_s, w.unsafe_count_s));
+                                   kth_vals + 2 * D.T, kth_idx + 2 * D.T, st, w.unsafe_list_s, w.unsafe_count_s, w.unsafe_span_s,
+                                   w.chain_list_s));
     } else {
         MOE_TRY(launch_projection(x, D.act, P1, (int32_t)D.d, (int32_t)D.b, Wg_s, Wn_s, clean + lp, raw_noise + lp,
                                   w.offsets_p, (int32_t)D.a, w.perm_p, (int32_t)D.k1, w.tile_prefix, st));

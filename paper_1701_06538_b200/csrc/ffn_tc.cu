@@ -861,11 +861,20 @@ template <int KIND> struct PairTiles {
         const uint32_t par = (uint32_t)(i / SCHED_SLOTS) & 1u;
         if (!mbar_wait(full0 + 8u * slot, par, abort_flag, p.status)) return false;
         mbar_try_wait_cluster(full0 + 8u * slot, par);  // acquire at cluster scope: the record came from the other CTA's thread
+        // The slot is overwritten once every reader has reported it read, so a reader's copy has to be in its registers
+        // before its report leaves. The report is a relaxed arrive (a release at cluster scope would wait for the thread's
+        // earlier output stores, 3 % of a step), which by itself orders nothing: with an ordinary load the assembler was
+        // free to fetch the record again later instead of keeping it in registers, and in the register-heaviest epilogue
+        // (mask bits + column sums) one warp then now and again worked on the record of four tiles ahead and left its
+        // piece of the output unwritten. Hence a volatile load (issued once, where it stands) and an arrive whose address
+        // is computed from the loaded words of all lanes (sign bit of the tile id, always 0), which cannot issue before
+        // those loads have returned.
         int4 rec;
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rec.x), "=r"(rec.y), "=r"(rec.z), "=r"(rec.w)
+        asm volatile("ld.volatile.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rec.x), "=r"(rec.y), "=r"(rec.z), "=r"(rec.w)
                      : "r"(ring + 16u * slot) : "memory");
-        if (warp_wide) __syncwarp();  // every lane has its copy before the slot is reported as read
-        if (arrives) mbar_arrive_leader_relaxed(empty0 + 8u * slot);
+        uint32_t seen = (uint32_t)rec.w;
+        if (warp_wide) seen = __reduce_or_sync(0xffffffffu, seen);
+        if (arrives) mbar_arrive_leader_relaxed(empty0 + 8u * slot + ((seen >> 31) << 3));
         ++i;
         if (rec.x < 0) return false;
         MOE_BOUNDS_NOTE(rec.x < p.nseg && rec.y >= 0 && rec.y <= rec.z && (int64_t)rec.z <= p.R);

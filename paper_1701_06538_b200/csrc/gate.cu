@@ -210,11 +210,17 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
                                                           float *__restrict__ gates, float *__restrict__ kth_vals,
                                                           int32_t *__restrict__ kth_idx,
                                                           const int32_t *__restrict__ row_list,
-                                                          const int32_t *__restrict__ row_count) {
+                                                          const int32_t *__restrict__ row_count,
+                                                          const int2 *__restrict__ row_span,
+                                                          const int2 *__restrict__ chain_list) {
     const int lane = threadIdx.x & 31;
     int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // row_span (with a row list): {first chain entry, number of candidate columns} of a listed row whose other
+    // columns are known to rank below k + 1, so only the candidates are looked at; {., -1}: every column
+    int32_t cand_base = 0, cand_total = -1;
     if (row_list) {  // only the listed rows (their number is read on the device)
         if (row >= *row_count) return;
+        if (row_span) { const int2 sp = row_span[row]; cand_base = sp.x; cand_total = sp.y; }
         row = row_list[row];
     } else if (row >= rows) {
         return;
@@ -224,7 +230,10 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
 #pragma unroll
     for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; }
     const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
-    for (int32_t j = lane; j < n; j += 32) {
+    const int32_t visits = cand_total >= 0 ? cand_total : n;
+    for (int32_t q = lane; q < visits; q += 32) {
+        // a candidate's column is the code of its first chain entry (the clean one), modulo the group's block of 2n
+        const int32_t j = cand_total >= 0 ? chain_list[cand_base + 2 * q].y % (2 * n) : q;
         const double rd = (double)r[j];
         const float sigma = (float)(fmax(rd, 0.0) + log1p(exp(-fabs(rd))));
         float v = fmaf(e[j], sigma, c[j]);
@@ -283,11 +292,13 @@ __global__ void __launch_bounds__(256) gate_select_kernel(const float *__restric
 
 int32_t launch_gate_select(const float *clean, const float *raw, const float *noise, int64_t rows, int32_t n,
                            int32_t k, int32_t *idx, float *gates, float *kth_vals, int32_t *kth_idx,
-                           cudaStream_t st, const int32_t *row_list, const int32_t *row_count) {
+                           cudaStream_t st, const int32_t *row_list, const int32_t *row_count, const void *row_span,
+                           const void *chain_list) {
     if (rows == 0) return MOE_OK;
     const unsigned grid = (unsigned)cdiv(rows, 8);
-#define MOE_SELECT(KL) \
-    gate_select_kernel<KL><<<grid, 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates, kth_vals, kth_idx, row_list, row_count)
+#define MOE_SELECT(KL)                                                                                                 \
+    gate_select_kernel<KL><<<grid, 256, 0, st>>>(clean, raw, noise, rows, n, k, idx, gates, kth_vals, kth_idx, row_list, \
+                                                 row_count, (const int2 *)row_span, (const int2 *)chain_list)
     if (k <= 2) MOE_SELECT(3);
     else if (k <= 4) MOE_SELECT(5);
     else MOE_SELECT(MOE_MAX_K + 1);
@@ -352,194 +363,300 @@ __global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x
     if (lane == 0) xnorm[t] = sqrtf(s) * (1.0f + 1e-5f);
 }
 
-// NV: columns per lane (n <= 32 * NV), 0: any n, plain loop. KL: length of the per-lane sorted lists, >= k + 2
-// (short lists for small k: the insertion into them is most of this kernel's instructions)
-template <int NV, int KL>
-__global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
-                                                          const float *__restrict__ xnorm,
-                                                          const float *__restrict__ wnorm, float theta, int64_t T,
-                                                          int32_t n, int32_t k, int32_t *__restrict__ idx,
-                                                          float *__restrict__ gates, float *__restrict__ clean,
-                                                          float *__restrict__ raw, float *__restrict__ kth_vals,
-                                                          int32_t *__restrict__ kth_idx,
-                                                          int32_t *__restrict__ unsafe_list,
-                                                          int32_t *__restrict__ unsafe_count,
-                                                          int2 *__restrict__ chain_list,
-                                                          int32_t *__restrict__ full_list,
-                                                          const int32_t *__restrict__ perm, int32_t kdiv,
-                                                          const int32_t *__restrict__ group_of) {
-    // Grouped use (secondary gates of the hierarchical layer): cr rows are sorted by group; perm maps a sorted row to
-    // its output row (the slot t * k1 + s1), the token is output row / kdiv, group_of gives the slot's group, whose
-    // column norms and weight rows are used. Flat use: perm = group_of = nullptr, kdiv = 1.
-    const int lane = threadIdx.x & 31;
-    const int64_t srow = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (srow >= T) return;
-    const int64_t row = perm ? perm[srow] : srow;
-    const int32_t group = group_of ? group_of[row] : 0;
-    wnorm += (int64_t)group * 2 * n;
-    // per-lane sorted list of (value, index, uncertainty); rest_hi = largest possible chain value of anything
-    // that is not in a list
+// Approximate noisy logit v of one column and a bound u on its distance from the fma chain's value; c, r = the
+// tensor-core products, e = the noise, xn = theta |x|, wg / wn = the column norms of W_g / W_noise. Both screening
+// kernels call this one function, written with the non-contracting intrinsics so that they get the same bits.
+// The hardware exponential and logarithm are enough here: their error is an absolute 7.2e-7 at most on sigma (2.4e-7
+// from __expf on [-inf, 0], 1.2e-7 from rounding 1 + y, 2^-21.41 from __logf on [1, 2]) and goes into u with a margin
+// (2e-6 |noise|).
+__device__ __forceinline__ void screen_eval(float c, float r, float e, float xn, float wg, float wn, float &v, float &u) {
+    const float sigma = __fadd_rn(fmaxf(r, 0.0f), __logf(__fadd_rn(1.0f, __expf(-fabsf(r)))));
+    v = __fmaf_rn(e, sigma, c);
+    // |H~_j - H_j|: projection errors through c and through softplus(r) (slope <= 1) times |noise|, plus the error of
+    // softplus (here approximate, there double rounded once) and of the final fma on both sides
+    const float ae = fabsf(e);
+    const float rounding = __fmul_rn(1.1920929e-7f, __fmaf_rn(16.0f * ae, sigma, 8.0f * fabsf(v)));
+    u = __fmaf_rn(2.0e-6f, ae, __fmaf_rn(xn, __fmaf_rn(ae, wn, wg), rounding));
+}
+
+// The screen, one thread per token (sorted row): a warp stages 16 columns of its 32 rows at a time through shared memory
+// (16-byte loads along the rows, 16-byte reads down the rows, both conflict free with a pitch of 20 words), copies
+// them to clean / raw on the way, and every thread then walks its own row: a sorted list of the KL >= k + 2 largest
+// approximate logits with their bounds, and the largest possible value of everything else. No shuffles, no arg-max
+// rounds: a few dozen instructions per column. Certified rows get their routing here; the others are listed
+// with `low`, the bound that decides which of their columns need an exact chain (gate_candidates_kernel).
+// Grouped use (secondary gates of the hierarchical layer): cr rows are sorted by group; perm maps a sorted row to its
+// output row (the slot t * k1 + s1), the token is output row / kdiv, group_of gives the slot's group, whose column
+// norms are used. Flat use: perm = group_of = nullptr, kdiv = 1.
+constexpr int SCREEN_CH = 16, SCREEN_PITCH = 20;
+// four floats at p: one 16-byte access where the tensor allows it (V16), else four 4-byte ones (the secondary gates'
+// part of noise / clean / raw starts T * a floats into the tensor, not always a multiple of four)
+template <bool V16>
+__device__ __forceinline__ float4 load4(const float *p) {
+    if constexpr (V16) return *reinterpret_cast<const float4 *>(p);
+    else return make_float4(p[0], p[1], p[2], p[3]);
+}
+template <bool V16>
+__device__ __forceinline__ void store4(float *p, float4 v) {
+    if constexpr (V16) *reinterpret_cast<float4 *>(p) = v;
+    else { p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w; }
+}
+template <int KL, bool V16>
+__global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
+                                                               const bf16 *__restrict__ x, int32_t d,
+                                                               float *__restrict__ xnorm,
+                                                               const float *__restrict__ wnorm, float theta, int64_t T,
+                                                               int32_t n, int32_t k, int32_t *__restrict__ idx,
+                                                               float *__restrict__ gates, float *__restrict__ clean,
+                                                               float *__restrict__ raw, float *__restrict__ kth_vals,
+                                                               int32_t *__restrict__ kth_idx,
+                                                               int32_t *__restrict__ unsafe_list,
+                                                               float *__restrict__ unsafe_low,
+                                                               int32_t *__restrict__ unsafe_count,
+                                                               const int32_t *__restrict__ perm, int32_t kdiv,
+                                                               const int32_t *__restrict__ group_of) {
+    __shared__ __align__(16) float tile[4][3][32 * SCREEN_PITCH];
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int64_t s0 = ((int64_t)blockIdx.x * 4 + wp) * 32;  // first sorted row of this warp
+    if (s0 >= T) return;
+    const int64_t srow = s0 + lane;
+    const bool live = srow < T;
+    const int64_t row = live ? (perm ? (int64_t)perm[srow] : srow) : 0;
+    const float *wn = wnorm + (int64_t)(group_of && live ? group_of[row] : 0) * 2 * n;
+    float xnr;
+    if (x) {
+        // |x_t|_2 of the warp's 32 rows, here rather than in a pass of its own (flat use: row = srow; d a multiple of
+        // 256): the warp reads a row with 16-byte loads, four rows in flight, lane i keeps the norm of row i and
+        // publishes it for the later kernels
+        xnr = 0.0f;
+        for (int i0 = 0; i0 < 32; i0 += 4) {
+            float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            for (int32_t q = lane * 8; q < d; q += 256) {
+                uint4 raw4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int64_t sr = min(s0 + i0 + i, T - 1);
+                    raw4[i] = *reinterpret_cast<const uint4 *>(x + sr * d + q);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const bf16 *hx = reinterpret_cast<const bf16 *>(&raw4[i]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { const float v = __bfloat162float(hx[e]); part[i] = fmaf(v, v, part[i]); }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) part[i] += __shfl_xor_sync(0xffffffffu, part[i], off);
+                if (lane == i0 + i) xnr = sqrtf(part[i]) * (1.0f + 1e-5f);
+            }
+        }
+        if (live) xnorm[row] = xnr;
+    } else {
+        xnr = live ? xnorm[row / kdiv] : 0.0f;
+    }
+    const float xn = theta * xnr;
     float lv[KL], lu[KL];
     int32_t li[KL];
 #pragma unroll
     for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
-    const float *c = cr + srow * 2 * n, *r = c + n, *e = noise + row * n;
-    const float xn = theta * xnorm[row / kdiv];
-    float rest_hi = -CUDART_INF_F;
-    // approximate noisy logit v of column j and a bound u on its distance from the fma chain's value
-    auto eval = [&](int32_t j, float cj, float rj, float ej, float &v, float &u) {
-        // the hardware exponential and logarithm are enough for screening: their error is an absolute 7.2e-7 at most
-        // on sigma (2.4e-7 from __expf on [-inf, 0], 1.2e-7 from rounding 1 + y, 2^-21.41 from __logf on [1, 2]) and
-        // goes into the uncertainty below with a margin (2e-6 |noise|)
-        const float sigma = fmaxf(rj, 0.0f) + __logf(1.0f + __expf(-fabsf(rj)));
-        v = fmaf(ej, sigma, cj);
-        // |H~_j - H_j|: projection errors through c and through softplus(r) (slope <= 1) times |noise|, plus the
-        // error of softplus (here approximate, there double rounded once) and of the final fma on both sides
-        u = xn * fmaf(fabsf(ej), wnorm[n + j], wnorm[j]) +
-            1.1920929e-7f * (8.0f * fabsf(v) + 16.0f * fabsf(ej) * sigma) + 2.0e-6f * fabsf(ej);
-    };
+    float rest_hi = -CUDART_INF_F;  // largest possible chain value of anything that is not in the list
     auto consider = [&](int32_t j, float cj, float rj, float ej) {
-        clean[row * n + j] = cj;
-        raw[row * n + j] = rj;
         float v, u;
-        eval(j, cj, rj, ej, v, u);
-        int32_t id = j;
-        bool shifting = false;
+        screen_eval(cj, rj, ej, xn, wn[j], wn[n + j], v, u);
+        if (v > lv[KL - 1]) {
+            // enters the list behind every entry that is at least as large (those have lower indices), the last
+            // entry falls off
+            rest_hi = fmaxf(rest_hi, lv[KL - 1] + lu[KL - 1]);
 #pragma unroll
-        for (int s = 0; s < KL; ++s) {
-            if (shifting || v > lv[s]) {
-                float tv = lv[s], tu = lu[s]; int32_t ti = li[s];
-                lv[s] = v; li[s] = id; lu[s] = u; v = tv; id = ti; u = tu;
-                shifting = true;
+            for (int s = KL - 1; s >= 1; --s) {
+                const bool stays = lv[s] >= v && s != KL - 1, here = lv[s - 1] >= v;
+                if (!stays) {
+                    lv[s] = here ? v : lv[s - 1];
+                    lu[s] = here ? u : lu[s - 1];
+                    li[s] = here ? j : li[s - 1];
+                }
             }
+            if (!(lv[0] >= v)) { lv[0] = v; lu[0] = u; li[0] = j; }
+        } else {
+            rest_hi = fmaxf(rest_hi, v + u);
         }
-        if (id != INT32_MAX) rest_hi = fmaxf(rest_hi, v + u);  // fell off (or never entered) the list
     };
-    if (NV > 0) {
-        float cv[NV > 0 ? NV : 1], rv[NV > 0 ? NV : 1], ev[NV > 0 ? NV : 1];
+    // loads: instruction i covers the rows 8 i + lane / 4 of the warp, four columns per lane
+    const int lr = lane >> 2, lq = (lane & 3) * 4;
+    float *tc = tile[wp][0], *tr = tile[wp][1], *te = tile[wp][2];
+    for (int32_t j0 = 0; j0 < n; j0 += SCREEN_CH) {
+        float4 c4[4], r4[4], e4[4];
+        int32_t orow[4];  // output rows fit 31 bits (they go into the int32 row lists)
 #pragma unroll
-        for (int q = 0; q < NV; ++q) {
-            const int32_t j = lane + 32 * q;
-            const bool in = j < n;
-            cv[q] = in ? c[j] : 0.0f; rv[q] = in ? r[j] : 0.0f; ev[q] = in ? e[j] : 0.0f;
+        for (int i = 0; i < 4; ++i) {
+            const int64_t sr = s0 + 8 * i + lr;
+            orow[i] = __shfl_sync(0xffffffffu, (int32_t)row, 8 * i + lr);
+            c4[i] = r4[i] = e4[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (sr < T) {
+                c4[i] = load4<V16>(cr + sr * 2 * n + j0 + lq);
+                r4[i] = load4<V16>(cr + sr * 2 * n + n + j0 + lq);
+                e4[i] = load4<V16>(noise + (int64_t)orow[i] * n + j0 + lq);
+            }
         }
 #pragma unroll
-        for (int q = 0; q < NV; ++q)
-            if (lane + 32 * q < n) consider(lane + 32 * q, cv[q], rv[q], ev[q]);
-    } else {
-        for (int32_t j = lane; j < n; j += 32) consider(j, c[j], r[j], e[j]);
+        for (int i = 0; i < 4; ++i) {
+            const int at = (8 * i + lr) * SCREEN_PITCH + lq;
+            *reinterpret_cast<float4 *>(tc + at) = c4[i];
+            *reinterpret_cast<float4 *>(tr + at) = r4[i];
+            *reinterpret_cast<float4 *>(te + at) = e4[i];
+            if (s0 + 8 * i + lr < T) {
+                store4<V16>(clean + (int64_t)orow[i] * n + j0 + lq, c4[i]);
+                store4<V16>(raw + (int64_t)orow[i] * n + j0 + lq, r4[i]);
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < SCREEN_CH / 4; ++q) {
+            const float4 cq = *reinterpret_cast<const float4 *>(tc + lane * SCREEN_PITCH + 4 * q);
+            const float4 rq = *reinterpret_cast<const float4 *>(tr + lane * SCREEN_PITCH + 4 * q);
+            const float4 eq = *reinterpret_cast<const float4 *>(te + lane * SCREEN_PITCH + 4 * q);
+            const int32_t j = j0 + 4 * q;
+            consider(j, cq.x, rq.x, eq.x);
+            consider(j + 1, cq.y, rq.y, eq.y);
+            consider(j + 2, cq.z, rq.z, eq.z);
+            consider(j + 3, cq.w, rq.w, eq.w);
+        }
+        __syncwarp();
     }
+    // the first `rounds` entries are the ranked ones, whatever else is in the list is "rest" as well
     const int rounds = min(k + 2, n);
-    float hvv[KL], huu[KL];
-    float myv = -CUDART_INF_F;
-    int32_t myi = -1;
-    float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
-    int32_t i_k = -1, i_k1 = -1;
-#pragma unroll
-    for (int s = 0; s < KL; ++s) {
-        hvv[s] = -CUDART_INF_F; huu[s] = 0.0f;
-        if (s < rounds) {
-            float hv = lv[0], hu = lu[0];
-            int32_t hi = li[0];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                float ov = __shfl_xor_sync(0xffffffffu, hv, off), ou = __shfl_xor_sync(0xffffffffu, hu, off);
-                int32_t oi = __shfl_xor_sync(0xffffffffu, hi, off);
-                if (ov > hv || (ov == hv && oi < hi)) { hv = ov; hi = oi; hu = ou; }
-            }
-            if (li[0] == hi) {
-#pragma unroll
-                for (int q = 0; q < KL - 1; ++q) { lv[q] = lv[q + 1]; li[q] = li[q + 1]; lu[q] = lu[q + 1]; }
-                lv[KL - 1] = -CUDART_INF_F;
-                li[KL - 1] = INT32_MAX;
-            }
-            hvv[s] = hv; huu[s] = hu;
-            if (s < k && lane == s) { myv = hv; myi = hi; }
-            if (s == k - 1) { v_k = hv; i_k = hi; }
-            if (s == k && k < n) { v_k1 = hv; i_k1 = hi; }
-        }
-    }
-    // whatever is still in the lists is "rest" as well
 #pragma unroll
     for (int s = 0; s < KL; ++s)
-        if (li[s] != INT32_MAX) rest_hi = fmaxf(rest_hi, lv[s] + lu[s]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) rest_hi = fmaxf(rest_hi, __shfl_xor_sync(0xffffffffu, rest_hi, off));
-    // ranks 1..k+1 are certain iff each one's lowest possible value beats the highest possible value of
-    // everything ranked after it
+        if (s >= rounds && li[s] != INT32_MAX) rest_hi = fmaxf(rest_hi, lv[s] + lu[s]);
+    // ranks 1..k+1 are certain iff each one's lowest possible value beats the highest possible value of everything
+    // ranked after it
     bool safe = true;
     float suffix = rest_hi;
 #pragma unroll
     for (int s = KL - 1; s >= 0; --s) {
         if (s < rounds) {
-            if (s <= k && !(hvv[s] - huu[s] > suffix)) safe = false;
-            suffix = fmaxf(suffix, hvv[s] + huu[s]);
+            if (s <= k && !(lv[s] - lu[s] > suffix)) safe = false;
+            suffix = fmaxf(suffix, lv[s] + lu[s]);
         }
     }
-    if (!safe) {
-        // Not provably the chain's routing. Only the columns that can still reach rank k+1 matter: those whose
-        // highest possible value is at least `low`, a lower bound of the (k+1)-th largest chain value (the (k+1)-th
-        // largest lower end among the extracted columns). They get their two fma chains redone (chain_list), the
-        // selection is then repeated on the patched row. Rows with too many candidates (ties) take the full chain.
-        float low = -CUDART_INF_F;
-        if (k < rounds) {
+    // Not provably the chain's routing: only the columns that can still reach rank k+1 matter, those whose highest
+    // possible value is at least `low`, a lower bound of the (k+1)-th largest chain value (the (k+1)-th largest lower end
+    // among the ranked columns).
+    float low = -CUDART_INF_F;
+    if (!safe && k < rounds) {
 #pragma unroll
-            for (int s = 0; s < KL; ++s) {
-                if (s < rounds) {
-                    const float ls = hvv[s] - huu[s];
-                    int above = 0;
+        for (int s = 0; s < KL; ++s) {
+            if (s < rounds) {
+                const float ls = lv[s] - lu[s];
+                int above = 0;
 #pragma unroll
-                    for (int s2 = 0; s2 < KL; ++s2)
-                        if (s2 < rounds && s2 != s) {
-                            const float l2 = hvv[s2] - huu[s2];
-                            above += (l2 > ls || (l2 == ls && s2 < s)) ? 1 : 0;
-                        }
-                    if (above == k) low = ls;
-                }
+                for (int s2 = 0; s2 < KL; ++s2)
+                    if (s2 < rounds && s2 != s) {
+                        const float l2 = lv[s2] - lu[s2];
+                        above += (l2 > ls || (l2 == ls && s2 < s)) ? 1 : 0;
+                    }
+                if (above == k) low = ls;
             }
         }
-        // (the row is re-read and re-evaluated here: keeping every column's value in registers through the
-        // selection above would cost the certified rows, the common case, their occupancy)
-        int total = 0;
-        uint32_t mine = 0;  // NV > 0: bit q = this lane's column lane + 32 q is a candidate
-        if (NV > 0) {
-#pragma unroll
-            for (int q = 0; q < NV; ++q) {
-                const int32_t j = lane + 32 * q;
-                float v = -CUDART_INF_F, u = 0.0f;
-                if (j < n) eval(j, c[j], r[j], e[j], v, u);
-                const bool cand = j < n && v + u >= low;
-                if (cand) mine |= 1u << q;
-                total += __popc(__ballot_sync(0xffffffffu, cand));
-            }
-        } else {
-            for (int32_t j0 = 0; j0 < n; j0 += 32) {
-                const int32_t j = j0 + lane;
-                float v = -CUDART_INF_F, u = 0.0f;
-                if (j < n) eval(j, c[j], r[j], e[j], v, u);
-                total += __popc(__ballot_sync(0xffffffffu, j < n && v + u >= low));
-            }
-        }
+    }
+    const bool listed = live && !safe;
+    const uint32_t lb = __ballot_sync(0xffffffffu, listed);
+    if (lb) {
         int32_t base = 0;
-        const bool few = total <= SCREEN_MAX_CAND;
+        if (lane == 0) base = atomicAdd(unsafe_count, __popc(lb));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (listed) {
+            const int32_t at = base + __popc(lb & ((1u << lane) - 1u));
+            unsafe_list[at] = (int32_t)row;
+            unsafe_low[at] = low;
+        }
+    }
+    if (!live || !safe) return;
+    float ex[KL], den = 0.0f;
+#pragma unroll
+    for (int s = 0; s < KL; ++s) {
+        ex[s] = 0.0f;
+        if (s < k) { ex[s] = expf(lv[s] - lv[0]); den += ex[s]; }
+    }
+#pragma unroll
+    for (int s = 0; s < KL; ++s)
+        if (s < k) {
+            idx[row * k + s] = li[s];
+            gates[row * k + s] = ex[s] / den;
+        }
+    float v_k = -CUDART_INF_F, v_k1 = -CUDART_INF_F;
+    int32_t i_k = -1, i_k1 = -1;
+#pragma unroll
+    for (int s = 0; s < KL; ++s) {
+        if (s == k - 1) { v_k = lv[s]; i_k = li[s]; }
+        if (s == k && k < n) { v_k1 = lv[s]; i_k1 = li[s]; }
+    }
+    kth_vals[row * 2 + 0] = v_k;
+    kth_vals[row * 2 + 1] = v_k1;
+    kth_idx[row * 2 + 0] = i_k;
+    kth_idx[row * 2 + 1] = i_k1;
+}
+
+// The rows the screen listed, one warp per row: the columns whose highest possible value reaches the row's `low` get
+// their two fma chains redone (chain_list), the selection is then repeated on the patched row. Rows with more than
+// SCREEN_MAX_CAND candidates (ties) take the full chain (full_list), or, where there is no whole-row fallback
+// (full_list == nullptr), the chains of all their columns.
+__global__ void __launch_bounds__(256) gate_candidates_kernel(const float *__restrict__ clean, const float *__restrict__ raw,
+                                                              const float *__restrict__ noise,
+                                                              const float *__restrict__ xnorm,
+                                                              const float *__restrict__ wnorm, float theta, int32_t n,
+                                                              const int32_t *__restrict__ unsafe_list,
+                                                              const float *__restrict__ unsafe_low,
+                                                              int32_t *__restrict__ unsafe_count,
+                                                              int2 *__restrict__ chain_list,
+                                                              int32_t *__restrict__ full_list, int32_t kdiv,
+                                                              const int32_t *__restrict__ group_of, int32_t k,
+                                                              int2 *__restrict__ unsafe_span) {
+    // unsafe_span[i] = {first entry of the row's chains in chain_list, number of candidate columns}, or {0, -1}
+    // where the repeated selection has to look at every column
+    const int lane = threadIdx.x & 31;
+    const int32_t total_rows = *unsafe_count;  // complete: the screen ran before this kernel
+    const int32_t nwarps = gridDim.x * (blockDim.x >> 5);
+    for (int32_t it = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < total_rows; it += nwarps) {
+        const int64_t row = unsafe_list[it];
+        const float low = unsafe_low[it];
+        const int32_t group = group_of ? group_of[row] : 0;
+        const float *wn = wnorm + (int64_t)group * 2 * n;
+        const float xn = theta * xnorm[row / kdiv];
+        const float *c = clean + row * n, *r = raw + row * n, *e = noise + row * n;
+        auto candidate = [&](int32_t j) {
+            if (j >= n) return false;
+            float v, u;
+            screen_eval(c[j], r[j], e[j], xn, wn[j], wn[n + j], v, u);
+            return v + u >= low;
+        };
+        int total = 0;
+        for (int32_t j0 = 0; j0 < n; j0 += 32) total += __popc(__ballot_sync(0xffffffffu, candidate(j0 + lane)));
+        // (fewer than k + 1 candidates happens only with NaN logits, which are nobody's candidate)
+        const bool few = total <= SCREEN_MAX_CAND && total >= min(k + 1, n);
         const int32_t wbase = group * 2 * n;  // this group's rows of the transposed weights
+        int32_t base = 0;
         if (lane == 0) {
-            unsafe_list[atomicAdd(unsafe_count, 1)] = (int32_t)row;
             if (few) base = atomicAdd(unsafe_count + 1, 2 * total);
             else if (full_list) full_list[atomicAdd(unsafe_count + 2, 1)] = (int32_t)row;
-            else base = atomicAdd(unsafe_count + 1, 2 * n);  // no whole-row fallback: every column gets its chains
+            else base = atomicAdd(unsafe_count + 1, 2 * n);
         }
         base = __shfl_sync(0xffffffffu, base, 0);
+        if (lane == 0) unsafe_span[it] = few ? make_int2(base, total) : make_int2(0, -1);
         if (!few) {
             if (!full_list)
                 for (int32_t j = lane; j < n; j += 32) {
                     chain_list[base + 2 * j] = make_int2((int32_t)row, wbase + j);
                     chain_list[base + 2 * j + 1] = make_int2((int32_t)row, wbase + n + j);
                 }
-            return;
+            continue;
         }
         int pos = 0;
-        auto emit = [&](int32_t j, bool cand) {
+        for (int32_t j0 = 0; j0 < n; j0 += 32) {
+            const int32_t j = j0 + lane;
+            const bool cand = candidate(j);
             const uint32_t b = __ballot_sync(0xffffffffu, cand);
             if (cand) {
                 const int at = base + 2 * (pos + __popc(b & ((1u << lane) - 1u)));
@@ -547,33 +664,7 @@ __global__ void __launch_bounds__(256) gate_screen_kernel(const float *__restric
                 chain_list[at + 1] = make_int2((int32_t)row, wbase + n + j);
             }
             pos += __popc(b);
-        };
-        if (NV > 0) {
-#pragma unroll
-            for (int q = 0; q < NV; ++q) emit(lane + 32 * q, (mine >> q) & 1u);
-        } else {
-            for (int32_t j0 = 0; j0 < n; j0 += 32) {
-                const int32_t j = j0 + lane;
-                float v = -CUDART_INF_F, u = 0.0f;
-                if (j < n) eval(j, c[j], r[j], e[j], v, u);
-                emit(j, j < n && v + u >= low);
-            }
         }
-        return;
-    }
-    const float m = __shfl_sync(0xffffffffu, myv, 0);
-    const float ex = lane < k ? expf(myv - m) : 0.0f;
-    float den = 0.0f;
-    for (int s = 0; s < k; ++s) den += __shfl_sync(0xffffffffu, ex, s);
-    if (lane < k) {
-        idx[row * k + lane] = myi;
-        gates[row * k + lane] = ex / den;
-    }
-    if (lane == 0) {
-        kth_vals[row * 2 + 0] = v_k;
-        kth_vals[row * 2 + 1] = v_k1;
-        kth_idx[row * 2 + 0] = i_k;
-        kth_idx[row * 2 + 1] = i_k1;
     }
 }
 
@@ -715,35 +806,44 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
     return MOE_OK;
 }
 
-int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
+int32_t launch_gate_screen(const float *cr, const float *noise, float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
-                           float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, int32_t *unsafe_count,
-                           void *chain_list, int32_t *full_list, cudaStream_t st, const int32_t *perm, int32_t kdiv,
-                           const int32_t *group_of) {
+                           float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, float *unsafe_low,
+                           int32_t *unsafe_count, void *chain_list, int32_t *full_list, cudaStream_t st,
+                           const int32_t *perm, int32_t kdiv, const int32_t *group_of, void *unsafe_span,
+                           const void *x) {
+    // x != nullptr (flat use, bf16 rows of d values): the row norms are formed here and written to xnorm
     // worst-case rounding of the fma chain, plus two truncations of an fp32 accumulator per MMA step of the
     // three-term tensor-core product (3d/16 steps and the additions inside a step), plus the split residual
     const double u = ldexp(1.0, -24);
     const double chain = d * u / (1.0 - d * u);
     const double tc = 2.0 * (3.0 * d / 16.0 + 8.0) * ldexp(1.0, -23) + ldexp(1.0, -22);
     const float theta = (float)((chain + tc) * 1.01);
-    const unsigned grid = (unsigned)cdiv(T, 8);
-#define MOE_SCREEN_KL(NV, KL)                                                                                            \
-    gate_screen_kernel<NV, KL><<<grid, 256, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n, k, idx, gates, clean, raw,  \
-                                                     kth_vals, kth_idx, unsafe_list, unsafe_count, (int2 *)chain_list, \
-                                                     full_list, perm, kdiv, group_of)
-#define MOE_SCREEN(NV)                                \
-    do {                                              \
-        if (k <= 2) MOE_SCREEN_KL(NV, 4);             \
-        else if (k <= 4) MOE_SCREEN_KL(NV, 6);        \
-        else MOE_SCREEN_KL(NV, MOE_MAX_K + 2);        \
+    if (T == 0) return MOE_OK;
+    if (n % SCREEN_CH != 0) return MOE_ERR_INVALID_ARG;  // the screened path has 2n a multiple of 64
+    const unsigned grid = (unsigned)cdiv(T, 128);
+    const bool v16 = (((uintptr_t)noise | (uintptr_t)clean | (uintptr_t)raw | (uintptr_t)cr) & 15) == 0;
+#define MOE_SCREEN_KL(KL)                                                                                              \
+    do {                                                                                                               \
+        if (v16)                                                                                                       \
+            gate_screen_rows_kernel<KL, true><<<grid, 128, 0, st>>>(cr, noise, (const bf16 *)x, d, xnorm, wnorm, theta, T, n, \
+                                                                    k, idx, gates, clean, raw, kth_vals, kth_idx,      \
+                                                                    unsafe_list, unsafe_low, unsafe_count, perm, kdiv, \
+                                                                    group_of);                                         \
+        else                                                                                                           \
+            gate_screen_rows_kernel<KL, false><<<grid, 128, 0, st>>>(cr, noise, (const bf16 *)x, d, xnorm, wnorm, theta, T, \
+                                                                     n, k, idx, gates, clean, raw, kth_vals, kth_idx,  \
+                                                                     unsafe_list, unsafe_low, unsafe_count, perm,      \
+                                                                     kdiv, group_of);                                  \
     } while (0)
-    if (n <= 32) MOE_SCREEN(1);
-    else if (n <= 64) MOE_SCREEN(2);
-    else if (n <= 128) MOE_SCREEN(4);
-    else if (n <= 256) MOE_SCREEN(8);
-    else MOE_SCREEN(0);
-#undef MOE_SCREEN
+    if (k <= 2) MOE_SCREEN_KL(4);
+    else if (k <= 4) MOE_SCREEN_KL(6);
+    else MOE_SCREEN_KL(MOE_MAX_K + 2);
 #undef MOE_SCREEN_KL
+    MOE_LAUNCHED();
+    gate_candidates_kernel<<<148 * 4, 256, 0, st>>>(clean, raw, noise, xnorm, wnorm, theta, n, unsafe_list, unsafe_low,
+                                                    unsafe_count, (int2 *)chain_list, full_list, kdiv, group_of, k,
+                                                    (int2 *)unsafe_span);
     MOE_LAUNCHED();
     return MOE_OK;
 }

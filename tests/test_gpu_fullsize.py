@@ -179,3 +179,35 @@ def test_full_size_fused(name):
     # sum_j dclean_j ~ 0: that column of dX_gate is a cancelling sum, and fp32 accumulation (any order)
     # leaves ~1e-5 of the result there; the mean error stays at the 1e-7 level.
     assert_close(host(dXg_d), want_dXg, dict(max=5e-5, mean=1e-6), "dX_gate (full)")
+
+
+REPEATS = {"c3": 40, "c4": 20, "c5": 60}
+
+
+@pytest.mark.parametrize("name", ["c3", "c4", "c5"])
+def test_full_size_repeated_steps_agree_bit_for_bit(name):
+    """Tiles are handed to the SM pairs at run time, so which pair computes a tile changes from run to run; the
+    result must not. Every output of the fused step and the saved context is compared byte for byte with the first
+    run. The forward between two backward passes overwrites the workspace, so a piece of a backward tensor that a
+    run fails to write shows up as different bytes instead of hiding behind the previous run's identical values."""
+    w = synth.CONFIGS[name]
+    cfg, S, D, _ = bench.build_device_state(w, keep_host_experts=False)
+    outs = ("y", "losses", "importance", "load", "counts", "dX", "dWg", "dWnoise", "dW1", "db1", "dW2", "db2")
+
+    def step():
+        B.moe_forward(cfg, D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"], D["y"],
+                      D["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+        B.moe_backward(cfg, D["dY"], D["x"], D["Wg"], D["Wnoise"], D["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
+                       D["ctx"], D["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"], D["db2"], D["ws"])
+        torch.cuda.synchronize()
+        assert B.moe_check_status(D["ws"]) == 0
+
+    step()
+    first = {k: D[k].clone() for k in outs}
+    first_ctx = D["ctx"].clone()
+    for it in range(REPEATS[name]):
+        step()
+        differing = [k for k in outs if not torch.equal(first[k].view(torch.uint8), D[k].view(torch.uint8))]
+        if not torch.equal(first_ctx.view(torch.uint8), D["ctx"].view(torch.uint8)):
+            differing.append("ctx")
+        assert not differing, f"run {it + 1} differs from the first in {differing}"
