@@ -337,11 +337,11 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
     auto first_gate = [&](int32_t n1, int32_t k1, int32_t *idx_out, float *gates_out) -> int32_t {
         if (w.screen) {
             MOE_TRY(launch_gate_screen_prepare(x, D.act, D.T, (int32_t)D.d, n1, Wg, Wnoise, w.wsplit, w.wnorm, w.xnorm,
-                                               w.unsafe_count, w.wt, st, 1, false));  // the screen forms the row norms
+                                               w.unsafe_count, w.wt, st));
             MOE_TRY(launch_tc_gate_fwd(x, D.T, (int32_t)D.d, n1, w.wsplit, w.cr, status_word(ws_base), st));
             MOE_TRY(launch_gate_screen(w.cr, noise, w.xnorm, w.wnorm, (int32_t)D.d, D.T, n1, k1, idx_out, gates_out,
                                        clean, raw_noise, kth_vals, kth_idx, w.unsafe_list, w.unsafe_low, w.unsafe_count,
-                                       w.chain_list, w.full_list, st, nullptr, 1, nullptr, w.unsafe_span, x));
+                                       w.chain_list, w.full_list, st, nullptr, 1, nullptr, w.unsafe_span));
             // exact chains for the few columns that decide an uncertain row; whole rows only where there are many
             MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, n1, w.wt, w.chain_list, w.unsafe_count + 1, clean, raw_noise,
                                        st));
@@ -374,7 +374,7 @@ int32_t do_gate(const moe_config *c, const Dims &D, const void *x, const float *
         MOE_TRY(launch_gate_screen(w.cr_s, noise + lp, w.xnorm, w.wnorm_s, (int32_t)D.d, P1, (int32_t)D.b, (int32_t)D.k2,
                                    w.idx_s, g_s, clean + lp, raw_noise + lp, kth_vals + 2 * D.T, kth_idx + 2 * D.T,
                                    w.unsafe_list_s, w.unsafe_low_s, w.unsafe_count_s, w.chain_list_s, nullptr, st, w.perm_p,
-                                   (int32_t)D.k1, w.idx_p, w.unsafe_span_s, nullptr));
+                                   (int32_t)D.k1, w.idx_p, w.unsafe_span_s));
         MOE_TRY(launch_gate_chains(x, D.act, (int32_t)D.d, (int32_t)D.b, w.wt_s, w.chain_list_s, w.unsafe_count_s + 1,
                                    clean + lp, raw_noise + lp, st, (int32_t)D.k1));
         MOE_TRY(launch_gate_select(clean + lp, raw_noise + lp, noise + lp, P1, (int32_t)D.b, (int32_t)D.k2, w.idx_s, g_s,

@@ -350,6 +350,7 @@ __global__ void __launch_bounds__(256) gate_col_norms_kernel(const float *__rest
     if (lane == 0) wnorm[j] = (float)(sqrt(s) * (1.0 + 1e-6));
 }
 
+// |x_t|_2 (slightly rounded up), one warp per row; bf16 rows are read 16 bytes per lane, four loads in flight
 template <typename XT>
 __global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x, int64_t T, int32_t d,
                                                         float *__restrict__ xnorm) {
@@ -357,6 +358,27 @@ __global__ void __launch_bounds__(256) row_norms_kernel(const XT *__restrict__ x
     const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= T) return;
     float s = 0.0f;
+    if constexpr (sizeof(XT) == 2) {
+        if (d % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+            const uint4 *row = reinterpret_cast<const uint4 *>(x + t * d);
+            const int32_t pieces = d / 8;
+            for (int32_t q0 = lane; q0 < pieces; q0 += 128) {
+                uint4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) v[i] = q0 + 32 * i < pieces ? row[q0 + 32 * i] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const bf16 *h = reinterpret_cast<const bf16 *>(&v[i]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { const float f = __bfloat162float(h[e]); s = fmaf(f, f, s); }
+                }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+            if (lane == 0) xnorm[t] = sqrtf(s) * (1.0f + 1e-5f);
+            return;
+        }
+    }
     for (int32_t q = lane; q < d; q += 32) { const float v = to_f32(x[t * d + q]); s = fmaf(v, v, s); }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
@@ -403,8 +425,7 @@ __device__ __forceinline__ void store4(float *p, float4 v) {
 }
 template <int KL, bool V16>
 __global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__restrict__ cr, const float *__restrict__ noise,
-                                                               const bf16 *__restrict__ x, int32_t d,
-                                                               float *__restrict__ xnorm,
+                                                               const float *__restrict__ xnorm,
                                                                const float *__restrict__ wnorm, float theta, int64_t T,
                                                                int32_t n, int32_t k, int32_t *__restrict__ idx,
                                                                float *__restrict__ gates, float *__restrict__ clean,
@@ -423,40 +444,7 @@ __global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__re
     const bool live = srow < T;
     const int64_t row = live ? (perm ? (int64_t)perm[srow] : srow) : 0;
     const float *wn = wnorm + (int64_t)(group_of && live ? group_of[row] : 0) * 2 * n;
-    float xnr;
-    if (x) {
-        // |x_t|_2 of the warp's 32 rows, here rather than in a pass of its own (flat use: row = srow; d a multiple of
-        // 256): the warp reads a row with 16-byte loads, four rows in flight, lane i keeps the norm of row i and
-        // publishes it for the later kernels
-        xnr = 0.0f;
-        for (int i0 = 0; i0 < 32; i0 += 4) {
-            float part[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-            for (int32_t q = lane * 8; q < d; q += 256) {
-                uint4 raw4[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int64_t sr = min(s0 + i0 + i, T - 1);
-                    raw4[i] = *reinterpret_cast<const uint4 *>(x + sr * d + q);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const bf16 *hx = reinterpret_cast<const bf16 *>(&raw4[i]);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) { const float v = __bfloat162float(hx[e]); part[i] = fmaf(v, v, part[i]); }
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) part[i] += __shfl_xor_sync(0xffffffffu, part[i], off);
-                if (lane == i0 + i) xnr = sqrtf(part[i]) * (1.0f + 1e-5f);
-            }
-        }
-        if (live) xnorm[row] = xnr;
-    } else {
-        xnr = live ? xnorm[row / kdiv] : 0.0f;
-    }
-    const float xn = theta * xnr;
+    const float xn = live ? theta * xnorm[row / kdiv] : 0.0f;
     float lv[KL], lu[KL];
     int32_t li[KL];
 #pragma unroll
@@ -806,13 +794,11 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
     return MOE_OK;
 }
 
-int32_t launch_gate_screen(const float *cr, const float *noise, float *xnorm, const float *wnorm, int32_t d,
+int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, float *unsafe_low,
                            int32_t *unsafe_count, void *chain_list, int32_t *full_list, cudaStream_t st,
-                           const int32_t *perm, int32_t kdiv, const int32_t *group_of, void *unsafe_span,
-                           const void *x) {
-    // x != nullptr (flat use, bf16 rows of d values): the row norms are formed here and written to xnorm
+                           const int32_t *perm, int32_t kdiv, const int32_t *group_of, void *unsafe_span) {
     // worst-case rounding of the fma chain, plus two truncations of an fp32 accumulator per MMA step of the
     // three-term tensor-core product (3d/16 steps and the additions inside a step), plus the split residual
     const double u = ldexp(1.0, -24);
@@ -826,12 +812,12 @@ int32_t launch_gate_screen(const float *cr, const float *noise, float *xnorm, co
 #define MOE_SCREEN_KL(KL)                                                                                              \
     do {                                                                                                               \
         if (v16)                                                                                                       \
-            gate_screen_rows_kernel<KL, true><<<grid, 128, 0, st>>>(cr, noise, (const bf16 *)x, d, xnorm, wnorm, theta, T, n, \
+            gate_screen_rows_kernel<KL, true><<<grid, 128, 0, st>>>(cr, noise, xnorm, wnorm, theta, T, n,                   \
                                                                     k, idx, gates, clean, raw, kth_vals, kth_idx,      \
                                                                     unsafe_list, unsafe_low, unsafe_count, perm, kdiv, \
                                                                     group_of);                                         \
         else                                                                                                           \
-            gate_screen_rows_kernel<KL, false><<<grid, 128, 0, st>>>(cr, noise, (const bf16 *)x, d, xnorm, wnorm, theta, T, \
+            gate_screen_rows_kernel<KL, false><<<grid, 128, 0, st>>>(cr, noise, xnorm, wnorm, theta, T,                     \
                                                                      n, k, idx, gates, clean, raw, kth_vals, kth_idx,  \
                                                                      unsafe_list, unsafe_low, unsafe_count, perm,      \
                                                                      kdiv, group_of);                                  \

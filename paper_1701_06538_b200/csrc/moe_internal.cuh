@@ -103,12 +103,11 @@ int32_t launch_gate_screen_prepare(const void *x, int32_t act, int64_t T, int32_
                                    const float *Wn, void *wsplit, float *wnorm, float *xnorm,
                                    int32_t *unsafe_count, float *wt /* [2n, d]: columns as rows */, cudaStream_t st,
                                    int32_t groups = 1, bool with_xnorm = true);
-int32_t launch_gate_screen(const float *cr, const float *noise, float *xnorm, const float *wnorm, int32_t d,
+int32_t launch_gate_screen(const float *cr, const float *noise, const float *xnorm, const float *wnorm, int32_t d,
                            int64_t T, int32_t n, int32_t k, int32_t *idx, float *gates, float *clean, float *raw,
                            float *kth_vals, int32_t *kth_idx, int32_t *unsafe_list, float *unsafe_low,
                            int32_t *unsafe_count, void *chain_list, int32_t *full_list, cudaStream_t st,
-                           const int32_t *perm, int32_t kdiv, const int32_t *group_of, void *unsafe_span,
-                           const void *x /* bf16 rows: form xnorm here; nullptr: read it */);
+                           const int32_t *perm, int32_t kdiv, const int32_t *group_of, void *unsafe_span);
 // Rows the screen cannot certify: unsafe_list / unsafe_count[0] = rows whose selection is repeated (unsafe_low: the
 // bound that picks their candidate columns); chain_list
 // (int2 {row, column code}, unsafe_count[1] entries, at most 2 * SCREEN_MAX_CAND per row) = single fma chains to
