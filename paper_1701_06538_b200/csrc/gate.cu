@@ -450,9 +450,7 @@ __global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__re
 #pragma unroll
     for (int s = 0; s < KL; ++s) { lv[s] = -CUDART_INF_F; li[s] = INT32_MAX; lu[s] = 0.0f; }
     float rest_hi = -CUDART_INF_F;  // largest possible chain value of anything that is not in the list
-    auto consider = [&](int32_t j, float cj, float rj, float ej) {
-        float v, u;
-        screen_eval(cj, rj, ej, xn, wn[j], wn[n + j], v, u);
+    auto insert = [&](int32_t j, float v, float u) {
         if (v > lv[KL - 1]) {
             // enters the list behind every entry that is at least as large (those have lower indices), the last
             // entry falls off
@@ -470,6 +468,20 @@ __global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__re
         } else {
             rest_hi = fmaxf(rest_hi, v + u);
         }
+    };
+    // four columns at a time: their values and bounds first (independent of each other, so the exponentials and
+    // logarithms overlap), then the four list updates, which depend on one another
+    auto consider4 = [&](int32_t j, const float4 &c4, const float4 &r4, const float4 &e4) {
+        const float4 wg4 = *reinterpret_cast<const float4 *>(wn + j), wn4 = *reinterpret_cast<const float4 *>(wn + n + j);
+        float v0, v1, v2, v3, u0, u1, u2, u3;
+        screen_eval(c4.x, r4.x, e4.x, xn, wg4.x, wn4.x, v0, u0);
+        screen_eval(c4.y, r4.y, e4.y, xn, wg4.y, wn4.y, v1, u1);
+        screen_eval(c4.z, r4.z, e4.z, xn, wg4.z, wn4.z, v2, u2);
+        screen_eval(c4.w, r4.w, e4.w, xn, wg4.w, wn4.w, v3, u3);
+        insert(j, v0, u0);
+        insert(j + 1, v1, u1);
+        insert(j + 2, v2, u2);
+        insert(j + 3, v3, u3);
     };
     // loads: instruction i covers the rows 8 i + lane / 4 of the warp, four columns per lane
     const int lr = lane >> 2, lq = (lane & 3) * 4;
@@ -505,11 +517,7 @@ __global__ void __launch_bounds__(128) gate_screen_rows_kernel(const float *__re
             const float4 cq = *reinterpret_cast<const float4 *>(tc + lane * SCREEN_PITCH + 4 * q);
             const float4 rq = *reinterpret_cast<const float4 *>(tr + lane * SCREEN_PITCH + 4 * q);
             const float4 eq = *reinterpret_cast<const float4 *>(te + lane * SCREEN_PITCH + 4 * q);
-            const int32_t j = j0 + 4 * q;
-            consider(j, cq.x, rq.x, eq.x);
-            consider(j + 1, cq.y, rq.y, eq.y);
-            consider(j + 2, cq.z, rq.z, eq.z);
-            consider(j + 3, cq.w, rq.w, eq.w);
+            consider4(j0 + 4 * q, cq, rq, eq);
         }
         __syncwarp();
     }
