@@ -375,9 +375,10 @@ __global__ void __launch_bounds__(256) bal_dispatch_bwd_kernel(const XT *__restr
 }  // namespace
 
 int64_t balanced_ws_bytes(int64_t T, int32_t n) {
-    // logits' twin of the projection, p^T, per-token counts, loss partials
-    const int64_t a = (T * n * 4 + 255) & ~255ll, b = a, c = (T * 4 + 255) & ~255ll, e = (cdiv(T, 8) * 8 + 255) & ~255ll;
-    return a + b + c + e + 256;
+    // p^T, per-token counts, loss partials, tile sums of the scan over the tokens
+    const int64_t a = (T * n * 4 + 255) & ~255ll, c = (T * 4 + 255) & ~255ll, e = (cdiv(T, 8) * 8 + 255) & ~255ll;
+    const int64_t f = (cdiv(T + 1, 4096) * 4 + 255) & ~255ll;
+    return a + c + e + f + 256;
 }
 
 int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, int32_t k, const float *Wg,
@@ -387,10 +388,10 @@ int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, i
     const int64_t R = T * k;
     const int32_t m = (int32_t)(R / n), words = (n + 31) / 32;
     Carver cv(ws);
-    float *twin = cv.take<float>(T * n);
     float *pT = cv.take<float>(T * n);
     int32_t *cnt = cv.take<int32_t>(T);
     double *loss_part = cv.take<double>(cdiv(T, 8));
+    int32_t *tile_sums = cv.take<int32_t>(cdiv(T + 1, 4096));
     MOE_CUDA(cudaMemsetAsync(mask_bits, 0, sizeof(uint32_t) * T * words, st));
     MOE_CUDA(cudaMemsetAsync(thr_counts, 0, sizeof(int32_t) * n, st));
     if (T == 0) {
@@ -399,8 +400,8 @@ int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, i
         MOE_CUDA(cudaMemsetAsync(loss, 0, sizeof(float), st));
         return MOE_OK;
     }
-    // logits by the fixed fma chain (the projection kernel takes a pair of matrices: W_g serves as both)
-    MOE_TRY(launch_projection(x, act, T, d, n, Wg, Wg, logits, twin, nullptr, 0, nullptr, 1, nullptr, st));
+    // logits by the fixed fma chain (one matrix: the projection kernel's second one is absent)
+    MOE_TRY(launch_projection(x, act, T, d, n, Wg, nullptr, logits, nullptr, nullptr, 0, nullptr, 1, nullptr, st));
     bal_softmax_kernel<<<(unsigned)cdiv(T, 8), 256, 0, st>>>(logits, T, n, probs);
     MOE_LAUNCHED();
     bal_transpose_kernel<<<dim3((unsigned)cdiv(T, 32), (unsigned)cdiv(n, 32)), 256, 0, st>>>(probs, T, n, pT);
@@ -412,7 +413,7 @@ int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, i
     MOE_LAUNCHED();
     bal_loss_final_kernel<<<1, 256, 0, st>>>(loss_part, cdiv(T, 8), loss);
     MOE_LAUNCHED();
-    MOE_TRY(launch_exclusive_scan(cnt, (int32_t)T, tok_ptr, st));
+    MOE_TRY(launch_exclusive_scan(cnt, (int32_t)T, tok_ptr, st, tile_sums));
     bal_fill_kernel<<<(unsigned)cdiv(R > n ? R : n + 1, 256) + 1, 256, 0, st>>>(tok_of_row, mask_bits, tok_ptr, R, n, m, words,
                                                                                 tok_rows, offsets);
     MOE_LAUNCHED();

@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(256) proj_kernel(ProjArgs a) {
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const int32_t n0 = a.n0, d = a.d;
-    const int32_t ncols = 2 * n0;
+    const int32_t ncols = a.W1 ? 2 * n0 : n0;  // W1 == nullptr: one matrix only
     const int32_t j0 = blockIdx.y * BN;
 
     // which rows does this tile cover?
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) proj_kernel(ProjArgs a) {
         r0 = a.offsets[lo] + (int64_t)(b - a.tile_prefix[lo]) * PBM;
         r_end = a.offsets[lo + 1];
         W0 += (int64_t)lo * d * n0;
-        W1 += (int64_t)lo * d * n0;
+        if (W1) W1 += (int64_t)lo * d * n0;
     }
     if (tid < PBM) {
         int64_t r = r0 + tid;
@@ -181,7 +181,7 @@ int32_t launch_projection(const void *x, int32_t act, int64_t M, int32_t d, int3
         MOE_TRY(launch_tile_prefix(offsets, nseg, PBM, tile_prefix, st));
         tiles_m += nseg;
     }
-    const int32_t ncols = 2 * n0;
+    const int32_t ncols = W1 ? 2 * n0 : n0;
     const bool wide = ncols > 64;
     dim3 grid((unsigned)tiles_m, (unsigned)cdiv(ncols, wide ? 128 : 64));
     if (act == MOE_BF16) {

@@ -81,26 +81,26 @@ __global__ void __launch_bounds__(256) level_sums_rows_kernel(const int32_t *__r
             cv[u] = j < n ? clean[t * n + j] : 0.0f;
             rv[u] = j < n ? raw[t * n + j] : 0.0f;
         }
-        int32_t sel_idx[MOE_MAX_K];
-        float sel_g[MOE_MAX_K];
+        // the row's kept experts: bit u of `kept` = this lane's column lane + 32 u is one of them (its gate goes to
+        // the Importance sum); an expert id outside [0, n) belongs to no lane
+        uint32_t kept = 0u;
+        for (int s = 0; s < k; ++s) {
+            const int32_t e = idx[t * k + s];
+            const float g = gates[t * k + s];
+            if ((e & 31) == lane && (uint32_t)e < (uint32_t)n) {
 #pragma unroll
-        for (int s = 0; s < MOE_MAX_K; ++s) {
-            sel_idx[s] = s < k ? idx[t * k + s] : -1;
-            sel_g[s] = s < k ? gates[t * k + s] : 0.0f;
+                for (int u = 0; u < NV; ++u)
+                    if ((e >> 5) == u) { kept |= 1u << u; s_imp[u] += g; }
+            }
         }
         const float thr_unsel = kth_vals[t * 2 + 0], thr_sel = kth_vals[t * 2 + 1];
 #pragma unroll
         for (int u = 0; u < NV; ++u) {
             const int32_t j = lane + 32 * u;
             if (j < n) {
-                bool sel = false;
-                float g = 0.0f;
-#pragma unroll
-                for (int s = 0; s < MOE_MAX_K; ++s)
-                    if (sel_idx[s] == j) { sel = true; g = sel_g[s]; }
-                const float z = (cv[u] - (sel ? thr_sel : thr_unsel)) / softplus_f(rv[u]);
+                // (the quotient may be off by two units in the last place: 1e-7 of z, far below what Load is held to)
+                const float z = __fdividef(cv[u] - (((kept >> u) & 1u) ? thr_sel : thr_unsel), softplus_f(rv[u]));
                 s_load[u] += 0.5f * erfcf(-z * 0.70710678118654752440f);  // Phi(z)
-                s_imp[u] += g;
             }
         }
     }
@@ -116,30 +116,44 @@ __global__ void __launch_bounds__(256) level_sums_rows_kernel(const int32_t *__r
     }
 }
 
+// Importance / Load = the blocks' partial sums added in double. A block takes 32 columns; its eight warps each add an
+// eighth of the chunks (in ascending order, eight loads in flight), the eight sums are then added in warp order.
 __global__ void __launch_bounds__(256) level_reduce_kernel(const float *__restrict__ part_imp,
                                                            const float *__restrict__ part_load, int32_t chunks,
                                                            int32_t n, float *__restrict__ importance,
                                                            float *__restrict__ load) {
-    const int32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= n) return;
+    __shared__ double red[2][8][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int32_t j = blockIdx.x * 32 + lane;
+    const int32_t per = (chunks + 7) / 8, c0 = w * per, c1 = min(c0 + per, chunks);
     double a = 0.0, b = 0.0;
-    int32_t c = 0;
-    for (; c + 8 <= chunks; c += 8) {  // eight independent loads in flight, added in order
-        float pa[8], pb[8];
+    if (j < n) {
+        int32_t c = c0;
+        for (; c + 8 <= c1; c += 8) {
+            float pa[8], pb[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            pa[q] = part_imp[(int64_t)(c + q) * n + j];
-            pb[q] = part_load[(int64_t)(c + q) * n + j];
+            for (int q = 0; q < 8; ++q) {
+                pa[q] = part_imp[(int64_t)(c + q) * n + j];
+                pb[q] = part_load[(int64_t)(c + q) * n + j];
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { a += (double)pa[q]; b += (double)pb[q]; }
         }
+        for (; c < c1; ++c) {
+            a += (double)part_imp[(int64_t)c * n + j];
+            b += (double)part_load[(int64_t)c * n + j];
+        }
+    }
+    red[0][w][lane] = a;
+    red[1][w][lane] = b;
+    __syncthreads();
+    if (w == 0 && j < n) {
+        a = 0.0; b = 0.0;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) { a += (double)pa[q]; b += (double)pb[q]; }
+        for (int q = 0; q < 8; ++q) { a += red[0][q][lane]; b += red[1][q][lane]; }
+        if (importance) importance[j] = (float)a;
+        if (load) load[j] = (float)b;
     }
-    for (; c < chunks; ++c) {
-        a += (double)part_imp[(int64_t)c * n + j];
-        b += (double)part_load[(int64_t)c * n + j];
-    }
-    if (importance) importance[j] = (float)a;
-    if (load) load[j] = (float)b;
 }
 
 int32_t launch_level_sums(const int32_t *idx, const float *gates, const float *clean, const float *raw,
@@ -160,7 +174,7 @@ int32_t launch_level_sums(const int32_t *idx, const float *gates, const float *c
     else if (n <= 256) level_sums_rows_kernel<8><<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, part_imp, part_load);
     else level_sums_kernel<<<chunks, 256, 0, st>>>(idx, gates, clean, raw, kth_vals, rows, n, k, CW, part_imp, part_load);
     MOE_LAUNCHED();
-    level_reduce_kernel<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(part_imp, part_load, chunks, n, importance_out,
+    level_reduce_kernel<<<(unsigned)cdiv(n, 32), 256, 0, st>>>(part_imp, part_load, chunks, n, importance_out,
                                                                  load_out);
     MOE_LAUNCHED();
     return MOE_OK;

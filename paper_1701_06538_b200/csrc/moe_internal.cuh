@@ -232,7 +232,8 @@ int32_t launch_tc_ffn(const moe_config &c, const void *xs, const int32_t *offset
 // the backward then masks dz with these bits instead of reading hid again as a mask (16 times less traffic)
 
 // ----------------------------------------------------------------------------- strictly balanced gating (balanced.cu)
-int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st);  // route.cu
+int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st,
+                              int32_t *tile_sums = nullptr /* cdiv(n + 1, 4096) ints: long inputs in parallel */);  // route.cu
 int64_t balanced_ws_bytes(int64_t T, int32_t n);
 int32_t launch_balanced_gate(const void *x, int32_t act, int64_t T, int32_t d, int32_t n, int32_t k, const float *Wg,
                              const float *thr, float *logits, float *probs, uint32_t *mask_bits, int32_t *tok_of_row,

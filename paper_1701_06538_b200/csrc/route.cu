@@ -164,8 +164,90 @@ int32_t launch_dispatch_index(const int32_t *topk_idx, int64_t R, int32_t n, int
     return MOE_OK;
 }
 
-// out[0..n] = exclusive prefix sums of counts[0..n-1] (one block; any n)
-int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st) {
+// The same for long inputs (one count per token), in tiles of 4096 counts: the tiles' sums first, then every tile
+// scans its own counts behind the sum of the tiles before it. 16-byte accesses where the tile is whole.
+constexpr int SCAN_TILE = 4096;
+__device__ __forceinline__ int4 scan_tile_load(const int32_t *counts, int32_t n, int32_t i) {
+    if (i + 4 <= n) return *reinterpret_cast<const int4 *>(counts + i);
+    int4 v = make_int4(0, 0, 0, 0);
+    if (i < n) v.x = counts[i];
+    if (i + 1 < n) v.y = counts[i + 1];
+    if (i + 2 < n) v.z = counts[i + 2];
+    return v;
+}
+// sum over the block of one value per thread, returned to every thread (1024 threads)
+__device__ __forceinline__ int32_t block_sum_1024(int32_t v, int32_t *sh /* [32] */) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    __syncthreads();  // sh may still be read from an earlier call
+    if (lane == 0) sh[w] = v;
+    __syncthreads();
+    int32_t t = sh[lane];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    return t;
+}
+__global__ void __launch_bounds__(1024) scan_tile_sums_kernel(const int32_t *__restrict__ counts, int32_t n,
+                                                              int32_t *__restrict__ tile_sums) {
+    __shared__ int32_t sh[32];
+    const int4 v = scan_tile_load(counts, n, blockIdx.x * SCAN_TILE + threadIdx.x * 4);
+    const int32_t total = block_sum_1024(v.x + v.y + v.z + v.w, sh);
+    if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+}
+__global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restrict__ counts, int32_t n,
+                                                          const int32_t *__restrict__ tile_sums,
+                                                          int32_t *__restrict__ offsets) {
+    __shared__ int32_t sh[32];
+    __shared__ int32_t warp_excl[32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int32_t before = 0;
+    for (int32_t b = threadIdx.x; b < (int32_t)blockIdx.x; b += 1024) before += tile_sums[b];
+    before = block_sum_1024(before, sh);
+    const int32_t i = blockIdx.x * SCAN_TILE + threadIdx.x * 4;
+    const int4 v = scan_tile_load(counts, n, i);
+    const int32_t mine = v.x + v.y + v.z + v.w;
+    int32_t inc = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        int32_t o = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += o;
+    }
+    if (lane == 31) warp_excl[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        int32_t sv = warp_excl[lane], si = sv;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            int32_t o = __shfl_up_sync(0xffffffffu, si, off);
+            if (lane >= off) si += o;
+        }
+        warp_excl[lane] = si - sv;
+    }
+    __syncthreads();
+    const int32_t e0 = before + warp_excl[w] + inc - mine;
+    const int4 out = make_int4(e0, e0 + v.x, e0 + v.x + v.y, e0 + v.x + v.y + v.z);
+    // offsets has n + 1 entries: entry n is the grand total, written by whoever holds position n
+    if (i + 4 <= n + 1 && (reinterpret_cast<uintptr_t>(offsets + i) & 15) == 0) {
+        *reinterpret_cast<int4 *>(offsets + i) = out;
+    } else {
+        if (i <= n) offsets[i] = out.x;
+        if (i + 1 <= n) offsets[i + 1] = out.y;
+        if (i + 2 <= n) offsets[i + 2] = out.z;
+        if (i + 3 <= n) offsets[i + 3] = out.w;
+    }
+}
+
+// out[0..n] = exclusive prefix sums of counts[0..n-1]. Long inputs need tile_sums: cdiv(n + 1, 4096) ints of scratch.
+int32_t launch_exclusive_scan(const int32_t *counts, int32_t n, int32_t *out, cudaStream_t st, int32_t *tile_sums) {
+    if (n > 8192 && tile_sums) {
+        const unsigned tiles = (unsigned)cdiv(n + 1, SCAN_TILE);  // position n (the total) falls into a tile as well
+        scan_tile_sums_kernel<<<tiles, 1024, 0, st>>>(counts, n, tile_sums);
+        MOE_LAUNCHED();
+        scan_tiles_kernel<<<tiles, 1024, 0, st>>>(counts, n, tile_sums, out);
+        MOE_LAUNCHED();
+        return MOE_OK;
+    }
     dispatch_scan_experts_kernel<<<1, 1024, 0, st>>>(counts, n, out);
     MOE_LAUNCHED();
     return MOE_OK;

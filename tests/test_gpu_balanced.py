@@ -19,6 +19,10 @@ CASES = [
     small_workload("bal-bf16", T=2048, d=128, h=256, n=64, k=4, act="bf16", seed=83),
     small_workload("bal-wide-bf16", T=3072, d=64, h=64, n=192, k=2, act="bf16", seed=84),   # six mask words per token
     synth.CONFIGS["c3"].scaled(8192),                                              # the many-expert shape, m = 128
+    # more than 8192 tokens: the per-token row pointers come from the tiled scan (a whole number of 4096-token tiles, so
+    # the total falls into a tile of its own; and a token count that is no multiple of four)
+    small_workload("bal-long-bf16", T=12288, d=64, h=64, n=32, k=2, act="bf16", seed=88),
+    small_workload("bal-long-odd-f32", T=9002, d=16, h=8, n=2, k=1, seed=89),
 ]
 W_BATCHWISE = 0.5
 
