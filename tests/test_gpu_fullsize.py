@@ -31,6 +31,7 @@ pytestmark = pytest.mark.gpu
 N_TOKENS = 48
 MAX_FLIP_RATE = 2e-5   # share of ReLU decisions that may differ (pre-activation within rounding of zero)
 UNITS_PER_TILE = 16    # hidden units of the largest expert sampled in every 256-wide tile
+DROP = 0.1             # DropProb of the layer epilogue check
 
 
 def slice_gate(G, rows):
@@ -86,6 +87,17 @@ def test_full_size_fused(name):
     hid, ys = O.expert_ffn(Ds.xs, Ds.offsets, W1, b1, W2, b2, "bf16")
     y = O.combine(ys, G.gates[toks], Ds.inv_perm, "bf16")
     assert_close(host(D["y"])[toks], y, TOL_BF16, "y (sampled tokens)")
+    # the layer epilogue (sigmoid, dropout, residual) at this size, through its stage calls on the saved context:
+    # the oracle evaluates the sampled tokens from scratch
+    keep_bits = synth.make_keep_bits(w, DROP)
+    keep = O.unpack_keep(keep_bits[toks], w.d)
+    out_d = torch.empty_like(D["y"])
+    kb_d = torch.from_numpy(keep_bits).cuda()
+    B.moe_combine_layer(cfg, V["ys"], V["gates"][:w.T * w.k], V["inv_perm"], D["x"], kb_d, DROP, out_d)
+    want_out = O.combine_layer(ys, G.gates[toks], Ds.inv_perm, x[toks], keep, DROP, "bf16")
+    assert_close(host(out_d)[toks], want_out, TOL_BF16, "layer output (sampled tokens)")
+    got_out = host(out_d)[toks]
+    assert (got_out[~keep] == np.asarray(x[toks], np.float32)[~keep]).all(), "a dropped activation leaves the residual alone"
     dg, dys = O.combine_bwd(dY[toks], ys, G.gates[toks], Ds.inv_perm, "bf16")
     E = O.expert_ffn_bwd(Ds.xs, hid, dys, Ds.offsets, W1, W2, "bf16")
     dX_exp = O.dispatch_bwd(E.dxs, Ds.inv_perm, len(toks), w.k, "bf16")
@@ -211,3 +223,85 @@ def test_full_size_repeated_steps_agree_bit_for_bit(name):
         if not torch.equal(first_ctx.view(torch.uint8), D["ctx"].view(torch.uint8)):
             differing.append("ctx")
         assert not differing, f"run {it + 1} differs from the first in {differing}"
+
+
+def test_full_size_balanced_gate():
+    """Strictly balanced gating at the bench's widest workload: logits, batchwise masks, row tables and per-token lists
+    bit for bit against the oracle (its gate handles the whole batch), probabilities, denominators and L_batchwise at the
+    gating tolerance, every expert with exactly m rows."""
+    w = synth.CONFIGS["c5"]
+    x, Wg = synth.make_x(w), synth.make_gate(w)[0]
+    logits, p = O.softmax_gate(x, Wg, "bf16")
+    m = w.T * w.k // w.n
+    srt = -np.sort(-np.asarray(p, np.float64), axis=0)
+    thr = (srt[m - 1] * (1 + 0.05 * np.random.default_rng(5).standard_normal(w.n))).astype(np.float32)
+    mask = O.batchwise_mask(p, m)
+    G_want, den = O.masked_gate(p, mask, "bf16")
+    Dw = O.dispatch_balanced(x, mask)
+    loss = O.batchwise_loss(p, mask, thr)
+    cfg = B.make_config(w.T, w.d, w.h, w.n, w.k, w.act, w.w_importance, w.w_load)
+    S = B.moe_query_balanced_sizes(cfg)
+    assert S.m == m
+    e = lambda *s_, dt=torch.float32: torch.empty(*s_, dtype=dt, device="cuda")
+    out = dict(logits=e(w.T, w.n), probs=e(w.T, w.n), mask_bits=e(w.T, S.mask_words, dt=torch.int32),
+               tok_of_row=e(S.R, dt=torch.int32), offsets=e(w.n + 1, dt=torch.int32), den=e(w.T),
+               tok_ptr=e(w.T + 1, dt=torch.int32), tok_rows=e(S.R, dt=torch.int32), loss=e(1),
+               thr_counts=e(w.n, dt=torch.int32), ws=B.empty_bytes(S.ws_bytes))
+    B.moe_gate_balanced(cfg, torch.from_numpy(x).to(torch.bfloat16).cuda(), torch.from_numpy(Wg).cuda(),
+                        torch.from_numpy(thr).cuda(), out["logits"], out["probs"], out["mask_bits"], out["tok_of_row"],
+                        out["offsets"], out["den"], out["tok_ptr"], out["tok_rows"], out["loss"], out["thr_counts"], out["ws"])
+    assert (host(out["logits"]) == np.asarray(logits)).all(), "logits by the fixed fma chain"
+    assert_close(host(out["probs"]), p, TOL_F32, "probs")
+    bits = np.packbits(mask, axis=1, bitorder="little")
+    assert (host(out["mask_bits"]).view(np.uint8).reshape(w.T, -1)[:, :bits.shape[1]] == bits).all(), "batchwise mask"
+    assert (host(out["offsets"]) == np.arange(w.n + 1) * m).all(), "every expert gets exactly m rows"
+    assert (host(out["tok_of_row"]) == Dw.tok_of_row).all()
+    ptr = np.zeros(w.T + 1, np.int64)
+    np.add.at(ptr, Dw.tok_of_row.astype(np.int64) + 1, 1)
+    assert (host(out["tok_ptr"]) == np.cumsum(ptr)).all()
+    assert (host(out["tok_rows"]) == np.lexsort((Dw.expert_of_row, Dw.tok_of_row))).all()
+    assert_close(host(out["den"]), den, TOL_F32, "den")
+    assert (host(out["thr_counts"]) == O.threshold_mask(p, thr).sum(axis=0)).all()
+    assert_close(host(out["loss"]), loss, TOL_F32, "L_batchwise")
+
+
+def test_full_size_factored_adam():
+    """The optimiser step on all 128 experts of the widest workload (2.1 GB of weights and as much of gradients); the
+    oracle steps three of them: the first, one in the middle, the last."""
+    w = synth.CONFIGS["c5"]
+    cfg = B.make_config(w.T, w.d, w.h, w.n, w.k, w.act, w.w_importance, w.w_load)
+    S = B.moe_query_sizes(cfg)
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    bf = torch.bfloat16
+    rnd = lambda *s_, scale=1.0: (torch.randn(*s_, device="cuda", generator=gen) * scale).to(bf)
+    W1, b1, W2, b2 = rnd(w.n, w.d, w.h, scale=0.03), rnd(w.n, w.h, scale=0.1), rnd(w.n, w.h, w.d, scale=0.02), rnd(w.n, w.d, scale=0.1)
+    # gradients with a row structure so that the factored estimate matters
+    g1 = (torch.randn(w.n, w.d, w.h, device="cuda", generator=gen) * (1 + 3 * torch.rand(w.n, w.d, 1, device="cuda", generator=gen))).to(bf)
+    g2 = (torch.randn(w.n, w.h, w.d, device="cuda", generator=gen) * (1 + 3 * torch.rand(w.n, w.h, 1, device="cuda", generator=gen))).to(bf)
+    gb1, gb2 = rnd(w.n, w.h), rnd(w.n, w.d)
+    state = torch.rand(S.adam_state_elems, device="cuda", generator=gen) + 0.5   # a running state, not the first step
+    picks = [0, w.n // 2, w.n - 1]
+    f = lambda t: t.float().cpu().numpy()
+    before = {e_: [f(a[e_]) for a in (W1, b1, W2, b2, g1, gb1, g2, gb2)] for e_ in picks}
+    st0 = f(state)
+    sizes = [("r1", w.d), ("c1", w.h), ("r2", w.h), ("c2", w.d), ("vb1", w.h), ("vb2", w.d)]
+    parts, at = {}, 0
+    for name, width in sizes:
+        parts[name] = st0[at:at + w.n * width].reshape(w.n, width)
+        at += w.n * width
+    lr, beta2, eps, step = 1e-2, 0.99, 1e-8, 7
+    B.moe_expert_adam_factored(cfg, W1, b1, W2, b2, g1, gb1, g2, gb2, state, lr, beta2, eps, step, B.empty_bytes(S.ws_adam_bytes))
+    torch.cuda.synchronize()
+    st1, at, got_parts = f(state), 0, {}
+    for name, width in sizes:
+        got_parts[name] = st1[at:at + w.n * width].reshape(w.n, width)
+        at += w.n * width
+    for e_ in picks:
+        a = before[e_]
+        one = {k_: v_[e_:e_ + 1] for k_, v_ in parts.items()}
+        want = O.expert_adam_factored(a[0][None], a[1][None], a[2][None], a[3][None], a[4][None], a[5][None], a[6][None],
+                                      a[7][None], one, lr, beta2, eps, step, "bf16")
+        for name, got, exp in zip(("W1", "b1", "W2", "b2"), (W1, b1, W2, b2), want[:4]):
+            assert_close(f(got[e_]), exp[0], TOL_BF16, f"{name} of expert {e_}")
+        for name, _ in sizes:
+            assert_close(got_parts[name][e_], np.asarray(want[4][name])[0], TOL_F32, f"state {name} of expert {e_}")
