@@ -628,8 +628,15 @@ __global__ void __launch_bounds__(256) gate_candidates_kernel(const float *__res
             screen_eval(c[j], r[j], e[j], xn, wn[j], wn[n + j], v, u);
             return v + u >= low;
         };
+        // one pass over the row: lane g keeps the ballot of the g-th group of 32 columns (rows wider than 1024
+        // columns are evaluated again when their entries are written)
         int total = 0;
-        for (int32_t j0 = 0; j0 < n; j0 += 32) total += __popc(__ballot_sync(0xffffffffu, candidate(j0 + lane)));
+        uint32_t kept_word = 0u;
+        for (int32_t j0 = 0; j0 < n; j0 += 32) {
+            const uint32_t b = __ballot_sync(0xffffffffu, candidate(j0 + lane));
+            if ((j0 >> 5) == lane) kept_word = b;
+            total += __popc(b);
+        }
         // (fewer than k + 1 candidates happens only with NaN logits, which are nobody's candidate)
         const bool few = total <= SCREEN_MAX_CAND && total >= min(k + 1, n);
         const int32_t wbase = group * 2 * n;  // this group's rows of the transposed weights
@@ -652,8 +659,9 @@ __global__ void __launch_bounds__(256) gate_candidates_kernel(const float *__res
         int pos = 0;
         for (int32_t j0 = 0; j0 < n; j0 += 32) {
             const int32_t j = j0 + lane;
-            const bool cand = candidate(j);
-            const uint32_t b = __ballot_sync(0xffffffffu, cand);
+            const uint32_t b = n <= 1024 ? __shfl_sync(0xffffffffu, kept_word, j0 >> 5)
+                                         : __ballot_sync(0xffffffffu, candidate(j));
+            const bool cand = (b >> lane) & 1u;
             if (cand) {
                 const int at = base + 2 * (pos + __popc(b & ((1u << lane) - 1u)));
                 chain_list[at] = make_int2((int32_t)row, wbase + j);
