@@ -1590,36 +1590,36 @@ static int32_t launch_tile_table(const int32_t *offsets, int32_t nseg, int32_t t
 }
 
 // Sum of the epilogue's 32-row column sums over each segment (bias gradient), G blocks per M tile.
-// A thread block takes 128 columns of one segment (a lane four adjacent ones, 16-byte loads); its 8 warps take the blocks
-// b = b0 + w, b0 + w + 8, ... and the 8 sums are added in warp order: the result does not depend on timing.
+// A thread block takes 64 columns of one segment: 16 column lanes (four adjacent columns each, 16-byte loads) by 16 row
+// lanes; row lane q takes the blocks b = b0 + q, b0 + q + 16, ... (eight loads in flight: the largest expert of a skewed
+// batch has over a thousand blocks and sets this kernel's duration) and the 16 sums are added in lane order: the
+// result does not depend on timing.
 __global__ void __launch_bounds__(256) colsum_blocks_final_kernel(const float *__restrict__ part, int32_t N,
                                                                   const int32_t *__restrict__ tile_prefix, int32_t G,
                                                                   bf16 *__restrict__ out) {
-    __shared__ float4 sh[8][32];
-    const int32_t e = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int32_t j = blockIdx.y * 128 + lane * 4;  // N is a multiple of 64
+    __shared__ float4 sh[16][16];
+    const int32_t e = blockIdx.x, q = threadIdx.x >> 4, cl = threadIdx.x & 15;
+    const int32_t j = blockIdx.y * 64 + cl * 4;  // N is a multiple of 64
     const int32_t b0 = tile_prefix[e] * G, b1 = tile_prefix[e + 1] * G;
     float4 s = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-    if (j < N) {
-        int32_t b = b0 + w;
-        for (; b + 24 < b1; b += 32) {
-            float4 v[4];
+    int32_t b = b0 + q;
+    for (; b + 16 * 7 < b1; b += 16 * 8) {
+        float4 v[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4 *>(part + (int64_t)(b + 8 * u) * N + j);
+        for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const float4 *>(part + (int64_t)(b + 16 * u) * N + j);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
-        }
-        for (; b < b1; b += 8) {
-            const float4 v = *reinterpret_cast<const float4 *>(part + (int64_t)b * N + j);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-        }
+        for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
     }
-    sh[w][lane] = s;
+    for (; b < b1; b += 16) {
+        const float4 v = *reinterpret_cast<const float4 *>(part + (int64_t)b * N + j);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    sh[q][cl] = s;
     __syncthreads();
-    if (w == 0 && j < N) {
-        float4 t = sh[0][lane];
+    if (q == 0) {
+        float4 t = sh[0][cl];
 #pragma unroll
-        for (int u = 1; u < 8; ++u) { t.x += sh[u][lane].x; t.y += sh[u][lane].y; t.z += sh[u][lane].z; t.w += sh[u][lane].w; }
+        for (int u = 1; u < 16; ++u) { t.x += sh[u][cl].x; t.y += sh[u][cl].y; t.z += sh[u][cl].z; t.w += sh[u][cl].w; }
         __nv_bfloat162 o0 = __floats2bfloat162_rn(t.x, t.y), o1 = __floats2bfloat162_rn(t.z, t.w);
         uint2 pk;
         pk.x = *reinterpret_cast<uint32_t *>(&o0); pk.y = *reinterpret_cast<uint32_t *>(&o1);
@@ -1642,7 +1642,7 @@ int32_t tc_row_gemm(const void *A, const void *W, bool transposed, const int32_t
     }
     auto finish = [&](int32_t rc, int32_t G) -> int32_t {
         if (rc != MOE_OK || !colsum_out) return rc;
-        colsum_blocks_final_kernel<<<dim3((unsigned)nseg, (unsigned)cdiv(N, 128)), 256, 0, st>>>(colsum_part, N, tile_prefix, G,
+        colsum_blocks_final_kernel<<<dim3((unsigned)nseg, (unsigned)cdiv(N, 64)), 256, 0, st>>>(colsum_part, N, tile_prefix, G,
                                                                                                    (bf16 *)colsum_out);
         MOE_LAUNCHED();
         return MOE_OK;

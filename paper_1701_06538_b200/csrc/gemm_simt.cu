@@ -213,16 +213,36 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const XT *__restric
     }
 }
 
+// Sum of a segment's tile sums: a block takes 32 columns, its eight warps the tiles b0 + w, b0 + w + 8, ... (eight loads in
+// flight: the largest expert of a skewed batch has hundreds of tiles), the eight sums are added in warp order.
 template <typename XT>
 __global__ void __launch_bounds__(256) colsum_final_kernel(const float *__restrict__ part, int32_t N,
                                                            const int32_t *__restrict__ tile_prefix,
                                                            XT *__restrict__ out) {
-    const int32_t e = blockIdx.x;
-    const int32_t j = blockIdx.y * 256 + threadIdx.x;
-    if (j >= N) return;
+    __shared__ float sh[8][32];
+    const int32_t e = blockIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int32_t j = blockIdx.y * 32 + lane;
+    const int32_t b1 = tile_prefix[e + 1];
     float s = 0.0f;
-    for (int32_t b = tile_prefix[e]; b < tile_prefix[e + 1]; ++b) s += part[(int64_t)b * N + j];
-    out[(int64_t)e * N + j] = from_f32<XT>(s);
+    if (j < N) {
+        int32_t b = tile_prefix[e] + w;
+        for (; b + 8 * 7 < b1; b += 64) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = part[(int64_t)(b + 8 * u) * N + j];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += v[u];
+        }
+        for (; b < b1; b += 8) s += part[(int64_t)b * N + j];
+    }
+    sh[w][lane] = s;
+    __syncthreads();
+    if (w == 0 && j < N) {
+        float t = sh[0][lane];
+#pragma unroll
+        for (int u = 1; u < 8; ++u) t += sh[u][lane];
+        out[(int64_t)e * N + j] = from_f32<XT>(t);
+    }
 }
 
 int32_t launch_segment_colsum(const void *in, int32_t act, const int32_t *offsets, int32_t nseg, int64_t R,
@@ -230,7 +250,7 @@ int32_t launch_segment_colsum(const void *in, int32_t act, const int32_t *offset
     MOE_TRY(launch_tile_prefix(offsets, nseg, CS_ROWS, tile_prefix, st));
     const int vcols = act == MOE_BF16 ? 256 : 128;  // columns per block of the partial sums: 32 lanes x one 16-byte vector
     dim3 g1((unsigned)(cdiv(R, CS_ROWS) + nseg), (unsigned)cdiv(N, vcols));
-    dim3 g2((unsigned)nseg, (unsigned)cdiv(N, 256));
+    dim3 g2((unsigned)nseg, (unsigned)cdiv(N, 32));
     if (act == MOE_BF16) {
         colsum_partial_kernel<bf16><<<g1, 256, 0, st>>>((const bf16 *)in, offsets, nseg, N, tile_prefix, scratch);
         MOE_LAUNCHED();
