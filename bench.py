@@ -312,14 +312,15 @@ def run_ours(args, w):
     launches = per_step * args.steps if graph else B.moe_debug_launch_count() - l0
 
     # end to end: every step copies its inputs (x, noise, dY) from pinned host memory and copies its results
-    # (y, dX, losses) back, all inside the timed region. Three streams and two sets of device buffers let the
+    # (y, dX, losses) back, all inside the timed region. Three streams and three sets of device buffers let the
     # copies of neighbouring steps overlap the kernels of the current one; the kernels themselves are the
     # same calls in the same order as in the device-resident measurement.
     hx, hdY = torch.from_numpy(host["x"]).to(D["x"].dtype).pin_memory(), torch.from_numpy(host["dY"]).to(D["x"].dtype).pin_memory()
     hnoise = D["noise"].cpu().pin_memory()
     hy, hdX, hl = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory(), torch.empty(2).pin_memory()
+    NSETS = 3  # with two, the 0.6 GB of inputs of step i + 2 had one step's time to arrive: as long as the copy itself
     bufs = [{k: (D[k] if b == 0 else torch.empty_like(D[k])) for k in ("x", "noise", "dY", "y", "dX", "losses")}
-            for b in range(2)]
+            for b in range(NSETS)]
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
     def run_e2e(K):
@@ -333,18 +334,18 @@ def run_ours(args, w):
         with torch.cuda.stream(s_in):
             t0.record()
         for i in range(K):
-            Bf = bufs[i & 1]
+            Bf = bufs[i % NSETS]
             with torch.cuda.stream(s_in):
-                if i >= 2:
-                    s_in.wait_event(ev_comp[i - 2])  # the kernels that read this input set are done
+                if i >= NSETS:
+                    s_in.wait_event(ev_comp[i - NSETS])  # the kernels that read this input set are done
                 Bf["x"].copy_(hx, non_blocking=True); Bf["noise"].copy_(hnoise, non_blocking=True)
                 ev_in_f[i].record()
                 Bf["dY"].copy_(hdY, non_blocking=True)  # only the backward needs it: it arrives during the forward
                 ev_in_b[i].record()
             with torch.cuda.stream(s_comp):
                 s_comp.wait_event(ev_in_f[i])
-                if i >= 2:
-                    s_comp.wait_event(ev_out[i - 2])  # this output set has been copied out
+                if i >= NSETS:
+                    s_comp.wait_event(ev_out[i - NSETS])  # this output set has been copied out
                 B.moe_forward(cfg, Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
                               Bf["y"], Bf["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
                 ev_fwd[i].record()
