@@ -22,7 +22,7 @@ def pytest_collection_modifyitems(config, items):
 
 def pytest_sessionfinish(session, exitstatus):
     """When the session ran on the checking build of the library (MOE_B200_LIB points at it), no kernel may have
-    seen an index outside its range: the count is part of the verdict."""
+    seen an index outside its range: the count is part of the result."""
     if not os.environ.get("MOE_B200_LIB"):
         return
     from paper_1701_06538_b200 import binding as B
