@@ -324,6 +324,28 @@ def run_ours(args, w):
             for b in range(NSETS)]
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
+    def e2e_fwd(Bf):
+        B.moe_forward(cfg, Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
+                      Bf["y"], Bf["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+
+    def e2e_bwd(Bf):
+        B.moe_backward(cfg, Bf["dY"], Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"],
+                       D["b2"], D["ctx"], Bf["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"],
+                       D["db2"], D["ws"])
+
+    # the two calls of a step as one graph each per buffer set (the copies and the events between them stay outside)
+    e2e_graphs = None
+    if graph is not None:
+        e2e_graphs = []
+        for Bf in bufs:
+            gf, gb = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gf, stream=s_comp):
+                e2e_fwd(Bf)
+            with torch.cuda.graph(gb, stream=s_comp):
+                e2e_bwd(Bf)
+            e2e_graphs.append((gf, gb))
+        torch.cuda.synchronize()
+
     def run_e2e(K):
         ev_in_f = [torch.cuda.Event() for _ in range(K)]   # x and noise of step i are on the device
         ev_in_b = [torch.cuda.Event() for _ in range(K)]   # dY too
@@ -347,13 +369,12 @@ def run_ours(args, w):
                 s_comp.wait_event(ev_in_f[i])
                 if i >= NSETS:
                     s_comp.wait_event(ev_out[i - NSETS])  # this output set has been copied out
-                B.moe_forward(cfg, Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"], D["b2"],
-                              Bf["y"], Bf["losses"], D["importance"], D["load"], D["counts"], D["ctx"], D["ws"])
+                if e2e_graphs: e2e_graphs[i % NSETS][0].replay()
+                else: e2e_fwd(Bf)
                 ev_fwd[i].record()
                 s_comp.wait_event(ev_in_b[i])
-                B.moe_backward(cfg, Bf["dY"], Bf["x"], D["Wg"], D["Wnoise"], Bf["noise"], D["W1"], D["b1"], D["W2"],
-                               D["b2"], D["ctx"], Bf["dX"], D["dWg"], D["dWnoise"], D["dW1"], D["db1"], D["dW2"],
-                               D["db2"], D["ws"])
+                if e2e_graphs: e2e_graphs[i % NSETS][1].replay()
+                else: e2e_bwd(Bf)
                 ev_comp[i].record()
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_fwd[i])  # y and the losses leave while the backward runs
