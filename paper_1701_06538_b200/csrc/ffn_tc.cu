@@ -905,9 +905,12 @@ __global__ void __launch_bounds__(NTHREADS2, 1)
 grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmM, const __grid_constant__ CUtensorMap tmO,
                      const GemmParams p) {
-    // ROW_*: 5 stages and a 64 KiB region of four [128 rows][64 columns] blocks (128-byte swizzle) that holds the
-    // ReLU-mask tile (MASKT) and stages the bf16 output for bulk tensor stores; WGRAD: 6 stages + 32 KiB of staging
-    constexpr int NST = KIND == WGRAD ? 6 : 5;
+    // ROW_* with a mask tile: 5 stages and a 64 KiB region of four [128 rows][64 columns] blocks (128-byte swizzle) that
+    // holds the ReLU-mask tile and stages the bf16 output for bulk tensor stores; every other kind: 6 stages + 32 KiB of
+    // staging (row GEMMs: two such blocks, a warp's two output boxes of a tile pass through the same 4 KiB one after
+    // the other; the sixth stage took a seventh off the time the MMA thread waited for operands at 16 K blocks per tile)
+    constexpr int NST = (KIND == WGRAD || !MASKT) ? 6 : 5;  // the mask tile needs the 64 KiB region, everything else 32 KiB
+    constexpr bool ONE_BOX = KIND != WGRAD && !MASKT;       // row GEMM without a mask tile: one staging box per warp
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - smem_u32(smem_raw));
@@ -1266,7 +1269,13 @@ grouped_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (p.bits_out && row_ok) p.bits_out[out_row * (p.N >> 5) + (col0 >> 5)] = positive_bits(packed);
                     tr_pack += TILE_CLOCK() - tp0;
                     if (staged) {
-                        uint8_t *blk = smem + NST * STAGE2_BYTES + (c >> 1) * 16384;
+                        // with one box per warp (two [128][64] blocks, one per column half) the second box of a tile
+                        // goes where the first one was: its bulk store must have read the box out first
+                        uint8_t *blk = smem + NST * STAGE2_BYTES + (ONE_BOX ? half : (c >> 1)) * 16384;
+                        if (ONE_BOX && (c & 3) == 2) {
+                            if (lane == 0) tma_store_wait_read();
+                            __syncwarp();
+                        }
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
                             *reinterpret_cast<uint4 *>(blk + mrow * 128 + ((((c & 1) * 4 + q) ^ (mrow & 7)) << 4)) = packed[q];
